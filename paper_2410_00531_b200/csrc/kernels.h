@@ -1,0 +1,99 @@
+// Host-side launchers of the CUDA kernels (internal to the library).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace tpi {
+
+struct LaunchCtx {
+  cudaStream_t stream = nullptr;
+  bool pdl = false;        // programmatic dependent launch between consecutive kernels
+  int* launches = nullptr; // counter of kernels launched (may be null)
+};
+
+enum { DT_F32 = 0, DT_BF16 = 1 };
+// codes written to the device error word by kernel self-checks (the host reads it after a step)
+enum : int { DEVERR_NONE = 0, DEVERR_TOKEN_RANGE = 1, DEVERR_POS_RANGE = 2, DEVERR_WAIT_TIMEOUT = 3 };
+static inline size_t dt_size(int dt) { return dt == DT_BF16 ? 2 : 4; }
+
+// ---------------------------------------------------------------- decode (one position)
+// x = W_emb[tok_hist[*pos]] (fp32); xhat = x * rsqrt(mean(x^2) + eps).
+cudaError_t launch_embed(const LaunchCtx& c, int dt, const void* emb, const int* tok_hist,
+                         const int* pos, int vocab, int max_seq, int h, float eps, float* x,
+                         float* xhat, int* err);
+
+// Column-sharded QKV GEMV with fused rotary embedding and KV-cache append (Eq. 1 inputs).
+// Wqkv: shard-major [(a/N + 2b/N) d][h] per shard.  q_out fp32 [a d] (rotated, unscaled).
+cudaError_t launch_gemv_qkv(const LaunchCtx& c, int dt, const void* Wqkv, size_t shard_stride_elems,
+                            const float* xhat, const float* gain, int h, int n_shards, int a, int b,
+                            int d, int max_seq, const int* pos, const float2* rope, float* q_out,
+                            void* kcache_layer, void* vcache_layer);
+
+// Column-sharded gate/up GEMV (rows interleaved gate_j, up_j) with SwiGLU epilogue (Eq. 2).
+cudaError_t launch_gemv_gateup(const LaunchCtx& c, int dt, const void* Wgu, size_t shard_stride_elems,
+                               const float* xhat, const float* gain, int h, int n_shards, int s,
+                               float* act);
+
+// Row-sharded GEMV: partials[i][r] = W^i[r, :] . x[i*Ks : (i+1)*Ks]   (per-device partial sums).
+cudaError_t launch_gemv_partials(const LaunchCtx& c, int dt, const void* W, size_t shard_stride_elems,
+                                 const float* x, int rows, int Ks, int n_shards, float* partials);
+
+// The emulated star allreduce + shortcut + the next block's norm statistics:
+// x <- ((P_0 + P_1) + ... + P_{N-1}) + x ; xhat = x * rsqrt(mean(x^2) + eps); tap (may be null) <- x.
+cudaError_t launch_reduce_residual(const LaunchCtx& c, const float* partials, int n_shards, int h,
+                                   float eps, float* x, float* xhat, float* tap);
+
+// Split-K attention of one query position over the cache (Eq. 1), grouped heads.
+// scratch: float[b * nsplit * (a/b) * (d + 2)], tickets: unsigned[b] (zero between launches).
+cudaError_t launch_decode_attention(const LaunchCtx& c, int dt, const float* q, const void* kcache_layer,
+                                    const void* vcache_layer, const int* pos, int a, int b, int d,
+                                    int max_seq, int nsplit, float* scratch, unsigned* tickets,
+                                    float* o);
+size_t decode_attention_scratch_floats(int a, int b, int d, int nsplit);
+
+// Task head (Step 4): logits = W_head . (xhat * gain), greedy argmax (lowest index on ties);
+// writes tok_hist[*pos + 1] and advances *pos.  amax scratch: >= grid blocks entries.
+cudaError_t launch_head_argmax(const LaunchCtx& c, int dt, const void* Whead, const float* xhat,
+                               const float* gain, int h, int vocab, float* logits, float* amax_val,
+                               int* amax_idx, unsigned* ticket, int* tok_hist, int* pos, int advance);
+int head_argmax_blocks(int vocab);
+
+// cos/sin table for positions [0, max_seq): table[p][i] = (cos, sin)(p * inv_freq[i]), fp64 inside.
+cudaError_t launch_rope_table(const LaunchCtx& c, const double* inv_freq, int max_seq, int half,
+                              float2* table);
+
+// ---------------------------------------------------------------- prefill (T positions)
+cudaError_t launch_embed_rows(const LaunchCtx& c, int dt, const void* emb, const int* tok_hist, int pos0,
+                              int T, int vocab, int h, float* X, int* err);
+// Xn[t] = X[t] * rsqrt(mean + eps) * gain   (Xn fp32, or bf16 when out_bf16)
+cudaError_t launch_rmsnorm_rows(const LaunchCtx& c, const float* X, const float* gain, int T, int h,
+                                float eps, void* Xn, int out_bf16);
+// Y[t][o] = sum_k X[t][k] W[o][k] for a batch of `n_batch` independent problems
+// (batch = shard for the row-sharded projections).  X fp32, row stride ldx; Y fp32, row stride ldy.
+cudaError_t launch_gemm_simt(const LaunchCtx& c, int dt, const float* X, long long x_batch_stride, int ldx,
+                             const void* W, long long w_batch_stride_elems, float* Y,
+                             long long y_batch_stride, int ldy, int T, int n_out, int K, int n_batch);
+// rotate q and k of T positions, append k, v to the cache. QKV rows: [shard][q | k | v] packed as the GEMV.
+cudaError_t launch_rope_kv_rows(const LaunchCtx& c, int dt, const float* QKV, int T, int pos0, int n_shards,
+                                int a, int b, int d, int max_seq, const float2* rope, float* Q,
+                                void* kcache_layer, void* vcache_layer);
+// causal attention of T query positions [pos0, pos0+T) over cache positions [0, pos0+T)
+cudaError_t launch_prefill_attention(const LaunchCtx& c, int dt, const float* Q, const void* kcache_layer,
+                                     const void* vcache_layer, int T, int pos0, int a, int b, int d,
+                                     int max_seq, float* O);
+// act[t][j] = silu(GU[t][2j]) * GU[t][2j+1] per shard-major interleaved rows
+cudaError_t launch_swiglu_rows(const LaunchCtx& c, const float* GU, int T, int s, float* ACT);
+// X[t] <- sum_i P_i[t] + X[t]; optional tap of the last row
+cudaError_t launch_reduce_residual_rows(const LaunchCtx& c, const float* partials, int n_shards, int T,
+                                        int h, float* X, float* tap_last);
+// xhat of one row of X (to hand the last position to the decode-style head)
+// (also sets *pos = pos_value when pos is not null)
+cudaError_t launch_rmsnorm_stat_row(const LaunchCtx& c, const float* xrow, int h, float eps, float* x,
+                                    float* xhat, int* pos, int pos_value);
+
+// misc
+cudaError_t launch_fill_u32(const LaunchCtx& c, uint32_t* p, size_t n, uint32_t v);
+cudaError_t launch_kv_convert(const LaunchCtx& c, int dt, void* cache_rows, float* f32_rows, size_t n,
+                              int to_float);
+
+}  // namespace tpi

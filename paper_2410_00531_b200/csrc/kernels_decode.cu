@@ -1,0 +1,612 @@
+// Decode-step kernels (one position, batch 1): weight-streaming GEMVs with
+// fused epilogues, the emulated star allreduce, split-K attention, task head.
+//
+// All of them are HBM-bound on the weight (or KV) bytes: 16-byte streaming
+// loads, many in flight per lane, activations staged in shared memory, warp
+// shuffle reductions, and an L2 bulk prefetch of each CTA's weight rows issued
+// BEFORE the programmatic-dependent-launch wait so that the weight stream of
+// kernel k+1 starts while kernel k (often a one-CTA reduction) is still running.
+#include "common.cuh"
+#include "kernels.h"
+#include "launch.cuh"
+
+namespace tpi {
+
+// =====================================================================================
+// GEMV family
+// =====================================================================================
+enum { EPI_QKV = 0, EPI_SWIGLU = 1, EPI_PARTIAL = 2, EPI_LOGITS = 3 };
+
+struct GemvArgs {
+  const void* W;              // shard 0's matrix, [rows][K] row-major
+  long long shard_stride;     // elements between consecutive shards' matrices
+  const float* x;             // input vector (fp32)
+  int x_shard_stride;         // 0: every shard reads the same x; Ks: shard i reads x + i*Ks
+  const float* gain;          // optional per-element gain applied while staging x (norm gain)
+  int K;                      // dot length
+  int kc;                     // shared-memory chunk of K in floats (multiple of 8)
+  int items_per_shard;        // warp work items per shard
+  int n_shards;
+  float* out;
+  long long out_shard_stride;
+  // EPI_QKV
+  void* kcache;
+  void* vcache;
+  const int* pos;
+  const float2* rope;
+  int hps, kps, d, max_seq;   // q heads per shard, kv heads per shard, head dim
+  // EPI_LOGITS
+  float* amax_val;
+  int* amax_idx;
+  unsigned* ticket;
+  int* tok_hist;
+  int* pos_rw;
+  int rows_total;
+  int advance;
+};
+
+template <int EPI, int R>
+__device__ __forceinline__ void item_rows(const GemvArgs& A, int item, int (&rows)[R]) {
+  if constexpr (EPI == EPI_QKV) {
+    static_assert(R == 2, "qkv items are row pairs");
+    const int half = A.d >> 1;
+    const int qp = A.hps * half, kp = A.kps * half;
+    if (item < qp + kp) {  // rotary pair (i, i + d/2) of one q or k head
+      const int hl = item / half, ii = item - hl * half;
+      rows[0] = hl * A.d + ii;
+      rows[1] = rows[0] + half;
+    } else {  // two adjacent v rows
+      const int t = item - qp - kp;
+      rows[0] = (A.hps + A.kps) * A.d + 2 * t;
+      rows[1] = rows[0] + 1;
+    }
+  } else {
+#pragma unroll
+    for (int r = 0; r < R; ++r) rows[r] = item * R + r;
+  }
+}
+
+template <typename WT, int R, int EPI, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32) gemv_kernel(const GemvArgs A) {
+  extern __shared__ __align__(16) float xs[];
+  constexpr int VEC = Elem<WT>::VEC;
+  constexpr int U = 4;  // 16-byte loads in flight per row per lane
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int bps = (A.items_per_shard + WARPS - 1) / WARPS;
+  const int shard = blockIdx.x / bps;
+  const int item = (blockIdx.x - shard * bps) * WARPS + warp;
+  const bool valid = item < A.items_per_shard;
+
+  int rows[R];
+  item_rows<EPI, R>(A, valid ? item : 0, rows);
+  const WT* Wsh = reinterpret_cast<const WT*>(A.W) + (size_t)shard * A.shard_stride;
+  const uint4* wp[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) wp[r] = reinterpret_cast<const uint4*>(Wsh + (size_t)rows[r] * A.K);
+
+  // Weights do not depend on the previous kernel: start pulling them into L2 now.
+  if (valid && lane == 0) {
+    const uint32_t row_bytes = (uint32_t)(A.K * sizeof(WT));
+#pragma unroll
+    for (int r = 0; r < R; ++r) l2_prefetch_bulk(wp[r], row_bytes);
+  }
+  pdl_launch_dependents();
+  pdl_wait();  // the activation vector is written by the previous kernel
+
+  float acc[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) acc[r] = 0.f;
+
+  const float* xg = A.x + (size_t)shard * A.x_shard_stride;
+  for (int k0 = 0; k0 < A.K; k0 += A.kc) {
+    const int kc = min(A.kc, A.K - k0);
+    if (k0) __syncthreads();
+    for (int k = threadIdx.x * 4; k < kc; k += WARPS * 32 * 4) {
+      float4 v = *reinterpret_cast<const float4*>(xg + k0 + k);
+      if (A.gain) {
+        const float4 g = *reinterpret_cast<const float4*>(A.gain + k0 + k);
+        v.x *= g.x; v.y *= g.y; v.z *= g.z; v.w *= g.w;
+      }
+      *reinterpret_cast<float4*>(xs + k) = v;
+    }
+    __syncthreads();
+    if (valid) {
+      const int v0 = k0 / VEC, nvec = kc / VEC;
+      int v = lane;
+      for (; v + 32 * (U - 1) < nvec; v += 32 * U) {
+        uint4 w[U][R];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+          for (int r = 0; r < R; ++r) w[u][r] = ldg_stream16(wp[r] + v0 + v + 32 * u);
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+          for (int r = 0; r < R; ++r) acc[r] = Elem<WT>::dot(w[u][r], xs + (v + 32 * u) * VEC, acc[r]);
+      }
+      for (; v < nvec; v += 32) {
+        uint4 w[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) w[r] = ldg_stream16(wp[r] + v0 + v);
+#pragma unroll
+        for (int r = 0; r < R; ++r) acc[r] = Elem<WT>::dot(w[r], xs + v * VEC, acc[r]);
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < R; ++r) acc[r] = warp_sum(acc[r]);
+
+  // ---------------------------------------------------------------- epilogues
+  if constexpr (EPI == EPI_QKV) {
+    if (valid && lane == 0) {
+      const int half = A.d >> 1;
+      const int qp = A.hps * half, kp = A.kps * half;
+      const int p = *A.pos;
+      if (item < qp + kp) {
+        const bool is_q = item < qp;
+        const int t = is_q ? item : item - qp;
+        const int hl = t / half, ii = t - hl * half;
+        const float2 cs = A.rope[(size_t)p * half + ii];
+        const float lo = acc[0] * cs.x - acc[1] * cs.y;
+        const float hi = acc[1] * cs.x + acc[0] * cs.y;
+        if (is_q) {
+          float* q = A.out + (size_t)(shard * A.hps + hl) * A.d;
+          q[ii] = lo;
+          q[ii + half] = hi;
+        } else {
+          WT* kr = reinterpret_cast<WT*>(A.kcache) + ((size_t)(shard * A.kps + hl) * A.max_seq + p) * A.d;
+          Elem<WT>::store(kr + ii, lo);
+          Elem<WT>::store(kr + ii + half, hi);
+        }
+      } else {
+        const int t2 = 2 * (item - qp - kp);
+        const int hl = t2 / A.d, idx = t2 - hl * A.d;
+        WT* vr = reinterpret_cast<WT*>(A.vcache) + ((size_t)(shard * A.kps + hl) * A.max_seq + p) * A.d;
+        Elem<WT>::store(vr + idx, acc[0]);
+        Elem<WT>::store(vr + idx + 1, acc[1]);
+      }
+    }
+  } else if constexpr (EPI == EPI_SWIGLU) {
+    if (valid && lane == 0) {
+      const float g = acc[0], u = acc[1];
+      A.out[(size_t)shard * A.out_shard_stride + item] = g / (1.f + expf(-g)) * u;
+    }
+  } else if constexpr (EPI == EPI_PARTIAL) {
+    if (valid && lane == 0) {
+      float* o = A.out + (size_t)shard * A.out_shard_stride + (size_t)item * R;
+#pragma unroll
+      for (int r = 0; r < R; ++r) o[r] = acc[r];
+    }
+  } else {  // EPI_LOGITS: write logits, then a grid-wide argmax with lowest index on ties
+    __shared__ float s_val[WARPS];
+    __shared__ int s_idx[WARPS];
+    __shared__ bool s_last;
+    float bv = -INFINITY;
+    int bi = 0x7FFFFFFF;
+    if (valid && lane == 0) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        A.out[(size_t)item * R + r] = acc[r];
+        if (acc[r] > bv) { bv = acc[r]; bi = item * R + r; }
+      }
+    }
+    if (lane == 0) { s_val[warp] = bv; s_idx[warp] = bi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int w = 1; w < WARPS; ++w)
+        if (s_val[w] > bv || (s_val[w] == bv && s_idx[w] < bi)) { bv = s_val[w]; bi = s_idx[w]; }
+      A.amax_val[blockIdx.x] = bv;
+      A.amax_idx[blockIdx.x] = bi;
+      __threadfence();
+      const unsigned t = atomicAdd(A.ticket, 1u);
+      s_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (s_last && warp == 0) {
+      __threadfence();
+      bv = -INFINITY;
+      bi = 0x7FFFFFFF;
+      for (int b = lane; b < (int)gridDim.x; b += 32) {
+        const float v = __ldcg(A.amax_val + b);
+        const int i = __ldcg(A.amax_idx + b);
+        if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float v = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
+        const int i = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
+        if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+      }
+      if (lane == 0) {
+        const int p = *A.pos_rw;
+        A.tok_hist[p + 1] = bi;  // the token to feed at the next position
+        if (A.advance) *A.pos_rw = p + 1;
+        *A.ticket = 0u;
+      }
+    }
+  }
+}
+
+static int pick_kc(int K) {
+  // whole vector in shared memory up to 64 KiB, else chunks of 16384 floats
+  return K <= 16384 ? K : 16384;
+}
+
+template <typename WT, int R, int EPI>
+static cudaError_t launch_gemv_t(const LaunchCtx& c, GemvArgs& A) {
+  constexpr int WARPS = 8;
+  A.kc = pick_kc(A.K);
+  const int bps = (A.items_per_shard + WARPS - 1) / WARPS;
+  const size_t smem = (size_t)A.kc * sizeof(float);
+  auto kern = gemv_kernel<WT, R, EPI, WARPS>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  return launch_kernel(c, kern, dim3((unsigned)(bps * A.n_shards)), dim3(WARPS * 32), smem, A);
+}
+
+cudaError_t launch_gemv_qkv(const LaunchCtx& c, int dt, const void* Wqkv, size_t shard_stride_elems,
+                            const float* xhat, const float* gain, int h, int n_shards, int a, int b,
+                            int d, int max_seq, const int* pos, const float2* rope, float* q_out,
+                            void* kcache_layer, void* vcache_layer) {
+  GemvArgs A{};
+  A.W = Wqkv; A.shard_stride = (long long)shard_stride_elems; A.x = xhat; A.x_shard_stride = 0;
+  A.gain = gain; A.K = h; A.n_shards = n_shards;
+  A.hps = a / n_shards; A.kps = b / n_shards; A.d = d; A.max_seq = max_seq;
+  A.items_per_shard = (A.hps + 2 * A.kps) * (d / 2);
+  A.out = q_out; A.kcache = kcache_layer; A.vcache = vcache_layer; A.pos = pos; A.rope = rope;
+  return dt == DT_BF16 ? launch_gemv_t<__nv_bfloat16, 2, EPI_QKV>(c, A) : launch_gemv_t<float, 2, EPI_QKV>(c, A);
+}
+
+cudaError_t launch_gemv_gateup(const LaunchCtx& c, int dt, const void* Wgu, size_t shard_stride_elems,
+                               const float* xhat, const float* gain, int h, int n_shards, int s,
+                               float* act) {
+  GemvArgs A{};
+  A.W = Wgu; A.shard_stride = (long long)shard_stride_elems; A.x = xhat; A.x_shard_stride = 0;
+  A.gain = gain; A.K = h; A.n_shards = n_shards; A.items_per_shard = s / n_shards;
+  A.out = act; A.out_shard_stride = s / n_shards;
+  return dt == DT_BF16 ? launch_gemv_t<__nv_bfloat16, 2, EPI_SWIGLU>(c, A)
+                       : launch_gemv_t<float, 2, EPI_SWIGLU>(c, A);
+}
+
+cudaError_t launch_gemv_partials(const LaunchCtx& c, int dt, const void* W, size_t shard_stride_elems,
+                                 const float* x, int rows, int Ks, int n_shards, float* partials) {
+  GemvArgs A{};
+  A.W = W; A.shard_stride = (long long)shard_stride_elems; A.x = x; A.x_shard_stride = Ks;
+  A.gain = nullptr; A.K = Ks; A.n_shards = n_shards; A.out = partials; A.out_shard_stride = rows;
+  // rows per warp: keep >= ~8 KiB of weights per warp so that loads stay in flight
+  const size_t row_bytes = (size_t)Ks * dt_size(dt);
+  int R = 2;
+  if (row_bytes <= 4096 && rows % 4 == 0) R = 4;
+  if (rows % 2) R = 1;
+  A.items_per_shard = rows / R;
+  if (dt == DT_BF16) {
+    if (R == 4) return launch_gemv_t<__nv_bfloat16, 4, EPI_PARTIAL>(c, A);
+    if (R == 2) return launch_gemv_t<__nv_bfloat16, 2, EPI_PARTIAL>(c, A);
+    return launch_gemv_t<__nv_bfloat16, 1, EPI_PARTIAL>(c, A);
+  }
+  if (R == 4) return launch_gemv_t<float, 4, EPI_PARTIAL>(c, A);
+  if (R == 2) return launch_gemv_t<float, 2, EPI_PARTIAL>(c, A);
+  return launch_gemv_t<float, 1, EPI_PARTIAL>(c, A);
+}
+
+static int head_rows_per_warp(int vocab) { return vocab % 2 == 0 ? 2 : 1; }
+int head_argmax_blocks(int vocab) {
+  const int R = head_rows_per_warp(vocab);
+  return (vocab / R + 7) / 8;
+}
+
+cudaError_t launch_head_argmax(const LaunchCtx& c, int dt, const void* Whead, const float* xhat,
+                               const float* gain, int h, int vocab, float* logits, float* amax_val,
+                               int* amax_idx, unsigned* ticket, int* tok_hist, int* pos, int advance) {
+  GemvArgs A{};
+  A.W = Whead; A.shard_stride = 0; A.x = xhat; A.x_shard_stride = 0; A.gain = gain; A.K = h;
+  A.n_shards = 1; A.out = logits; A.amax_val = amax_val; A.amax_idx = amax_idx; A.ticket = ticket;
+  A.tok_hist = tok_hist; A.pos_rw = pos; A.rows_total = vocab; A.advance = advance;
+  const int R = head_rows_per_warp(vocab);
+  A.items_per_shard = vocab / R;
+  if (dt == DT_BF16)
+    return R == 2 ? launch_gemv_t<__nv_bfloat16, 2, EPI_LOGITS>(c, A) : launch_gemv_t<__nv_bfloat16, 1, EPI_LOGITS>(c, A);
+  return R == 2 ? launch_gemv_t<float, 2, EPI_LOGITS>(c, A) : launch_gemv_t<float, 1, EPI_LOGITS>(c, A);
+}
+
+// =====================================================================================
+// Embedding row + norm statistics (Algorithm 1 "Preprocess")
+// =====================================================================================
+template <typename WT>
+__global__ void __launch_bounds__(1024) embed_kernel(const WT* emb, const int* tok_hist, const int* pos,
+                                                    int vocab, int max_seq, int h, float eps, float* x,
+                                                    float* xhat, int* err) {
+  __shared__ float red[32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int p = *pos;
+  int tok = (p >= 0 && p < max_seq) ? tok_hist[p] : -1;
+  if (p < 0 || p >= max_seq) {
+    if (threadIdx.x == 0) atomicCAS(err, DEVERR_NONE, DEVERR_POS_RANGE);
+    tok = 0;
+  } else if (tok < 0 || tok >= vocab) {
+    if (threadIdx.x == 0) atomicCAS(err, DEVERR_NONE, DEVERR_TOKEN_RANGE);
+    tok = 0;
+  }
+  const WT* row = emb + (size_t)tok * h;
+  float ss = 0.f;
+  for (int k = threadIdx.x; k < h; k += blockDim.x) {
+    const float v = Elem<WT>::load(row + k);
+    x[k] = v;
+    ss = fmaf(v, v, ss);
+  }
+  ss = block_sum(ss, red);
+  const float r = rsqrtf(ss / (float)h + eps);
+  for (int k = threadIdx.x; k < h; k += blockDim.x) xhat[k] = x[k] * r;
+}
+
+cudaError_t launch_embed(const LaunchCtx& c, int dt, const void* emb, const int* tok_hist,
+                         const int* pos, int vocab, int max_seq, int h, float eps, float* x,
+                         float* xhat, int* err) {
+  if (dt == DT_BF16)
+    return launch_kernel(c, embed_kernel<__nv_bfloat16>, dim3(1), dim3(1024), 0,
+                         (const __nv_bfloat16*)emb, tok_hist, pos, vocab, max_seq, h, eps, x, xhat, err);
+  return launch_kernel(c, embed_kernel<float>, dim3(1), dim3(1024), 0, (const float*)emb, tok_hist, pos,
+                       vocab, max_seq, h, eps, x, xhat, err);
+}
+
+// =====================================================================================
+// Emulated star allreduce + shortcut (+ norm statistics of the next block)
+// =====================================================================================
+__global__ void __launch_bounds__(1024) reduce_residual_kernel(const float* __restrict__ partials,
+                                                              int n_shards, int h, float eps, float* x,
+                                                              float* xhat, float* tap) {
+  __shared__ float red[32];
+  pdl_launch_dependents();
+  pdl_wait();
+  float ss = 0.f;
+  for (int k = threadIdx.x; k < h; k += blockDim.x) {
+    float s = partials[k];  // master's own partial (rank 0) ...
+    for (int i = 1; i < n_shards; ++i) s += partials[(size_t)i * h + k];  // ... plus workers, rank order
+    s += x[k];              // shortcut is added after the allreduce (Eq. 1-2)
+    x[k] = s;
+    if (tap) tap[k] = s;
+    ss = fmaf(s, s, ss);
+  }
+  ss = block_sum(ss, red);
+  const float r = rsqrtf(ss / (float)h + eps);
+  for (int k = threadIdx.x; k < h; k += blockDim.x) xhat[k] = x[k] * r;
+}
+
+cudaError_t launch_reduce_residual(const LaunchCtx& c, const float* partials, int n_shards, int h,
+                                   float eps, float* x, float* xhat, float* tap) {
+  return launch_kernel(c, reduce_residual_kernel, dim3(1), dim3(1024), 0, partials, n_shards, h, eps, x,
+                       xhat, tap);
+}
+
+// =====================================================================================
+// Split-K decode attention (Eq. 1) over cache positions 0..p, grouped query heads
+// =====================================================================================
+// One CTA = (kv head, split).  A "row group" of LPR lanes owns one cached position at a
+// time (LPR * 16 bytes = one K or V row), keeps online-softmax state (m, l, acc) for the GRP
+// query heads of the kv head, and walks the split's positions in batches of P.
+template <typename KT, int GRP, int LPR>
+__global__ void __launch_bounds__(128) decode_attn_kernel(const float* __restrict__ q, const KT* kc,
+                                                          const KT* vc, const int* pos, int max_seq,
+                                                          int nsplit, float* scratch, unsigned* tickets,
+                                                          float* o) {
+  constexpr int VEC = Elem<KT>::VEC;
+  constexpr int D = LPR * VEC;
+  constexpr int WARPS = 4, RG = 32 / LPR, G = WARPS * RG, P = 4;
+  extern __shared__ __align__(16) float sm[];
+  float* sm_m = sm;                 // [G][GRP]
+  float* sm_l = sm + G * GRP;       // [G][GRP]
+  float* sm_acc = sm + 2 * G * GRP; // [G][GRP][D]
+  __shared__ bool s_last;
+
+  const int g = blockIdx.x, split = blockIdx.y;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int grp_id = warp * RG + lane / LPR, sub = lane % LPR;
+  pdl_launch_dependents();
+  pdl_wait();
+  const int n = *pos + 1;  // visible positions (the current one was appended by the QKV kernel)
+  int chunk = (n + nsplit - 1) / nsplit;
+  chunk = (chunk + 31) & ~31;
+  const int s0 = split * chunk, s1 = min(n, s0 + chunk);
+
+  // scores are kept in the log2 domain: q is scaled by log2(e)/sqrt(d)
+  const float qscale = 1.4426950408889634f * rsqrtf((float)D);
+  float qr[GRP][VEC], acc[GRP][VEC], m[GRP], l[GRP];
+#pragma unroll
+  for (int hh = 0; hh < GRP; ++hh) {
+    const float* qp = q + (size_t)(g * GRP + hh) * D + sub * VEC;
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) { qr[hh][v] = qp[v] * qscale; acc[hh][v] = 0.f; }
+    m[hh] = -INFINITY;
+    l[hh] = 0.f;
+  }
+  const KT* kbase = kc + (size_t)g * max_seq * D + sub * VEC;
+  const KT* vbase = vc + (size_t)g * max_seq * D + sub * VEC;
+
+  // The trip count is the same for every lane of the warp (the loop variable is the CTA-wide batch
+  // base), because the score reduction below shuffles across the whole warp.
+  for (int tb = s0; tb < s1; tb += G * P) {
+    const int t0 = tb + grp_id;
+    uint4 kv[P];
+#pragma unroll
+    for (int pp = 0; pp < P; ++pp) {
+      const int t = t0 + pp * G;
+      kv[pp] = (t < s1) ? *reinterpret_cast<const uint4*>(kbase + (size_t)t * D) : make_uint4(0, 0, 0, 0);
+    }
+    float sc[P][GRP];
+#pragma unroll
+    for (int pp = 0; pp < P; ++pp) {
+      float kf[VEC];
+      Elem<KT>::unpack(kv[pp], kf);
+#pragma unroll
+      for (int hh = 0; hh < GRP; ++hh) {
+        float s = 0.f;
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) s = fmaf(qr[hh][v], kf[v], s);
+#pragma unroll
+        for (int off = LPR / 2; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
+        sc[pp][hh] = (t0 + pp * G < s1) ? s : -INFINITY;
+      }
+    }
+#pragma unroll
+    for (int pp = 0; pp < P; ++pp) {
+      const int t = t0 + pp * G;
+      kv[pp] = (t < s1) ? *reinterpret_cast<const uint4*>(vbase + (size_t)t * D) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int hh = 0; hh < GRP; ++hh) {
+      float mx = sc[0][hh];
+#pragma unroll
+      for (int pp = 1; pp < P; ++pp) mx = fmaxf(mx, sc[pp][hh]);
+      const float mn = fmaxf(m[hh], mx);
+      // a group that has seen no position yet keeps m = -inf; use 0 as the reference then so that
+      // exp2(-inf - ref) = 0 instead of exp2(-inf + inf) = NaN
+      const float ref = (mn == -INFINITY) ? 0.f : mn;
+      const float scale = exp2f(m[hh] - ref);
+      m[hh] = mn;
+      l[hh] *= scale;
+#pragma unroll
+      for (int v = 0; v < VEC; ++v) acc[hh][v] *= scale;
+#pragma unroll
+      for (int pp = 0; pp < P; ++pp) sc[pp][hh] = exp2f(sc[pp][hh] - ref);  // 0 for masked positions
+    }
+#pragma unroll
+    for (int pp = 0; pp < P; ++pp) {
+      float vf[VEC];
+      Elem<KT>::unpack(kv[pp], vf);
+#pragma unroll
+      for (int hh = 0; hh < GRP; ++hh) {
+        l[hh] += sc[pp][hh];
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) acc[hh][v] = fmaf(sc[pp][hh], vf[v], acc[hh][v]);
+      }
+    }
+  }
+  // ---- merge the G row groups of this CTA (fixed order)
+#pragma unroll
+  for (int hh = 0; hh < GRP; ++hh) {
+    if (sub == 0) { sm_m[grp_id * GRP + hh] = m[hh]; sm_l[grp_id * GRP + hh] = l[hh]; }
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) sm_acc[(grp_id * GRP + hh) * D + sub * VEC + v] = acc[hh][v];
+  }
+  __syncthreads();
+  float* part = scratch + ((size_t)g * nsplit + split) * GRP * (D + 2);
+  for (int e = threadIdx.x; e < GRP * D; e += blockDim.x) {
+    const int hh = e / D, dd = e - hh * D;
+    float M = -INFINITY;
+    for (int gi = 0; gi < G; ++gi) M = fmaxf(M, sm_m[gi * GRP + hh]);
+    float A = 0.f, L = 0.f;
+    if (M > -INFINITY) {
+      for (int gi = 0; gi < G; ++gi) {
+        const float w = exp2f(sm_m[gi * GRP + hh] - M);
+        A = fmaf(w, sm_acc[(gi * GRP + hh) * D + dd], A);
+        L = fmaf(w, sm_l[gi * GRP + hh], L);
+      }
+    }
+    part[hh * (D + 2) + 2 + dd] = A;
+    if (dd == 0) { part[hh * (D + 2)] = M; part[hh * (D + 2) + 1] = L; }
+  }
+  // ---- the last CTA of this kv head to arrive merges the splits in split order
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned t = atomicAdd(tickets + g, 1u);
+    s_last = (t == (unsigned)nsplit - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const int nact = (n + chunk - 1) / chunk;  // splits that saw at least one position
+  const float* pg = scratch + (size_t)g * nsplit * GRP * (D + 2);
+  for (int e = threadIdx.x; e < GRP * D; e += blockDim.x) {
+    const int hh = e / D, dd = e - hh * D;
+    float M = -INFINITY;
+    for (int s = 0; s < nact; ++s) M = fmaxf(M, __ldcg(pg + (size_t)(s * GRP + hh) * (D + 2)));
+    float A = 0.f, L = 0.f;
+    for (int s = 0; s < nact; ++s) {
+      const float* ps = pg + (size_t)(s * GRP + hh) * (D + 2);
+      const float w = exp2f(__ldcg(ps) - M);
+      A = fmaf(w, __ldcg(ps + 2 + dd), A);
+      L = fmaf(w, __ldcg(ps + 1), L);
+    }
+    o[(size_t)(g * GRP + hh) * D + dd] = A / L;
+  }
+  if (threadIdx.x == 0) tickets[g] = 0u;
+}
+
+size_t decode_attention_scratch_floats(int a, int b, int d, int nsplit) {
+  return (size_t)b * nsplit * (a / b) * (d + 2);
+}
+
+template <typename KT, int GRP, int LPR>
+static cudaError_t launch_attn_t(const LaunchCtx& c, const float* q, const void* kc, const void* vc,
+                                 const int* pos, int b, int max_seq, int nsplit, float* scratch,
+                                 unsigned* tickets, float* o) {
+  constexpr int D = LPR * Elem<KT>::VEC, G = 4 * (32 / LPR);
+  const size_t smem = (size_t)(2 * G * GRP + G * GRP * D) * sizeof(float);
+  auto kern = decode_attn_kernel<KT, GRP, LPR>;
+  static bool attr_done = false;
+  if (!attr_done && smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  return launch_kernel(c, kern, dim3(b, nsplit), dim3(128), smem, q, (const KT*)kc, (const KT*)vc, pos,
+                       max_seq, nsplit, scratch, tickets, o);
+}
+
+template <typename KT, int LPR>
+static cudaError_t launch_attn_g(const LaunchCtx& c, int grp, const float* q, const void* kc,
+                                 const void* vc, const int* pos, int b, int max_seq, int nsplit,
+                                 float* scratch, unsigned* tickets, float* o) {
+  switch (grp) {
+    case 1: return launch_attn_t<KT, 1, LPR>(c, q, kc, vc, pos, b, max_seq, nsplit, scratch, tickets, o);
+    case 2: return launch_attn_t<KT, 2, LPR>(c, q, kc, vc, pos, b, max_seq, nsplit, scratch, tickets, o);
+    case 4: return launch_attn_t<KT, 4, LPR>(c, q, kc, vc, pos, b, max_seq, nsplit, scratch, tickets, o);
+    case 8: return launch_attn_t<KT, 8, LPR>(c, q, kc, vc, pos, b, max_seq, nsplit, scratch, tickets, o);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+cudaError_t launch_decode_attention(const LaunchCtx& c, int dt, const float* q, const void* kcache_layer,
+                                    const void* vcache_layer, const int* pos, int a, int b, int d,
+                                    int max_seq, int nsplit, float* scratch, unsigned* tickets,
+                                    float* o) {
+  const int grp = a / b;
+  const int lpr = (int)(d * dt_size(dt) / 16);
+  if (dt == DT_BF16) {
+    if (lpr == 16) return launch_attn_g<__nv_bfloat16, 16>(c, grp, q, kcache_layer, vcache_layer, pos, b, max_seq, nsplit, scratch, tickets, o);
+    if (lpr == 8) return launch_attn_g<__nv_bfloat16, 8>(c, grp, q, kcache_layer, vcache_layer, pos, b, max_seq, nsplit, scratch, tickets, o);
+    if (lpr == 4) return launch_attn_g<__nv_bfloat16, 4>(c, grp, q, kcache_layer, vcache_layer, pos, b, max_seq, nsplit, scratch, tickets, o);
+  } else {
+    if (lpr == 32) return launch_attn_g<float, 32>(c, grp, q, kcache_layer, vcache_layer, pos, b, max_seq, nsplit, scratch, tickets, o);
+    if (lpr == 16) return launch_attn_g<float, 16>(c, grp, q, kcache_layer, vcache_layer, pos, b, max_seq, nsplit, scratch, tickets, o);
+    if (lpr == 8) return launch_attn_g<float, 8>(c, grp, q, kcache_layer, vcache_layer, pos, b, max_seq, nsplit, scratch, tickets, o);
+  }
+  return cudaErrorInvalidValue;
+}
+
+// =====================================================================================
+// Rotary table (built once per model)
+// =====================================================================================
+__global__ void rope_table_kernel(const double* inv_freq, int max_seq, int half, float2* table) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (size_t)max_seq * half) return;
+  const int p = (int)(i / half), k = (int)(i - (size_t)p * half);
+  double s, cth;
+  sincos((double)p * inv_freq[k], &s, &cth);
+  table[i] = make_float2((float)cth, (float)s);
+}
+
+cudaError_t launch_rope_table(const LaunchCtx& c, const double* inv_freq, int max_seq, int half,
+                              float2* table) {
+  const size_t n = (size_t)max_seq * half;
+  return launch_kernel(c, rope_table_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, inv_freq,
+                       max_seq, half, table);
+}
+
+}  // namespace tpi

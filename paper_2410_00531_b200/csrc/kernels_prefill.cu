@@ -1,0 +1,363 @@
+// Prefill kernels: the same decoder block over T prompt positions at once
+// (Algorithm 1, first pass of the loop: causal mask, cache positions pos0..pos0+T-1).
+// This file holds the fp32-accurate SIMT path used for fp32 models and as the
+// general fallback; the bf16 tensor-core GEMM lives in gemm_tcgen05.cu.
+#include "common.cuh"
+#include "kernels.h"
+#include "launch.cuh"
+
+namespace tpi {
+
+// ------------------------------------------------------------------ embedding rows
+template <typename WT>
+__global__ void embed_rows_kernel(const WT* emb, const int* tok_hist, int pos0, int vocab, int h, float* X,
+                                  int* err) {
+  const int t = blockIdx.x;
+  int tok = tok_hist[pos0 + t];
+  if (tok < 0 || tok >= vocab) {
+    if (threadIdx.x == 0) atomicCAS(err, DEVERR_NONE, DEVERR_TOKEN_RANGE);
+    tok = 0;
+  }
+  const WT* row = emb + (size_t)tok * h;
+  for (int k = threadIdx.x; k < h; k += blockDim.x) X[(size_t)t * h + k] = Elem<WT>::load(row + k);
+}
+
+cudaError_t launch_embed_rows(const LaunchCtx& c, int dt, const void* emb, const int* tok_hist, int pos0,
+                              int T, int vocab, int h, float* X, int* err) {
+  LaunchCtx nc = c;
+  nc.pdl = false;
+  if (dt == DT_BF16)
+    return launch_kernel(nc, embed_rows_kernel<__nv_bfloat16>, dim3(T), dim3(256), 0,
+                         (const __nv_bfloat16*)emb, tok_hist, pos0, vocab, h, X, err);
+  return launch_kernel(nc, embed_rows_kernel<float>, dim3(T), dim3(256), 0, (const float*)emb, tok_hist,
+                       pos0, vocab, h, X, err);
+}
+
+// ------------------------------------------------------------------ RMSNorm rows
+template <int OUT_BF16>
+__global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float* X, const float* gain, int h, float eps,
+                                                          void* Xn) {
+  __shared__ float red[32];
+  const float* x = X + (size_t)blockIdx.x * h;
+  float ss = 0.f;
+  for (int k = threadIdx.x; k < h; k += blockDim.x) ss = fmaf(x[k], x[k], ss);
+  ss = block_sum(ss, red);
+  const float r = rsqrtf(ss / (float)h + eps);
+  for (int k = threadIdx.x; k < h; k += blockDim.x) {
+    const float v = x[k] * r * gain[k];
+    if (OUT_BF16)
+      reinterpret_cast<__nv_bfloat16*>(Xn)[(size_t)blockIdx.x * h + k] = __float2bfloat16_rn(v);
+    else
+      reinterpret_cast<float*>(Xn)[(size_t)blockIdx.x * h + k] = v;
+  }
+}
+
+cudaError_t launch_rmsnorm_rows(const LaunchCtx& c, const float* X, const float* gain, int T, int h,
+                                float eps, void* Xn, int out_bf16) {
+  LaunchCtx nc = c;
+  nc.pdl = false;
+  if (out_bf16) return launch_kernel(nc, rmsnorm_rows_kernel<1>, dim3(T), dim3(256), 0, X, gain, h, eps, Xn);
+  return launch_kernel(nc, rmsnorm_rows_kernel<0>, dim3(T), dim3(256), 0, X, gain, h, eps, Xn);
+}
+
+__global__ void __launch_bounds__(1024) rmsnorm_stat_row_kernel(const float* xrow, int h, float eps, float* x,
+                                                               float* xhat, int* pos, int pos_value) {
+  __shared__ float red[32];
+  float ss = 0.f;
+  for (int k = threadIdx.x; k < h; k += blockDim.x) {
+    const float v = xrow[k];
+    x[k] = v;
+    ss = fmaf(v, v, ss);
+  }
+  ss = block_sum(ss, red);
+  const float r = rsqrtf(ss / (float)h + eps);
+  for (int k = threadIdx.x; k < h; k += blockDim.x) xhat[k] = xrow[k] * r;
+  if (threadIdx.x == 0 && pos) *pos = pos_value;
+}
+
+cudaError_t launch_rmsnorm_stat_row(const LaunchCtx& c, const float* xrow, int h, float eps, float* x,
+                                    float* xhat, int* pos, int pos_value) {
+  LaunchCtx nc = c;
+  nc.pdl = false;
+  return launch_kernel(nc, rmsnorm_stat_row_kernel, dim3(1), dim3(1024), 0, xrow, h, eps, x, xhat, pos,
+                       pos_value);
+}
+
+// ------------------------------------------------------------------ SIMT GEMM (fp32 accumulate)
+// Y[b][t][o] = sum_k X[b][t][k] * W[b][o][k];   64x64 tile, 16-deep slices, 4x4 per thread.
+template <typename WT>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const float* __restrict__ X, long long xbs, int ldx,
+                                                        const WT* __restrict__ W, long long wbs,
+                                                        float* __restrict__ Y, long long ybs, int ldy, int T,
+                                                        int n_out, int K) {
+  constexpr int BM = 64, BN = 64, BK = 16;
+  __shared__ __align__(16) float Xs[BK][BM + 4];
+  __shared__ __align__(16) float Ws[BK][BN + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  X += (size_t)blockIdx.z * xbs;
+  W += (size_t)blockIdx.z * wbs;
+  Y += (size_t)blockIdx.z * ybs;
+  const int lrow = tid >> 2, lk = (tid & 3) * 4;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (int k0 = 0; k0 < K; k0 += BK) {
+    float xv[4] = {0.f, 0.f, 0.f, 0.f}, wv[4] = {0.f, 0.f, 0.f, 0.f};
+    if (m0 + lrow < T && k0 + lk < K) {
+      const float4 v = *reinterpret_cast<const float4*>(X + (size_t)(m0 + lrow) * ldx + k0 + lk);
+      xv[0] = v.x; xv[1] = v.y; xv[2] = v.z; xv[3] = v.w;
+    }
+    if (n0 + lrow < n_out && k0 + lk < K) {
+      const WT* wp = W + (size_t)(n0 + lrow) * K + k0 + lk;
+      if constexpr (sizeof(WT) == 2) {
+        const uint2 v = *reinterpret_cast<const uint2*>(wp);
+        wv[0] = bf16lo(v.x); wv[1] = bf16hi(v.x); wv[2] = bf16lo(v.y); wv[3] = bf16hi(v.y);
+      } else {
+        const float4 v = *reinterpret_cast<const float4*>(wp);
+        wv[0] = v.x; wv[1] = v.y; wv[2] = v.z; wv[3] = v.w;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { Xs[lk + i][lrow] = xv[i]; Ws[lk + i][lrow] = wv[i]; }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      const float4 a = *reinterpret_cast<const float4*>(&Xs[kk][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&Ws[kk][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + ty * 4 + i;
+    if (m >= T) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n < n_out) Y[(size_t)m * ldy + n] = acc[i][j];
+    }
+  }
+}
+
+cudaError_t launch_gemm_simt(const LaunchCtx& c, int dt, const float* X, long long x_batch_stride, int ldx,
+                             const void* W, long long w_batch_stride_elems, float* Y,
+                             long long y_batch_stride, int ldy, int T, int n_out, int K, int n_batch) {
+  LaunchCtx nc = c;
+  nc.pdl = false;
+  dim3 grid((n_out + 63) / 64, (T + 63) / 64, n_batch);
+  if (dt == DT_BF16)
+    return launch_kernel(nc, gemm_simt_kernel<__nv_bfloat16>, grid, dim3(256), 0, X, x_batch_stride, ldx,
+                         (const __nv_bfloat16*)W, w_batch_stride_elems, Y, y_batch_stride, ldy, T, n_out, K);
+  return launch_kernel(nc, gemm_simt_kernel<float>, grid, dim3(256), 0, X, x_batch_stride, ldx,
+                       (const float*)W, w_batch_stride_elems, Y, y_batch_stride, ldy, T, n_out, K);
+}
+
+// ------------------------------------------------------------------ rotary + KV append for T rows
+// QKV[t] holds, per shard i, [q heads | k heads | v heads] of that shard (the GEMM's column order).
+template <typename WT>
+__global__ void rope_kv_rows_kernel(const float* QKV, int pos0, int n_shards, int a, int b, int d, int max_seq,
+                                    const float2* rope, float* Q, WT* kc, WT* vc) {
+  const int t = blockIdx.x, half = d >> 1;
+  const int hps = a / n_shards, kps = b / n_shards;
+  const int per_shard = (hps + 2 * kps) * d;
+  const float* row = QKV + (size_t)t * per_shard * n_shards;
+  const int p = pos0 + t;
+  const int pairs = (a + b) * half;  // rotary pairs of q and k
+  for (int e = threadIdx.x; e < pairs + b * d; e += blockDim.x) {
+    if (e < pairs) {
+      const int head = e / half, ii = e - head * half;  // heads 0..a-1 are q, a..a+b-1 are k
+      const bool is_q = head < a;
+      const int gh = is_q ? head : head - a;
+      const int shard = is_q ? gh / hps : gh / kps;
+      const int hl = is_q ? gh - shard * hps : gh - shard * kps;
+      const float* src = row + (size_t)shard * per_shard + (is_q ? 0 : hps * d) + hl * d;
+      const float2 cs = rope[(size_t)p * half + ii];
+      const float lo = src[ii] * cs.x - src[ii + half] * cs.y;
+      const float hi = src[ii + half] * cs.x + src[ii] * cs.y;
+      if (is_q) {
+        float* q = Q + ((size_t)t * a + gh) * d;
+        q[ii] = lo;
+        q[ii + half] = hi;
+      } else {
+        WT* kr = kc + ((size_t)gh * max_seq + p) * d;
+        Elem<WT>::store(kr + ii, lo);
+        Elem<WT>::store(kr + ii + half, hi);
+      }
+    } else {
+      const int e2 = e - pairs, gh = e2 / d, idx = e2 - gh * d;
+      const int shard = gh / kps, hl = gh - shard * kps;
+      const float* src = row + (size_t)shard * per_shard + (hps + kps) * d + hl * d;
+      Elem<WT>::store(vc + ((size_t)gh * max_seq + p) * d + idx, src[idx]);
+    }
+  }
+}
+
+cudaError_t launch_rope_kv_rows(const LaunchCtx& c, int dt, const float* QKV, int T, int pos0, int n_shards,
+                                int a, int b, int d, int max_seq, const float2* rope, float* Q,
+                                void* kcache_layer, void* vcache_layer) {
+  LaunchCtx nc = c;
+  nc.pdl = false;
+  if (dt == DT_BF16)
+    return launch_kernel(nc, rope_kv_rows_kernel<__nv_bfloat16>, dim3(T), dim3(256), 0, QKV, pos0, n_shards, a,
+                         b, d, max_seq, rope, Q, (__nv_bfloat16*)kcache_layer, (__nv_bfloat16*)vcache_layer);
+  return launch_kernel(nc, rope_kv_rows_kernel<float>, dim3(T), dim3(256), 0, QKV, pos0, n_shards, a, b, d,
+                       max_seq, rope, Q, (float*)kcache_layer, (float*)vcache_layer);
+}
+
+// ------------------------------------------------------------------ causal attention, T queries
+// One warp = one (query position, head).  Per tile of 32 cached positions: each lane scores one
+// position (full dot product, q broadcast from shared memory), the tile's softmax statistics go
+// through shuffles, then each lane accumulates its d/32 output dims over the tile's values.
+template <typename KT, int D>
+__global__ void __launch_bounds__(128) prefill_attn_kernel(const float* __restrict__ Q, const KT* kc,
+                                                           const KT* vc, int T, int pos0, int a, int b,
+                                                           int max_seq, float* O) {
+  constexpr int VEC = Elem<KT>::VEC, DPL = D / 32;
+  __shared__ __align__(16) float qs[4][D];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t = blockIdx.x * 4 + warp, j = blockIdx.y, g = j / (a / b);
+  const bool active = t < T;
+  const float qscale = 1.4426950408889634f * rsqrtf((float)D);
+  if (active)
+    for (int i = lane; i < D; i += 32) qs[warp][i] = Q[((size_t)t * a + j) * D + i] * qscale;
+  __syncwarp();
+  if (!active) return;
+  const int n = pos0 + t + 1;
+  const KT* kb = kc + (size_t)g * max_seq * D;
+  const KT* vb = vc + (size_t)g * max_seq * D;
+  float m = -INFINITY, l = 0.f, acc[DPL];
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
+  for (int p0 = 0; p0 < n; p0 += 32) {
+    const int p = p0 + lane;
+    float s = -INFINITY;
+    if (p < n) {
+      s = 0.f;
+      const uint4* kr = reinterpret_cast<const uint4*>(kb + (size_t)p * D);
+#pragma unroll 4
+      for (int v = 0; v < D / VEC; ++v) s = Elem<KT>::dot(kr[v], &qs[warp][v * VEC], s);
+    }
+    float mx = s;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    const float mn = fmaxf(m, mx);
+    const float scale = exp2f(m - mn);
+    const float w = exp2f(s - mn);
+    l = l * scale + warp_sum(w);
+    m = mn;
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) acc[i] *= scale;
+    const int cnt = min(32, n - p0);
+    for (int u = 0; u < cnt; ++u) {
+      const float wu = __shfl_sync(0xFFFFFFFFu, w, u);
+      const KT* vr = vb + (size_t)(p0 + u) * D + lane * DPL;
+#pragma unroll
+      for (int i = 0; i < DPL; ++i) acc[i] = fmaf(wu, Elem<KT>::load(vr + i), acc[i]);
+    }
+  }
+  float* o = O + ((size_t)t * a + j) * D + lane * DPL;
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) o[i] = acc[i] / l;
+}
+
+cudaError_t launch_prefill_attention(const LaunchCtx& c, int dt, const float* Q, const void* kcache_layer,
+                                     const void* vcache_layer, int T, int pos0, int a, int b, int d,
+                                     int max_seq, float* O) {
+  LaunchCtx nc = c;
+  nc.pdl = false;
+  dim3 grid((T + 3) / 4, a);
+#define TPI_PA(KT, DD)                                                                                     \
+  return launch_kernel(nc, prefill_attn_kernel<KT, DD>, grid, dim3(128), 0, Q, (const KT*)kcache_layer,     \
+                       (const KT*)vcache_layer, T, pos0, a, b, max_seq, O)
+  if (dt == DT_BF16) {
+    if (d == 128) TPI_PA(__nv_bfloat16, 128);
+    if (d == 64) TPI_PA(__nv_bfloat16, 64);
+    if (d == 32) TPI_PA(__nv_bfloat16, 32);
+  } else {
+    if (d == 128) TPI_PA(float, 128);
+    if (d == 64) TPI_PA(float, 64);
+    if (d == 32) TPI_PA(float, 32);
+  }
+#undef TPI_PA
+  return cudaErrorInvalidValue;
+}
+
+// ------------------------------------------------------------------ SwiGLU rows
+__global__ void swiglu_rows_kernel(const float* GU, size_t n_pairs, float* ACT) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_pairs) return;
+  const float2 gu = reinterpret_cast<const float2*>(GU)[i];
+  ACT[i] = gu.x / (1.f + expf(-gu.x)) * gu.y;
+}
+
+cudaError_t launch_swiglu_rows(const LaunchCtx& c, const float* GU, int T, int s, float* ACT) {
+  LaunchCtx nc = c;
+  nc.pdl = false;
+  const size_t n = (size_t)T * s;
+  return launch_kernel(nc, swiglu_rows_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, GU, n, ACT);
+}
+
+// ------------------------------------------------------------------ allreduce + shortcut, T rows
+__global__ void reduce_residual_rows_kernel(const float* __restrict__ partials, int n_shards, int T, int h,
+                                            float* X, float* tap_last) {
+  const size_t n = (size_t)T * h;
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  float s = partials[i];
+  for (int k = 1; k < n_shards; ++k) s += partials[(size_t)k * n + i];
+  s += X[i];
+  X[i] = s;
+  if (tap_last && i >= n - h) tap_last[i - (n - h)] = s;
+}
+
+cudaError_t launch_reduce_residual_rows(const LaunchCtx& c, const float* partials, int n_shards, int T,
+                                        int h, float* X, float* tap_last) {
+  LaunchCtx nc = c;
+  nc.pdl = false;
+  const size_t n = (size_t)T * h;
+  return launch_kernel(nc, reduce_residual_rows_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0,
+                       partials, n_shards, T, h, X, tap_last);
+}
+
+// ------------------------------------------------------------------ misc
+__global__ void fill_u32_kernel(uint32_t* p, size_t n, uint32_t v) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    p[i] = v;
+}
+cudaError_t launch_fill_u32(const LaunchCtx& c, uint32_t* p, size_t n, uint32_t v) {
+  LaunchCtx nc = c;
+  nc.pdl = false;
+  const unsigned blocks = (unsigned)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184);
+  return launch_kernel(nc, fill_u32_kernel, dim3(blocks ? blocks : 1), dim3(256), 0, p, n, v);
+}
+
+template <typename WT, int TO_FLOAT>
+__global__ void kv_convert_kernel(WT* cache, float* f, size_t n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  if (TO_FLOAT) f[i] = Elem<WT>::load(cache + i);
+  else Elem<WT>::store(cache + i, f[i]);
+}
+cudaError_t launch_kv_convert(const LaunchCtx& c, int dt, void* cache_rows, float* f32_rows, size_t n,
+                              int to_float) {
+  LaunchCtx nc = c;
+  nc.pdl = false;
+  dim3 grid((unsigned)((n + 255) / 256));
+  if (dt == DT_BF16) {
+    if (to_float) return launch_kernel(nc, kv_convert_kernel<__nv_bfloat16, 1>, grid, dim3(256), 0, (__nv_bfloat16*)cache_rows, f32_rows, n);
+    return launch_kernel(nc, kv_convert_kernel<__nv_bfloat16, 0>, grid, dim3(256), 0, (__nv_bfloat16*)cache_rows, f32_rows, n);
+  }
+  if (to_float) return launch_kernel(nc, kv_convert_kernel<float, 1>, grid, dim3(256), 0, (float*)cache_rows, f32_rows, n);
+  return launch_kernel(nc, kv_convert_kernel<float, 0>, grid, dim3(256), 0, (float*)cache_rows, f32_rows, n);
+}
+
+}  // namespace tpi

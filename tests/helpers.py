@@ -36,3 +36,44 @@ def rel_l2(got, want) -> float:
 
 
 TINY = S.ModelShape("tiny-test", 2, 32, 4, 2, 8, 48, 37, 1e-5, 10000.0, "f32", 7, 2, 5, 3)
+
+
+# ------------------------------------------------------------------ GPU harness
+def tpi_config(shape: S.ModelShape, max_seq: int, max_prefill: int):
+    import paper_2410_00531_b200 as P
+    return P.make_config(n_layers=shape.n_layers, hidden=shape.hidden, n_heads=shape.n_heads,
+                         n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim, ffn=shape.ffn,
+                         vocab=shape.vocab, max_seq=max_seq, max_prefill=max_prefill,
+                         rms_eps=shape.rms_eps, rope_base=shape.rope_base, dtype=shape.dtype)
+
+
+def gpu_session(shape: S.ModelShape, max_seq: int, max_prefill: int, n_shards: int | None = None,
+                window: int = 0, alias_layers: int | None = None, **kw):
+    import paper_2410_00531_b200 as P
+    cfg = tpi_config(shape, max_seq, max_prefill)
+    return P.Session(cfg, S.synth_fill(shape, alias_layers), n_shards or shape.n_shards, window, **kw)
+
+
+def tol_for(shape: S.ModelShape) -> float:
+    """Relative-L2 bar on hidden states and logits: 1e-5 for fp32 weights, 1e-2 for bf16."""
+    return 1e-5 if shape.dtype == "f32" else 1e-2
+
+
+def check_logits(gpu_logits, gpu_token, oracle_logits, tol) -> tuple[bool, bool]:
+    """The token rule.  Returns (token_matches, step_was_ambiguous); raises on a violation.
+
+    (1) rel-L2(logits) <= tol; (2) each of the oracle's top-8 logits is reproduced within
+    e = 3 * tol * rms(oracle logits); (3) the GPU's greedy token equals the oracle's, or the
+    oracle's top-2 gap is <= 2e and the GPU picked the runner-up."""
+    o = np.asarray(oracle_logits, np.float64)
+    g = np.asarray(gpu_logits, np.float64)
+    assert rel_l2(g, o) <= tol, f"logits rel-L2 {rel_l2(g, o):.3e} > {tol}"
+    e = 3 * tol * float(np.sqrt(np.mean(o * o)))
+    top = np.argsort(-o, kind="stable")[:8]
+    assert np.abs(g[top] - o[top]).max() <= e
+    ambiguous = (o[top[0]] - o[top[1]]) <= 2 * e
+    assert int(np.argmax(g)) == gpu_token, "device argmax disagrees with the logits it returned"
+    if gpu_token == int(top[0]):
+        return True, ambiguous
+    assert ambiguous and gpu_token == int(top[1]), "token differs although the oracle's gap exceeds the tolerance"
+    return False, True

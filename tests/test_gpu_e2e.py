@@ -1,0 +1,132 @@
+"""End-to-end parity of the CUDA library against the CPU oracle through the C ABI
+(tiny fp32 workload C1, full depth; small bf16 / grouped-head variants)."""
+import numpy as np
+import pytest
+
+import tpi_synth as S
+from tests.helpers import check_logits, gpu_session, make_oracle, rel_l2, tol_for
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_and_compare(shape, n_shards, window=0, n_decode=8, prompt_len=None, max_prefill=None, opts=()):
+    import paper_2410_00531_b200 as P
+    tol = tol_for(shape)
+    toks = S.prompt_tokens(shape, prompt_len or shape.prompt_len)
+    T = len(toks)
+    orc = make_oracle(shape)
+    with gpu_session(shape, T + n_decode + 1, max_prefill or T, n_shards, window) as ses:
+        for o, v in opts:
+            P.set_option(ses.h, o, v)
+        tok, lg = P.prefill(ses.h, toks, shape.vocab)
+        want = orc.forward(toks)
+        check_logits(lg, tok, want, tol)
+        for l in range(shape.n_layers):
+            assert rel_l2(P.get_hidden(ses.h, l, 0, shape.hidden), orc.taps[(l, "attn")][-1]) <= tol
+            assert rel_l2(P.get_hidden(ses.h, l, 1, shape.hidden), orc.taps[(l, "ffn")][-1]) <= tol
+        # cache contents and indexing: slot p holds position p
+        for l in range(shape.n_layers):
+            for g in range(shape.n_kv_heads):
+                k, v = P.get_kv(ses.h, l, g, 0, T, shape.head_dim)
+                assert rel_l2(k, orc.cache.K[l][g]) <= tol and rel_l2(v, orc.cache.V[l][g]) <= tol
+        out_tokens, mismatches = [tok], 0
+        feed = int(np.argmax(want))
+        for step in range(n_decode):
+            tok, lg = P.decode_step(ses.h, feed, shape.vocab)   # teacher-forced with the oracle's token
+            want = orc.forward([feed])
+            ok, _ = check_logits(lg, tok, want, tol)
+            mismatches += (not ok)
+            for l in range(shape.n_layers):
+                assert rel_l2(P.get_hidden(ses.h, l, 1, shape.hidden), orc.taps[(l, "ffn")][-1]) <= tol
+            feed = int(np.argmax(want))
+            out_tokens.append(tok)
+        assert P.position(ses.h) == T + n_decode
+        k, v = P.get_kv(ses.h, shape.n_layers - 1, 0, T, n_decode, shape.head_dim)
+        assert rel_l2(k, orc.cache.K[-1][0][T:]) <= tol
+        return out_tokens, mismatches
+
+
+@pytest.mark.parametrize("n_shards", [1, 2, 4])
+def test_c1_full_depth(n_shards):
+    shape = S.CONFIGS["C1"]
+    toks, mism = _run_and_compare(shape, n_shards)
+    assert mism == 0                           # fp32: gaps are far above the tolerance
+    ref, _ = make_oracle(shape).greedy(S.prompt_tokens(shape), 9)
+    assert toks == list(ref)                   # "identical to single-server inference"
+
+
+def test_c1_without_graph_and_pdl():
+    import paper_2410_00531_b200 as P
+    shape = S.CONFIGS["C1"]
+    _run_and_compare(shape, 2, opts=((P.OPT_GRAPH, 0), (P.OPT_PDL, 0)))
+    _run_and_compare(shape, 2, opts=((P.OPT_GRAPH, 0), (P.OPT_PDL, 1)))
+
+
+def test_chunked_prefill_matches():
+    shape = S.CONFIGS["C1"]
+    _run_and_compare(shape, 2, prompt_len=23, max_prefill=8, n_decode=3)
+
+
+def test_small_bf16_gqa():
+    shape = S.CONFIGS["C1"].with_(dtype="bf16", n_heads=8, n_kv_heads=2, head_dim=32, seed=77, rope_base=500000.0)
+    _run_and_compare(shape, 2)
+
+
+def test_small_f32_gqa8_d128():
+    shape = S.ModelShape("gqa8", 2, 1024, 8, 1, 128, 1408, 3001, 1e-5, 500000.0, "f32", 78, 1, 40, 4)
+    _run_and_compare(shape, 1)
+
+
+@pytest.mark.parametrize("window", [1, 2, 3, 4])
+def test_streamed_is_bit_identical_to_resident(window):
+    import paper_2410_00531_b200 as P
+    shape = S.CONFIGS["C1"].with_(n_layers=4)
+    toks = S.prompt_tokens(shape)
+    res = {}
+    for w in (0, window):
+        with gpu_session(shape, 64, 16, 2, w) as ses:
+            t0, lg0 = P.prefill(ses.h, toks, shape.vocab)
+            seq = P.decode_run(ses.h, t0, 6)
+            t1, lg1 = P.decode_step(ses.h, int(seq[-1]), shape.vocab)
+            res[w] = (t0, lg0, seq, t1, lg1)
+            st = P.get_stats(ses.h)
+            if w:
+                assert st["blocks_loaded"] >= 8 * 8 and st["link_bytes_total"] > 0
+    a, b = res[0], res[window]
+    assert a[0] == b[0] and a[3] == b[3] and (a[2] == b[2]).all()
+    assert np.array_equal(a[1], b[1]) and np.array_equal(a[4], b[4])
+
+
+def test_set_shards_and_set_window_roundtrip():
+    import paper_2410_00531_b200 as P
+    shape = S.CONFIGS["C1"]
+    toks = S.prompt_tokens(shape)
+    want = make_oracle(shape).forward(toks)
+    with gpu_session(shape, 64, 16, 2, 0, other_windows=(2,)) as ses:
+        for n, w in ((2, 0), (4, 0), (4, 2), (1, 2), (1, 0)):
+            P.set_shards(ses.h, n)
+            P.set_window(ses.h, w)
+            tok, lg = P.prefill(ses.h, toks, shape.vocab)
+            check_logits(lg, tok, want, 1e-5)
+            st = P.get_stats(ses.h)
+            assert st["n_shards"] == n and st["window_blocks"] == w
+
+
+def test_error_codes():
+    import paper_2410_00531_b200 as P
+    shape = S.CONFIGS["C1"]
+    with pytest.raises(P.TpiError) as e:
+        gpu_session(shape, 64, 16, 3)                      # 3 does not divide 4 heads
+    assert e.value.code == -2
+    with gpu_session(shape, 20, 16, 2) as ses:
+        with pytest.raises(P.TpiError) as e:
+            P.prefill(ses.h, [1, 2, shape.vocab], 0)
+        assert e.value.code == -5
+        tok, _ = P.prefill(ses.h, S.prompt_tokens(shape), 0)
+        P.decode_run(ses.h, tok, 4)
+        with pytest.raises(P.TpiError) as e:
+            P.decode_step(ses.h, 1, 0)                     # position 20 == max_seq
+        assert e.value.code == -4
+        with pytest.raises(P.TpiError) as e:
+            P.set_window(ses.h, 2)                         # resident load kept no host images
+        assert e.value.code in (-9, -3)

@@ -201,3 +201,23 @@ def kv_contents(seed: int, shape_: tuple[int, ...], scale: float = 1.3) -> np.nd
     """Float32 stand-in for cached keys/values: N(0, 1.3^2) matches 0.02*sqrt(h)."""
     rng = np.random.Generator(np.random.PCG64(seed))
     return (rng.standard_normal(shape_) * scale).astype(np.float32)
+
+
+def synth_fill(shape: ModelShape, alias_layers: int | None = None):
+    """Weight source for the GPU library's load callback:
+    fill(tensor_id, layer, row0, n_rows, dst_address, n_bytes) writes rows of the unsharded tensor.
+
+    alias_layers = K maps layer l to l mod K (declared stand-in when a model's
+    distinct layers would not fit in host memory; the oracle side must alias too)."""
+    esz = 2 if shape.dtype == "bf16" else 4
+
+    def fill(tid: int, layer: int, row0: int, n_rows: int, dst: int, n_bytes: int) -> None:
+        dims = shape.tensor_shape(tid)
+        row_len = dims[-1]
+        if alias_layers:
+            layer = layer % alias_layers
+        assert n_bytes == n_rows * row_len * esz
+        off, sc = offset_scale(tid)
+        fill_raw(shape.seed, tensor_uid(layer, tid), row0 * row_len, n_rows * row_len, off, sc,
+                 shape.dtype == "bf16", dst)
+    return fill
