@@ -1,0 +1,298 @@
+#!/usr/bin/env python
+"""Benchmark of the TPI-LLM decoder hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload C2]
+
+One "step" is one pass of the whole per-token hot path (embedding, L x [norm,
+column-sharded QKV + RoPE + KV append, attention over the cache, row-sharded O ->
+N partials, rank-ordered sum + shortcut, norm, gate/up + SwiGLU, down -> partials,
+sum + shortcut], final norm, task head, greedy argmax) on the workload C2:
+a Llama-2-7B-shaped decoder, bf16 weights, fp32 accumulation, N = 4 shards
+emulated on one GPU, prompt of 128 random tokens, all weights resident.
+
+Prints ONE JSON line.  `value` is decode tokens/s with everything resident on the
+device (token ids chained on the device, one host wait for the K steps, CUDA
+events on the launching stream); `e2e` is the same metric through the public
+per-token call with the token id copied host->device and the result device->host
+every step.  TTFT (the prompt pass) and the whole-token roofline are extra keys.
+With --gpus N > 1 (torchrun) every rank runs an independent replica: the method's
+path on one GPU has no exchange step (all shards are emulated on-device).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import re
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import tpi_synth as S  # noqa: E402
+
+METRIC = "decode_tokens_per_s_batch1"
+UNIT = "tokens/s"
+
+
+# ------------------------------------------------------------------ helpers
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def traffic_from_profile(workload: str):
+    """DRAM bytes per launch of the dominant kernel, from the committed ncu summary (or None)."""
+    p = os.path.join(ROOT, "profiles", f"gemv_gateup_{workload.lower()}.md")
+    if os.path.exists(p):
+        m = re.search(r"traffic_bytes_per_launch:\s*([0-9.eE+]+)", open(p).read())
+        if m:
+            return float(m.group(1))
+    return None
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.rows, self.proc = index, [], None
+
+    def run(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            for line in self.proc.stdout:
+                self.rows.append([c.strip() for c in line.split(",")])
+        except Exception:
+            pass
+
+    def stop(self) -> dict:
+        if self.proc:
+            self.proc.terminate()
+        self.join(timeout=2)
+        sm, mx, reasons = [], 0.0, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = max(mx, float(r[1]))
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except (ValueError, IndexError):
+                continue
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx or None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(shape: S.ModelShape, n_tokens: int, l_red: int = 2, ctx: int = 16):
+    """Time the CPU fp64 oracle, as it stands, on a bounded sample of the workload:
+    `l_red` layers at full width + the task head, `n_tokens` decode steps after a `ctx`-token
+    prompt; per-layer time is scaled linearly to the full depth.  Weight generation is excluded."""
+    from tests.helpers import make_oracle
+    red = shape.with_(n_layers=l_red)
+    orc = make_oracle(red, cache=64)
+    toks = S.prompt_tokens(red, ctx)
+    orc.forward(toks)                       # also pulls every weight through the generator once
+    t_steps = []
+    tok = 1
+    for _ in range(n_tokens):
+        t0 = time.perf_counter()
+        lg = orc.forward([tok])
+        t_steps.append(time.perf_counter() - t0)
+        tok = int(np.argmax(lg))
+    # split one more step into layer part and head part
+    t0 = time.perf_counter()
+    x = orc.w(0, S.EMB)[[tok]]
+    pos = np.array([orc.cache.length])
+    for l in range(l_red):
+        _, x, _, _ = orc.layer_unsharded(l, x, pos, orc.cache.K[l], orc.cache.V[l])
+    t_layers = time.perf_counter() - t0
+    t_step = float(np.median(t_steps))
+    t_head = max(t_step - t_layers, 0.0)
+    t_full = t_layers / l_red * shape.n_layers + t_head
+    return 1.0 / t_full, t_steps, f"{l_red} of {shape.n_layers} layers at full width + head, {n_tokens} decode steps at context {ctx}, per-layer time scaled to {shape.n_layers} layers"
+
+
+def run_reference(args, shape):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = len(os.sched_getaffinity(0))
+    # warm-up and timed steps are both bounded samples (2 layers + head per step)
+    n = max(1, args.steps)
+    t0 = time.perf_counter()
+    value, steps, sample = oracle_sample(shape, args.warmup + n)
+    steps = steps[args.warmup:]
+    ms = float(np.mean(steps)) * 1e3
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / value, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": workload_name(shape, args), "sample_ms_per_step": ms},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0, "wall_s": time.perf_counter() - t0}
+    print(json.dumps(out), flush=True)
+
+
+def workload_name(shape, args):
+    return (f"{args.workload}: {shape.name}, L{shape.n_layers} h{shape.hidden} a{shape.n_heads} b{shape.n_kv_heads} "
+            f"s{shape.ffn} v{shape.vocab}, {shape.dtype} weights/KV, fp32 accumulate, N={shape.n_shards} shards "
+            f"emulated on one GPU, prompt {shape.prompt_len}, all weights resident")
+
+
+# ------------------------------------------------------------------ GPU arm
+def run_gpu(args, shape):
+    import torch
+    import paper_2410_00531_b200 as P
+    from tests.helpers import tpi_config
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    K, W, T = args.steps, args.warmup, shape.prompt_len
+    max_seq = T + W + K + 8
+    cfg = tpi_config(shape, max_seq, min(T, 512))
+    t_load = time.perf_counter()
+    ses = P.Session(cfg, S.synth_fill(shape), shape.n_shards, 0, device=local)
+    t_load = time.perf_counter() - t_load
+    toks = S.prompt_tokens(shape)
+    h = ses.h
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- TTFT: prompt pass (host wall time of the call incl. the token's D2H), best of 3 after a warm pass
+    ttft = []
+    for _ in range(4):
+        P.reset(h)
+        t0 = time.perf_counter()
+        first, _ = P.prefill(h, toks, 0)
+        ttft.append((time.perf_counter() - t0) * 1e3)
+    ttft_ms = min(ttft[1:])
+
+    # ---- device-resident decode: W warm-up steps, then K timed steps in one enqueue
+    tok = int(P.decode_run(h, first, W)[-1]) if W else first
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(ses.compute):
+        e0.record()
+        out = P.decode_run(h, tok, K)
+        e1.record()
+    barrier()
+    dev_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    st = P.get_stats(h)
+    launches = st["kernel_launches_last"]
+    if world > 1:
+        t = torch.tensor([dev_ms], device=f"cuda:{local}")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dev_ms = float(t.item())
+    value = world * K / (dev_ms * 1e-3)
+
+    # ---- end to end: the per-token public call, token id H2D and result D2H every step
+    P.reset(h)
+    first, _ = P.prefill(h, toks, 0)
+    tok = first
+    for _ in range(W):
+        tok, _ = P.decode_step(h, tok, 0)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(K):
+        tok, _ = P.decode_step(h, tok, 0)
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], device=f"cuda:{local}")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = world * K / e2e_s
+
+    # ---- roofline of the dominant kernel (gate/up GEMV), CUDA events around each launch
+    P.set_option(h, P.OPT_PROFILE, 1)
+    for _ in range(3):
+        tok, _ = P.decode_step(h, tok, 0)
+    sp = P.get_stats(h)
+    P.set_option(h, P.OPT_PROFILE, 0)
+    peak, peak_kind = measured_peaks()
+    achieved = sp["dominant_kernel_bytes"] / (sp["dominant_kernel_ms"] * 1e-3) / 1e9 if sp["dominant_kernel_ms"] else None
+    B = 2 if shape.dtype == "bf16" else 4
+    ctx_mid = T + W + K / 2
+    kv_bytes = 2 * shape.n_layers * shape.n_kv_heads * shape.head_dim * B * (ctx_mid + 1)
+    token_bytes = st["weight_bytes_per_token"] + kv_bytes
+    token_gbs = token_bytes / (dev_ms / K * 1e-3) / 1e9
+
+    if rank != 0:
+        ses.close()
+        return
+    # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        v, _, sample = oracle_sample(shape, 4)
+        cpu = {"value": v, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle", "sample": sample}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": shape.dtype, "data": "synthetic",
+        "config": {"workload": workload_name(shape, args), "context": f"{T + W}..{T + W + K}",
+                   "l2": "inputs larger than L2: every step streams %.2f GB of weights" % (st["weight_bytes_per_token"] / 1e9),
+                   "parallelism": "replicas" if world > 1 else "single GPU, N shards emulated",
+                   "graph": bool(st["graph_active"]), "load_s": round(t_load, 1)},
+        "clocks": clocks,
+        "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": 4, "d2h_bytes_per_step": 8},
+        "gpu_launches": launches,
+        "ttft_ms": ttft_ms, "ttft_prompt_tokens": T,
+        "token_roofline": {"bound": "hbm", "bytes_per_token": token_bytes, "achieved": token_gbs, "peak": peak,
+                           "unit": "GB/s", "frac": token_gbs / peak, "peak_kind": peak_kind},
+        "roofline": {"bound": "hbm", "kernel": "gemv_kernel<bf16,2,EPI_SWIGLU> (gate/up + SwiGLU)",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak if achieved else None, "traffic": traffic_from_profile(args.workload),
+                     "bytes_per_launch": sp["dominant_kernel_bytes"], "ms_per_launch": sp["dominant_kernel_ms"],
+                     "launches_timed": sp["dominant_kernel_samples"], "peak_kind": peak_kind},
+        "cpu_baseline": cpu,
+        "tokens_tail": [int(x) for x in out[-4:]],
+    }
+    print(json.dumps(line), flush=True)
+    ses.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=128)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C2", choices=sorted(S.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    shape = S.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, shape)
+    else:
+        run_gpu(args, shape)
+
+
+if __name__ == "__main__":
+    main()
