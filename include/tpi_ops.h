@@ -1,0 +1,89 @@
+/* tpi_ops.h - single-operation entry points of libtpi.so.
+ *
+ * Each call launches one step of the decoder path (the same kernels the model
+ * driver in tpi.h strings together) on caller-provided DEVICE buffers, so that a
+ * step can be checked or timed alone at any shape.  All pointers are DEVICE
+ * pointers unless they say HOST; `stream` is a cudaStream_t (NULL = default
+ * stream).  Calls are asynchronous: they return after the launch.  dtype is a
+ * tpi_dtype (storage type of weights / KV); activations are fp32.
+ * Return value: 0 or a negative tpi_status (see tpi.h).
+ */
+#ifndef TPI_OPS_H
+#define TPI_OPS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Column-sharded gate/up projection with SwiGLU (Eq. 2, inner part):
+ *   act[i*s/N + j] = SiLU(W_gate^i[j,:] . xn) * (W_up^i[j,:] . xn),  xn = xhat * gain.
+ * Wgu: per shard i a [2 s/N][h] matrix whose rows alternate gate_j, up_j; shards
+ * are contiguous.  xhat, gain: float[h]; act: float[s]. */
+int tpi_op_gemv_gateup(int dtype, const void *Wgu, const float *xhat, const float *gain, int h, int s,
+                       int n_shards, float *act, void *stream);
+
+/* Column-sharded QKV projection + rotary embedding + KV append (Eq. 1 inputs,
+ * Algorithm 1 "store (K, V) in KVCache").  Wqkv: per shard i rows
+ * [W_Q^i ; W_K^i ; W_V^i] x h.  pos: int32* current position p.  rope:
+ * float2[max_seq][d/2] = (cos, sin)(p * base^(-2i/d)).  q_out: float[a d]
+ * (rotated).  kcache/vcache: [b][max_seq][d] in dtype; row p is written. */
+int tpi_op_gemv_qkv(int dtype, const void *Wqkv, const float *xhat, const float *gain, int h, int a, int b,
+                    int d, int n_shards, int max_seq, const int32_t *pos, const void *rope, float *q_out,
+                    void *kcache, void *vcache, void *stream);
+
+/* cos/sin table for tpi_op_gemv_qkv: rope[p][i] for p < max_seq, i < d/2 (fp64 inside).
+ * inv_freq_scratch: double[d/2] device scratch the call fills from rope_base. */
+int tpi_op_rope_table(float rope_base, int d, int max_seq, double *inv_freq_scratch, void *rope, void *stream);
+
+/* Row-sharded projection (W_O of Eq. 1 / W_down of Eq. 2): one partial sum per shard,
+ *   partials[i][r] = W^i[r,:] . x[i*Ks : (i+1)*Ks],  W: [N][rows][Ks] contiguous. */
+int tpi_op_gemv_partials(int dtype, const void *W, const float *x, int rows, int Ks, int n_shards,
+                         float *partials, void *stream);
+
+/* The star allreduce of Sec. 3.2 emulated on one GPU, plus the shortcut of Eq. 1-2
+ * and the next norm's statistics:  x <- ((P_0 + P_1) + ... + P_{N-1}) + x;
+ * xhat <- x * rsqrt(mean(x^2) + eps).  partials: float[N][h]; x, xhat: float[h]. */
+int tpi_op_reduce_residual(const float *partials, int n_shards, int h, float eps, float *x, float *xhat,
+                           void *stream);
+
+/* Both of the above back to back: x <- sum_i W^i x_i + x, xhat as above.
+ * scratch: float[n_shards * rows] DEVICE memory owned by the caller (the N partials). */
+int tpi_op_rowshard_project(int dtype, const void *W, const float *x_in, int rows, int Ks, int n_shards,
+                            float eps, float *scratch, float *x, float *xhat, void *stream);
+
+/* Split-K attention of one query position over cache positions 0..*pos (Eq. 1).
+ * q: float[a d] rotated queries; kcache/vcache [b][max_seq][d]; o: float[a d].
+ * scratch: float[tpi_op_attention_scratch_floats(...)]; tickets: uint32[b], zero on entry
+ * (the kernel leaves them zero). */
+size_t tpi_op_attention_scratch_floats(int a, int b, int d, int nsplit);
+int tpi_op_decode_attention(int dtype, const float *q, const void *kcache, const void *vcache,
+                            const int32_t *pos, int a, int b, int d, int max_seq, int nsplit, float *scratch,
+                            uint32_t *tickets, float *o, void *stream);
+
+/* Task head + greedy argmax (Step 4): logits = W_head . (xhat * gain); token =
+ * lowest index of the maximum.  amax_val/amax_idx: scratch of tpi_op_head_blocks(vocab)
+ * entries; ticket: uint32, zero on entry.  token_out: int32[2]; token_out[1] receives the id. */
+int tpi_op_head_blocks(int vocab);
+int tpi_op_head_argmax(int dtype, const void *Whead, const float *xhat, const float *gain, int h, int vocab,
+                       float *logits, float *amax_val, int32_t *amax_idx, uint32_t *ticket,
+                       int32_t *token_out, void *stream);
+
+/* Prompt-pass projection: Y[b][t][o] = sum_k X[b][t][k] W[b][o][k] for n_batch independent
+ * problems (batch = shard for the row-sharded projections), fp32 accumulate.
+ * X: float, row stride ldx, batch stride x_bs; W: dtype, [n_out][K], batch stride w_bs elements;
+ * Y: float, row stride ldy, batch stride y_bs. */
+int tpi_op_gemm(int dtype, const float *X, long long x_bs, int ldx, const void *W, long long w_bs, float *Y,
+                long long y_bs, int ldy, int T, int n_out, int K, int n_batch, void *stream);
+
+/* Causal attention of T query positions [pos0, pos0+T) over cache positions [0, pos0+T).
+ * Q, O: float[T][a][d]. */
+int tpi_op_prefill_attention(int dtype, const float *Q, const void *kcache, const void *vcache, int T, int pos0,
+                             int a, int b, int d, int max_seq, float *O, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TPI_OPS_H */

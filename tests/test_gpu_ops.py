@@ -1,0 +1,249 @@
+"""Kernel-level parity at the workloads' real shapes: each step of the decoder path,
+called alone through the C ABI (tpi_ops.h) on seeded inputs, against the CPU oracle's
+definition of that step (fp64).  Shapes span many tiles and ragged tails."""
+import numpy as np
+import pytest
+
+import tpi_synth as S
+from oracle import llama_oracle as O
+from tests.helpers import rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def T():
+    import torch
+    assert torch.cuda.is_available()
+    return torch
+
+
+_KEEP = []          # device tensors must outlive the asynchronous launches that read them
+
+
+def dev(T, a):
+    """numpy array -> device tensor holding the same bytes (uint16 bf16 bits travel as int16).
+    The tensor is kept alive until the end of the test (see the autouse fixture)."""
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.uint16:
+        a = a.view(np.int16)
+    if a.dtype == np.uint32:
+        a = a.view(np.int32)
+    t = T.from_numpy(a).cuda()
+    _KEEP.append(t)
+    return t
+
+
+@pytest.fixture(autouse=True)
+def _release_device_tensors():
+    yield
+    import torch
+    torch.cuda.synchronize()
+    _KEEP.clear()
+
+
+def dt_of(shape):
+    return 1 if shape.dtype == "bf16" else 0
+
+
+def pack_rows_sharded(w, n):           # row-sharded [h][K] -> [N][h][K/N]
+    h, K = w.shape
+    return np.ascontiguousarray(w.reshape(h, n, K // n).transpose(1, 0, 2))
+
+
+def pack_gate_up(wg, wu, n):           # -> per shard rows gate_0, up_0, gate_1, up_1, ...
+    s, h = wg.shape
+    g = wg.reshape(n, s // n, 1, h)
+    u = wu.reshape(n, s // n, 1, h)
+    return np.ascontiguousarray(np.concatenate([g, u], axis=2).reshape(2 * s, h))
+
+
+@pytest.mark.parametrize("cfg,n_shards", [("C2", 4), ("C1", 2), ("C3", 8)])
+def test_gateup_swiglu(T, cfg, n_shards):
+    import paper_2410_00531_b200.ops as K
+    shape = S.CONFIGS[cfg]
+    h, s = shape.hidden, shape.ffn
+    wg, wu = S.gen_tensor(shape, 1, S.WGATE), S.gen_tensor(shape, 1, S.WUP)
+    gain = S.as_f64(S.gen_tensor(shape, 1, S.FFN_NORM)).astype(np.float32)
+    xhat = S.hidden_state(5, h, 1.0)
+    act = T.empty(s, dtype=T.float32, device="cuda")
+    K.gemv_gateup(dt_of(shape), dev(T, pack_gate_up(wg, wu, n_shards)).data_ptr(), dev(T, xhat).data_ptr(),
+                  dev(T, gain).data_ptr(), h, s, n_shards, act.data_ptr())
+    xn = xhat.astype(np.float64) * gain
+    want = O.silu(S.as_f64(wg) @ xn) * (S.as_f64(wu) @ xn)
+    assert rel_l2(act.cpu().numpy(), want) < 2e-6
+
+
+@pytest.mark.parametrize("cfg,n_shards,which", [("C2", 4, S.WDOWN), ("C2", 4, S.WO), ("C3", 8, S.WO),
+                                                ("C1", 2, S.WDOWN), ("C2", 1, S.WDOWN), ("C2", 2, S.WDOWN)])
+def test_rowshard_partials_and_star_sum(T, cfg, n_shards, which):
+    import paper_2410_00531_b200.ops as K
+    shape = S.CONFIGS[cfg]
+    w = S.gen_tensor(shape, 0, which)
+    h, Kdim = w.shape
+    x_in = S.hidden_state(6, Kdim, 0.7)
+    resid = S.hidden_state(7, h, 0.5)
+    Wd = dev(T, pack_rows_sharded(w, n_shards))
+    part = T.empty((n_shards, h), dtype=T.float32, device="cuda")
+    K.gemv_partials(dt_of(shape), Wd.data_ptr(), dev(T, x_in).data_ptr(), h, Kdim // n_shards, n_shards, part.data_ptr())
+    w64, x64 = S.as_f64(w), x_in.astype(np.float64)
+    cols = Kdim // n_shards
+    want_p = np.stack([w64[:, i * cols:(i + 1) * cols] @ x64[i * cols:(i + 1) * cols] for i in range(n_shards)])
+    assert rel_l2(part.cpu().numpy(), want_p) < 2e-6
+    # allreduce + shortcut + norm statistics in one call, partials in caller scratch
+    x = dev(T, resid.copy())
+    xhat = T.empty(h, dtype=T.float32, device="cuda")
+    scratch = T.empty(n_shards * h, dtype=T.float32, device="cuda")
+    K.rowshard_project(dt_of(shape), Wd.data_ptr(), dev(T, x_in).data_ptr(), h, cols, n_shards, shape.rms_eps,
+                       scratch.data_ptr(), x.data_ptr(), xhat.data_ptr())
+    want_x = w64 @ x64 + resid
+    assert rel_l2(x.cpu().numpy(), want_x) < 2e-6
+    assert rel_l2(xhat.cpu().numpy(), O.rmsnorm(want_x, np.ones(h), shape.rms_eps)) < 2e-6
+    # rank order matters for bit-reproducibility: the device sum equals ((P0 + P1) + ...) + x in fp32
+    p32 = part.cpu().numpy()
+    acc = p32[0].copy()
+    for i in range(1, n_shards):
+        acc = acc + p32[i]
+    assert np.array_equal(x.cpu().numpy(), acc + resid)
+
+
+@pytest.mark.parametrize("cfg,n_shards,p", [("C3", 8, 4095), ("C2", 4, 0), ("C1", 2, 17), ("C5", 8, 8191)])
+def test_qkv_rope_kv_append(T, cfg, n_shards, p):
+    import paper_2410_00531_b200.ops as K
+    shape = S.CONFIGS[cfg]
+    h, a, b, d = shape.hidden, shape.n_heads, shape.n_kv_heads, shape.head_dim
+    max_seq = p + 3
+    wq, wk, wv = (S.gen_tensor(shape, 2, t) for t in (S.WQ, S.WK, S.WV))
+    hps, kps = a // n_shards * d, b // n_shards * d
+    packed = np.concatenate([np.concatenate([wq[i * hps:(i + 1) * hps], wk[i * kps:(i + 1) * kps],
+                                             wv[i * kps:(i + 1) * kps]]) for i in range(n_shards)])
+    gain = S.as_f64(S.gen_tensor(shape, 2, S.ATTN_NORM)).astype(np.float32)
+    xhat = S.hidden_state(8, h, 1.0)
+    esz = T.bfloat16 if shape.dtype == "bf16" else T.float32
+    kc = T.zeros((b, max_seq, d), dtype=esz, device="cuda")
+    vc = T.zeros((b, max_seq, d), dtype=esz, device="cuda")
+    rope = T.empty((max_seq, d // 2, 2), dtype=T.float32, device="cuda")
+    invf = T.empty(d // 2, dtype=T.float64, device="cuda")
+    K.rope_table(shape.rope_base, d, max_seq, invf.data_ptr(), rope.data_ptr())
+    q = T.empty(a * d, dtype=T.float32, device="cuda")
+    pos = T.tensor([p], dtype=T.int32, device="cuda")
+    K.gemv_qkv(dt_of(shape), dev(T, packed).data_ptr(), dev(T, xhat).data_ptr(), dev(T, gain).data_ptr(), h, a, b, d,
+               n_shards, max_seq, pos.data_ptr(), rope.data_ptr(), q.data_ptr(), kc.data_ptr(), vc.data_ptr())
+    xn = xhat.astype(np.float64) * gain
+    pp = np.array([p])
+    q_want = O.rope((S.as_f64(wq) @ xn).reshape(1, a, d), pp, shape.rope_base)[0]
+    k_want = O.rope((S.as_f64(wk) @ xn).reshape(1, b, d), pp, shape.rope_base)[0]
+    v_want = (S.as_f64(wv) @ xn).reshape(b, d)
+    assert rel_l2(q.cpu().numpy(), q_want) < 3e-6
+    kg, vg = kc.float().cpu().numpy(), vc.float().cpu().numpy()
+    tol = 4e-3 if shape.dtype == "bf16" else 3e-6
+    assert rel_l2(kg[:, p], k_want) < tol and rel_l2(vg[:, p], v_want) < tol
+    if shape.dtype == "bf16":       # apart from rare last-bit flips the stored values ARE the RNE-rounded ones
+        assert (kg[:, p] != O.round_bf16(k_want)).mean() < 0.02
+    # nothing but row p was touched
+    kg[:, p] = 0
+    vg[:, p] = 0
+    assert not kg.any() and not vg.any()
+    # the table itself against the fp64 definition
+    th = O.rope_angles(np.arange(max_seq), d, shape.rope_base)
+    r = rope.cpu().numpy()
+    assert np.abs(r[..., 0] - np.cos(th)).max() < 1e-7 and np.abs(r[..., 1] - np.sin(th)).max() < 1e-7
+
+
+@pytest.mark.parametrize("dtype,a,b,d,n,nsplit", [
+    ("bf16", 32, 8, 128, 4096, 34),      # C3: grouped heads, long cache
+    ("bf16", 64, 8, 128, 8192, 37),      # C5 at context 8192
+    ("bf16", 32, 32, 128, 200, 2),       # C2
+    ("f32", 4, 4, 64, 24, 1),            # C1
+    ("f32", 64, 8, 128, 577, 5),         # C4, ragged split
+    ("bf16", 8, 2, 32, 1, 3),            # a single cached position, empty splits
+    ("f32", 8, 4, 64, 33, 8),
+])
+def test_decode_attention(T, dtype, a, b, d, n, nsplit):
+    import paper_2410_00531_b200.ops as K
+    max_seq = n + 5
+    k = S.kv_contents(11, (b, max_seq, d))
+    v = S.kv_contents(12, (b, max_seq, d))
+    if dtype == "bf16":
+        k, v = S.bf16_bits_to_f32(S.f32_to_bf16_bits(k)).reshape(k.shape), S.bf16_bits_to_f32(S.f32_to_bf16_bits(v)).reshape(v.shape)
+    k[:, n:], v[:, n:] = np.nan, np.nan        # nothing beyond the current position may be read
+    q = S.hidden_state(13, a * d, 1.3)
+    tt = T.bfloat16 if dtype == "bf16" else T.float32
+    kc, vc = T.from_numpy(k).cuda().to(tt), T.from_numpy(v).cuda().to(tt)
+    scratch = T.empty(K.attention_scratch_floats(a, b, d, nsplit), dtype=T.float32, device="cuda")
+    tickets = T.zeros(b, dtype=T.int32, device="cuda")
+    o = T.empty(a * d, dtype=T.float32, device="cuda")
+    pos = T.tensor([n - 1], dtype=T.int32, device="cuda")
+    for _ in range(2):                         # twice: the tickets must come back to zero
+        K.decode_attention(1 if dtype == "bf16" else 0, dev(T, q).data_ptr(), kc.data_ptr(), vc.data_ptr(), pos.data_ptr(),
+                           a, b, d, max_seq, nsplit, scratch.data_ptr(), tickets.data_ptr(), o.data_ptr())
+    want = O.attention(q.astype(np.float64).reshape(1, a, d), k[:, :n].astype(np.float64), v[:, :n].astype(np.float64),
+                       np.array([n - 1]))[0]
+    assert rel_l2(o.cpu().numpy(), want) < 5e-6
+    assert not tickets.cpu().numpy().any()
+
+
+@pytest.mark.parametrize("cfg,vocab", [("C2", None), ("C1", None), ("C1", 999)])
+def test_head_argmax(T, cfg, vocab):
+    import paper_2410_00531_b200.ops as K
+    shape = S.CONFIGS[cfg]
+    if vocab:
+        shape = shape.with_(vocab=vocab)
+    h, v = shape.hidden, shape.vocab
+    w = S.gen_tensor(shape, 0, S.HEAD)
+    gain = S.as_f64(S.gen_tensor(shape, 0, S.FINAL_NORM)).astype(np.float32)
+    xhat = S.hidden_state(21, h, 1.0)
+    nb = K.head_blocks(v)
+    logits = T.empty(v, dtype=T.float32, device="cuda")
+    av, ai = T.empty(nb, dtype=T.float32, device="cuda"), T.empty(nb, dtype=T.int32, device="cuda")
+    ticket = T.zeros(1, dtype=T.int32, device="cuda")
+    tok = T.full((2,), -7, dtype=T.int32, device="cuda")
+    wd = dev(T, w)
+    K.head_argmax(dt_of(shape), wd.data_ptr(), dev(T, xhat).data_ptr(), dev(T, gain).data_ptr(), h, v,
+                  logits.data_ptr(), av.data_ptr(), ai.data_ptr(), ticket.data_ptr(), tok.data_ptr())
+    want = S.as_f64(w) @ (xhat.astype(np.float64) * gain)
+    lg = logits.cpu().numpy()
+    assert rel_l2(lg, want) < 2e-6
+    assert int(tok[1]) == int(np.argmax(lg)) and int(ticket[0]) == 0
+    # ties go to the lowest index: duplicate the winning row at a lower and a higher index
+    win = int(np.argmax(lg))
+    w2 = w.copy()
+    lo, hi = (win // 2, min(v - 1, win + 5)) if win > 0 else (0, 5)
+    w2[lo], w2[hi] = w[win], w[win]
+    K.head_argmax(dt_of(shape), dev(T, w2).data_ptr(), dev(T, xhat).data_ptr(), dev(T, gain).data_ptr(), h, v,
+                  logits.data_ptr(), av.data_ptr(), ai.data_ptr(), ticket.data_ptr(), tok.data_ptr())
+    assert int(tok[1]) == min(lo, win)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_gemm_batched_ragged(T, dtype):
+    import paper_2410_00531_b200.ops as K
+    rng = np.random.default_rng(3)
+    Tn, Kd, n_out, nb = 100, 344, 203, 2
+    X = rng.standard_normal((Tn, nb * Kd)).astype(np.float32)           # batch b reads columns [b*Kd, (b+1)*Kd)
+    W = (rng.standard_normal((nb, n_out, Kd)) * 0.02).astype(np.float32)
+    Wst = S.f32_to_bf16_bits(W).reshape(W.shape) if dtype == "bf16" else W
+    Y = T.zeros((nb, Tn, n_out), dtype=T.float32, device="cuda")
+    K.gemm(1 if dtype == "bf16" else 0, dev(T, X).data_ptr(), Kd, nb * Kd, dev(T, Wst).data_ptr(), n_out * Kd,
+           Y.data_ptr(), Tn * n_out, n_out, Tn, n_out, Kd, nb)
+    W64 = S.as_f64(Wst)
+    want = np.stack([X[:, b * Kd:(b + 1) * Kd].astype(np.float64) @ W64[b].T for b in range(nb)])
+    assert rel_l2(Y.cpu().numpy(), want) < 2e-6
+
+
+@pytest.mark.parametrize("dtype,a,b,d,Tq,pos0", [("f32", 4, 4, 64, 16, 0), ("bf16", 8, 2, 128, 37, 20), ("bf16", 8, 1, 32, 5, 0)])
+def test_prefill_attention(T, dtype, a, b, d, Tq, pos0):
+    import paper_2410_00531_b200.ops as K
+    n = pos0 + Tq
+    max_seq = n + 2
+    k, v = S.kv_contents(31, (b, max_seq, d)), S.kv_contents(32, (b, max_seq, d))
+    if dtype == "bf16":
+        k, v = S.bf16_bits_to_f32(S.f32_to_bf16_bits(k)).reshape(k.shape), S.bf16_bits_to_f32(S.f32_to_bf16_bits(v)).reshape(v.shape)
+    q = S.kv_contents(33, (Tq, a, d))
+    tt = T.bfloat16 if dtype == "bf16" else T.float32
+    kc, vc = T.from_numpy(k).cuda().to(tt), T.from_numpy(v).cuda().to(tt)
+    o = T.empty((Tq, a, d), dtype=T.float32, device="cuda")
+    K.prefill_attention(1 if dtype == "bf16" else 0, dev(T, q).data_ptr(), kc.data_ptr(), vc.data_ptr(), Tq, pos0, a, b, d,
+                        max_seq, o.data_ptr())
+    want = O.attention(q.astype(np.float64), k[:, :n].astype(np.float64), v[:, :n].astype(np.float64), np.arange(pos0, n))
+    assert rel_l2(o.cpu().numpy(), want) < 5e-6
