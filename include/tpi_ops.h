@@ -54,6 +54,21 @@ int tpi_op_reduce_residual(const float *partials, int n_shards, int h, float eps
 int tpi_op_rowshard_project(int dtype, const void *W, const float *x_in, int rows, int Ks, int n_shards,
                             float eps, float *scratch, float *x, float *xhat, void *stream);
 
+/* Allocation-free variant of tpi_op_rowshard_project (the paper has no counterpart: it is
+ * an addition for callers that cannot allocate device memory when they need this step,
+ * such as code inside a memory-capped plug-in or a real-time loop where cudaMalloc is
+ * off limits).  Same arguments minus `scratch`: the N partial sums live in an array built
+ * into the library (tpi_op_static_scratch_floats() floats = 256 KiB, held on every GPU that
+ * loads the library until the process exits).  Returns TPI_ERR_NOMEM, with a message in
+ * tpi_last_error(), when n_shards * rows exceeds that size.  The call allocates nothing.
+ * All calls on a GPU share the array and it keeps the previous call's contents (each call
+ * overwrites all it reads, so nothing needs clearing); calls that overlap on the GPU race,
+ * so issue them in one stream order.  The first call on each GPU looks up the array's
+ * device address; make that call before any stream capture begins. */
+size_t tpi_op_static_scratch_floats(void);
+int tpi_op_rowshard_project_static(int dtype, const void *W, const float *x_in, int rows, int Ks,
+                                   int n_shards, float eps, float *x, float *xhat, void *stream);
+
 /* Split-K attention of one query position over cache positions 0..*pos (Eq. 1).
  * q: float[a d] rotated queries; kcache/vcache [b][max_seq][d]; o: float[a d].
  * scratch: float[tpi_op_attention_scratch_floats(...)]; tickets: uint32[b], zero on entry

@@ -41,6 +41,8 @@ static int fail(int code, const char* fmt, ...) {
   } while (0)
 
 extern "C" const char* tpi_last_error(void) { return g_err; }
+// lets the library's other translation units leave a message for tpi_last_error()
+extern "C" void tpi_internal_set_error(const char* msg) { snprintf(g_err, sizeof g_err, "%s", msg ? msg : ""); }
 extern "C" const char* tpi_strerror(int code) {
   switch (code) {
     case TPI_OK: return "ok";

@@ -17,6 +17,8 @@ OPS_SYMBOLS = {
     "tpi_op_gemv_partials": (_I, [_I, _P, _P, _I, _I, _I, _P, _P]),
     "tpi_op_reduce_residual": (_I, [_P, _I, _I, _F, _P, _P, _P]),
     "tpi_op_rowshard_project": (_I, [_I, _P, _P, _I, _I, _I, _F, _P, _P, _P, _P]),
+    "tpi_op_static_scratch_floats": (C.c_size_t, []),
+    "tpi_op_rowshard_project_static": (_I, [_I, _P, _P, _I, _I, _I, _F, _P, _P, _P]),
     "tpi_op_attention_scratch_floats": (C.c_size_t, [_I, _I, _I, _I]),
     "tpi_op_decode_attention": (_I, [_I, _P, _P, _P, _P, _I, _I, _I, _I, _I, _P, _P, _P, _P]),
     "tpi_op_head_blocks": (_I, [_I]),
@@ -61,6 +63,16 @@ def reduce_residual(partials, n_shards, h, eps, x, xhat, stream=None):
 
 def rowshard_project(dtype, W, x_in, rows, Ks, n_shards, eps, scratch, x, xhat, stream=None):
     _check(_ops().tpi_op_rowshard_project(dtype, W, x_in, rows, Ks, n_shards, eps, scratch, x, xhat, stream))
+
+
+def static_scratch_floats() -> int:
+    return int(_ops().tpi_op_static_scratch_floats())
+
+
+def rowshard_project_static(dtype, W, x_in, rows, Ks, n_shards, eps, x, xhat, stream=None):
+    """Like rowshard_project, but the partial sums live in the library's built-in array, so the
+    call needs no scratch buffer (for callers that cannot allocate device memory)."""
+    _check(_ops().tpi_op_rowshard_project_static(dtype, W, x_in, rows, Ks, n_shards, eps, x, xhat, stream))
 
 
 def attention_scratch_floats(a, b, d, nsplit) -> int:
