@@ -54,6 +54,16 @@ int tpi_op_reduce_residual(const float *partials, int n_shards, int h, float eps
 int tpi_op_rowshard_project(int dtype, const void *W, const float *x_in, int rows, int Ks, int n_shards,
                             float eps, float *scratch, float *x, float *xhat, void *stream);
 
+/* The same step as the model driver runs it: the N per-shard partial sums are formed in
+ * registers (shard by shard, rank order) and folded straight into the shortcut, so they never
+ * pass through memory:  x[r] <- ((P_0[r] + P_1[r]) + ... + P_{N-1}[r]) + x[r].  Bit-identical
+ * to tpi_op_rowshard_project.  ss_part: float[tpi_op_rowshard_fused_parts(rows)], receives each
+ * CTA's sum of squares of its new x entries (the next RMSNorm's statistics; unused entries are
+ * zeroed).  The whole x_in must fit in shared memory: n_shards * Ks * 4 <= 200 KiB. */
+int tpi_op_rowshard_fused_parts(int rows);
+int tpi_op_rowshard_fused(int dtype, const void *W, const float *x_in, int rows, int Ks, int n_shards,
+                          float *x, float *ss_part, void *stream);
+
 /* Allocation-free variant of tpi_op_rowshard_project (the paper has no counterpart: it is
  * an addition for callers that cannot allocate device memory when they need this step,
  * such as code inside a memory-capped plug-in or a real-time loop where cudaMalloc is

@@ -471,6 +471,14 @@ extern "C" int tpi_load_model(const tpi_config* cfg, const tpi_resources* res, t
   m->dev = (char*)res->dev_arena;
   m->host = (char*)res->host_arena;
   m->plan.n_shards_max = n_shards > 8 ? n_shards : 8;
+  if (const char* tn = getenv("TPI_TUNE")) {  // "key=value,key=value": kernel tuning knobs (see kernels.h)
+    int k = 0, v = 0, n = 0;
+    while (sscanf(tn, "%d=%d%n", &k, &v, &n) == 2) {
+      set_tuning(k, v);
+      tn += n;
+      if (*tn == ',') ++tn;
+    }
+  }
   if (const char* dl = getenv("TPI_WAIT_DEADLINE_S")) {  // bound on every host-side wait for the device
     const double v = atof(dl);
     if (v > 0) m->wait_deadline_s = v;
@@ -635,19 +643,33 @@ static int enqueue_decode(tpi_model* m, LaunchCtx& lc) {
   unsigned* tickets = dptr<unsigned>(m, p.tickets);
   const size_t qkv_shard = (size_t)(a + 2 * b) / N * d * h;
 
-  CK(launch_embed(lc, dt, m->dev + p.emb, tok_hist, pos, c.vocab, c.max_seq, h, c.rms_eps, x, xhat, dptr<int>(m, p.err)));
+  // The kernel that ends a block leaves the raw residual x plus partial sums of x^2; the GEMV that
+  // starts the next block normalises and applies its own block's gain while staging x.
+  float* ss_part = dptr<float>(m, p.ss_part);
+  const int n_parts = rowshard_fused_parts(h);
+  auto norm_in = [&](const float* gain) { return NormIn{x, gain, ss_part, n_parts, c.rms_eps}; };
+  auto rowshard = [&](const void* W, const float* xin, int Ks, float* tap) -> int {
+    if (rowshard_fused_supported(Ks, N)) {
+      CK(launch_gemv_rowshard_fused(lc, dt, W, (size_t)h * Ks, xin, h, Ks, N, x, ss_part, tap));
+    } else {  // very long shard slices: partial sums through memory, then the sum kernel
+      CK(launch_gemv_partials(lc, dt, W, (size_t)h * Ks, xin, h, Ks, N, partials));
+      CK(launch_reduce_residual(lc, partials, N, h, c.rms_eps, x, xhat, tap, ss_part, n_parts));
+    }
+    return TPI_OK;
+  };
+  CK(launch_embed(lc, dt, m->dev + p.emb, tok_hist, pos, c.vocab, c.max_seq, h, c.rms_eps, x, xhat, ss_part, n_parts,
+                  dptr<int>(m, p.err)));
   for (int l = 0; l < c.n_layers; ++l) {
     BlockRef br;
     // ---- attention block: norm gain | QKV (column-sharded) | O (row-sharded)
     TRY(acquire_block(m, 2 * l, &br));
     void* kc = m->dev + p.kcache + (size_t)l * p.kv_layer_bytes;
     void* vc = m->dev + p.vcache + (size_t)l * p.kv_layer_bytes;
-    CK(launch_gemv_qkv(lc, dt, br.base + bl.off_qkv, qkv_shard, xhat, (const float*)br.base, h, N, a, b, d,
+    CK(launch_gemv_qkv(lc, dt, br.base + bl.off_qkv, qkv_shard, norm_in((const float*)br.base), h, N, a, b, d,
                        c.max_seq, pos, rope, q, kc, vc));
     CK(launch_decode_attention(lc, dt, q, kc, vc, pos, a, b, d, c.max_seq, p.nsplit,
                                dptr<float>(m, p.attn_scratch), tickets, o));
-    CK(launch_gemv_partials(lc, dt, br.base + bl.off_wo, (size_t)h * (a * d / N), o, h, a * d / N, N, partials));
-    CK(launch_reduce_residual(lc, partials, N, h, c.rms_eps, x, xhat, dptr<float>(m, p.taps) + (size_t)(2 * l) * h));
+    TRY(rowshard(br.base + bl.off_wo, o, a * d / N, dptr<float>(m, p.taps) + (size_t)(2 * l) * h));
     TRY(release_block(m, 2 * l));
     // ---- FFN block: norm gain | gate/up (column-sharded) | down (row-sharded)
     TRY(acquire_block(m, 2 * l + 1, &br));
@@ -657,13 +679,12 @@ static int enqueue_decode(tpi_model* m, LaunchCtx& lc) {
       e1 = m->prof_ev[m->prof_used++];
       CK(cudaEventRecord(e0, lc.stream));
     }
-    CK(launch_gemv_gateup(lc, dt, br.base + bl.off_gu, (size_t)2 * (s / N) * h, xhat, (const float*)br.base, h, N, s, act));
+    CK(launch_gemv_gateup(lc, dt, br.base + bl.off_gu, (size_t)2 * (s / N) * h, norm_in((const float*)br.base), h, N, s, act));
     if (e1) CK(cudaEventRecord(e1, lc.stream));
-    CK(launch_gemv_partials(lc, dt, br.base + bl.off_down, (size_t)h * (s / N), act, h, s / N, N, partials));
-    CK(launch_reduce_residual(lc, partials, N, h, c.rms_eps, x, xhat, dptr<float>(m, p.taps) + (size_t)(2 * l + 1) * h));
+    TRY(rowshard(br.base + bl.off_down, act, s / N, dptr<float>(m, p.taps) + (size_t)(2 * l + 1) * h));
     TRY(release_block(m, 2 * l + 1));
   }
-  CK(launch_head_argmax(lc, dt, m->dev + p.head, xhat, dptr<float>(m, p.final_gain), h, c.vocab,
+  CK(launch_head_argmax(lc, dt, m->dev + p.head, norm_in(dptr<float>(m, p.final_gain)), h, c.vocab,
                         dptr<float>(m, p.logits), dptr<float>(m, p.amax_val), dptr<int>(m, p.amax_idx),
                         tickets + b, tok_hist, pos, 1));
   return TPI_OK;
@@ -796,9 +817,13 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
     TRY(release_block(m, 2 * l + 1));
   }
   if (last) {
+    const int n_parts = rowshard_fused_parts(h);
     CK(launch_rmsnorm_stat_row(lc, X + (size_t)(T - 1) * h, h, c.rms_eps, dptr<float>(m, p.x), dptr<float>(m, p.xhat),
+                               dptr<float>(m, p.ss_part), n_parts,
                                dptr<int>(m, p.pos), pos0 + T - 1));
-    CK(launch_head_argmax(lc, dt, m->dev + p.head, dptr<float>(m, p.xhat), dptr<float>(m, p.final_gain), h, c.vocab,
+    CK(launch_head_argmax(lc, dt, m->dev + p.head,
+                          NormIn{dptr<float>(m, p.x), dptr<float>(m, p.final_gain), dptr<float>(m, p.ss_part), n_parts, c.rms_eps},
+                          h, c.vocab,
                           dptr<float>(m, p.logits), dptr<float>(m, p.amax_val), dptr<int>(m, p.amax_idx),
                           dptr<unsigned>(m, p.tickets) + b, dptr<int>(m, p.tok_hist), dptr<int>(m, p.pos), 1));
   }

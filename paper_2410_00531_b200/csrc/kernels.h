@@ -16,23 +16,33 @@ enum { DT_F32 = 0, DT_BF16 = 1 };
 enum : int { DEVERR_NONE = 0, DEVERR_TOKEN_RANGE = 1, DEVERR_POS_RANGE = 2, DEVERR_WAIT_TIMEOUT = 3 };
 static inline size_t dt_size(int dt) { return dt == DT_BF16 ? 2 : 4; }
 
+// Input of a GEMV that starts a block: x is either already normalised (ss_part == nullptr) or the
+// raw residual stream together with the producer's partial sums of squares, in which case the kernel
+// applies x * rsqrt(sum(ss_part) / h + eps) while staging; gain (may be null) is the block's norm gain.
+struct NormIn {
+  const float* x;
+  const float* gain;
+  const float* ss_part;
+  int n_parts;
+  float eps;
+};
+
 // ---------------------------------------------------------------- decode (one position)
 // x = W_emb[tok_hist[*pos]] (fp32); xhat = x * rsqrt(mean(x^2) + eps).
 cudaError_t launch_embed(const LaunchCtx& c, int dt, const void* emb, const int* tok_hist,
                          const int* pos, int vocab, int max_seq, int h, float eps, float* x,
-                         float* xhat, int* err);
+                         float* xhat, float* ss_part, int n_parts, int* err);
 
 // Column-sharded QKV GEMV with fused rotary embedding and KV-cache append (Eq. 1 inputs).
 // Wqkv: shard-major [(a/N + 2b/N) d][h] per shard.  q_out fp32 [a d] (rotated, unscaled).
 cudaError_t launch_gemv_qkv(const LaunchCtx& c, int dt, const void* Wqkv, size_t shard_stride_elems,
-                            const float* xhat, const float* gain, int h, int n_shards, int a, int b,
+                            const NormIn& in, int h, int n_shards, int a, int b,
                             int d, int max_seq, const int* pos, const float2* rope, float* q_out,
                             void* kcache_layer, void* vcache_layer);
 
 // Column-sharded gate/up GEMV (rows interleaved gate_j, up_j) with SwiGLU epilogue (Eq. 2).
 cudaError_t launch_gemv_gateup(const LaunchCtx& c, int dt, const void* Wgu, size_t shard_stride_elems,
-                               const float* xhat, const float* gain, int h, int n_shards, int s,
-                               float* act);
+                               const NormIn& in, int h, int n_shards, int s, float* act);
 
 // Row-sharded GEMV: partials[i][r] = W^i[r, :] . x[i*Ks : (i+1)*Ks]   (per-device partial sums).
 cudaError_t launch_gemv_partials(const LaunchCtx& c, int dt, const void* W, size_t shard_stride_elems,
@@ -40,8 +50,20 @@ cudaError_t launch_gemv_partials(const LaunchCtx& c, int dt, const void* W, size
 
 // The emulated star allreduce + shortcut + the next block's norm statistics:
 // x <- ((P_0 + P_1) + ... + P_{N-1}) + x ; xhat = x * rsqrt(mean(x^2) + eps); tap (may be null) <- x.
+// ss_part (may be null): also publish the sum of squares as ss_part[0], zeros in [1, n_parts).
 cudaError_t launch_reduce_residual(const LaunchCtx& c, const float* partials, int n_shards, int h,
-                                   float eps, float* x, float* xhat, float* tap);
+                                   float eps, float* x, float* xhat, float* tap, float* ss_part,
+                                   int n_parts);
+
+// Row-sharded projection fused with the star sum and the shortcut: x[r] <- ((P_0[r] + P_1[r]) + ...) + x[r]
+// with P_i[r] = W^i[r,:] . x_in[i*Ks:(i+1)*Ks] formed in registers; ss_part[cta] <- sum of squares of the
+// CTA's new entries (rowshard_fused_parts(rows) entries, zeros beyond the grid); tap (may be null) <- new x.
+// Needs the whole x_in in shared memory (N * Ks * 4 <= 200 KiB).
+cudaError_t launch_gemv_rowshard_fused(const LaunchCtx& c, int dt, const void* W, size_t shard_stride_elems,
+                                       const float* x_in, int rows, int Ks, int n_shards, float* x,
+                                       float* ss_part, float* tap);
+int rowshard_fused_parts(int rows);
+bool rowshard_fused_supported(int Ks, int n_shards);
 
 // Split-K attention of one query position over the cache (Eq. 1), grouped heads.
 // scratch: float[b * nsplit * (a/b) * (d + 2)], tickets: unsigned[b] (zero between launches).
@@ -53,9 +75,9 @@ size_t decode_attention_scratch_floats(int a, int b, int d, int nsplit);
 
 // Task head (Step 4): logits = W_head . (xhat * gain), greedy argmax (lowest index on ties);
 // writes tok_hist[*pos + 1] and advances *pos.  amax scratch: >= grid blocks entries.
-cudaError_t launch_head_argmax(const LaunchCtx& c, int dt, const void* Whead, const float* xhat,
-                               const float* gain, int h, int vocab, float* logits, float* amax_val,
-                               int* amax_idx, unsigned* ticket, int* tok_hist, int* pos, int advance);
+cudaError_t launch_head_argmax(const LaunchCtx& c, int dt, const void* Whead, const NormIn& in, int h,
+                               int vocab, float* logits, float* amax_val, int* amax_idx, unsigned* ticket,
+                               int* tok_hist, int* pos, int advance);
 int head_argmax_blocks(int vocab);
 
 // cos/sin table for positions [0, max_seq): table[p][i] = (cos, sin)(p * inv_freq[i]), fp64 inside.
@@ -89,7 +111,11 @@ cudaError_t launch_reduce_residual_rows(const LaunchCtx& c, const float* partial
 // xhat of one row of X (to hand the last position to the decode-style head)
 // (also sets *pos = pos_value when pos is not null)
 cudaError_t launch_rmsnorm_stat_row(const LaunchCtx& c, const float* xrow, int h, float eps, float* x,
-                                    float* xhat, int* pos, int pos_value);
+                                    float* xhat, float* ss_part, int n_parts, int* pos, int pos_value);
+
+// tuning knobs (0: CTAs per SM of the column-sharded GEMVs, 1: of the fused row-sharded GEMVs,
+// 2: L2 prefetch bytes per row before the dependency wait)
+void set_tuning(int key, int value);
 
 // misc
 cudaError_t launch_fill_u32(const LaunchCtx& c, uint32_t* p, size_t n, uint32_t v);

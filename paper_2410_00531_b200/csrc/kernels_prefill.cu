@@ -61,7 +61,8 @@ cudaError_t launch_rmsnorm_rows(const LaunchCtx& c, const float* X, const float*
 }
 
 __global__ void __launch_bounds__(1024) rmsnorm_stat_row_kernel(const float* xrow, int h, float eps, float* x,
-                                                               float* xhat, int* pos, int pos_value) {
+                                                               float* xhat, float* ss_part, int n_parts,
+                                                               int* pos, int pos_value) {
   __shared__ float red[32];
   float ss = 0.f;
   for (int k = threadIdx.x; k < h; k += blockDim.x) {
@@ -72,15 +73,16 @@ __global__ void __launch_bounds__(1024) rmsnorm_stat_row_kernel(const float* xro
   ss = block_sum(ss, red);
   const float r = rsqrtf(ss / (float)h + eps);
   for (int k = threadIdx.x; k < h; k += blockDim.x) xhat[k] = xrow[k] * r;
+  for (int i = threadIdx.x; i < n_parts; i += blockDim.x) ss_part[i] = i ? 0.f : ss;
   if (threadIdx.x == 0 && pos) *pos = pos_value;
 }
 
 cudaError_t launch_rmsnorm_stat_row(const LaunchCtx& c, const float* xrow, int h, float eps, float* x,
-                                    float* xhat, int* pos, int pos_value) {
+                                    float* xhat, float* ss_part, int n_parts, int* pos, int pos_value) {
   LaunchCtx nc = c;
   nc.pdl = false;
-  return launch_kernel(nc, rmsnorm_stat_row_kernel, dim3(1), dim3(1024), 0, xrow, h, eps, x, xhat, pos,
-                       pos_value);
+  return launch_kernel(nc, rmsnorm_stat_row_kernel, dim3(1), dim3(1024), 0, xrow, h, eps, x, xhat, ss_part,
+                       n_parts, pos, pos_value);
 }
 
 // ------------------------------------------------------------------ SIMT GEMM (fp32 accumulate)

@@ -18,7 +18,7 @@ extern "C" int tpi_op_gemv_gateup(int dtype, const void* Wgu, const float* xhat,
                                   int n_shards, float* act, void* stream) {
   if (bad_dtype(dtype) || !Wgu || !xhat || !act || h < 1 || s < 1 || n_shards < 1) return TPI_ERR_INVALID_ARG;
   if (s % n_shards || h % vec_of(dtype) || h % 4) return TPI_ERR_SHAPE;
-  return cu(launch_gemv_gateup(ctx(stream), dtype, Wgu, (size_t)2 * (s / n_shards) * h, xhat, gain, h, n_shards, s, act));
+  return cu(launch_gemv_gateup(ctx(stream), dtype, Wgu, (size_t)2 * (s / n_shards) * h, NormIn{xhat, gain, nullptr, 0, 0.f}, h, n_shards, s, act));
 }
 
 extern "C" int tpi_op_gemv_qkv(int dtype, const void* Wqkv, const float* xhat, const float* gain, int h, int a, int b,
@@ -26,7 +26,7 @@ extern "C" int tpi_op_gemv_qkv(int dtype, const void* Wqkv, const float* xhat, c
                                void* kcache, void* vcache, void* stream) {
   if (bad_dtype(dtype) || !Wqkv || !xhat || !pos || !rope || !q_out || !kcache || !vcache) return TPI_ERR_INVALID_ARG;
   if (a % n_shards || b % n_shards || d % 2 || h % vec_of(dtype) || h % 4) return TPI_ERR_SHAPE;
-  return cu(launch_gemv_qkv(ctx(stream), dtype, Wqkv, (size_t)(a + 2 * b) / n_shards * d * h, xhat, gain, h, n_shards, a,
+  return cu(launch_gemv_qkv(ctx(stream), dtype, Wqkv, (size_t)(a + 2 * b) / n_shards * d * h, NormIn{xhat, gain, nullptr, 0, 0.f}, h, n_shards, a,
                             b, d, max_seq, pos, (const float2*)rope, q_out, kcache, vcache));
 }
 
@@ -52,7 +52,7 @@ extern "C" int tpi_op_gemv_partials(int dtype, const void* W, const float* x, in
 extern "C" int tpi_op_reduce_residual(const float* partials, int n_shards, int h, float eps, float* x, float* xhat,
                                       void* stream) {
   if (!partials || !x || !xhat || n_shards < 1 || h < 1) return TPI_ERR_INVALID_ARG;
-  return cu(launch_reduce_residual(ctx(stream), partials, n_shards, h, eps, x, xhat, nullptr));
+  return cu(launch_reduce_residual(ctx(stream), partials, n_shards, h, eps, x, xhat, nullptr, nullptr, 0));
 }
 
 extern "C" int tpi_op_rowshard_project(int dtype, const void* W, const float* x_in, int rows, int Ks, int n_shards,
@@ -61,6 +61,15 @@ extern "C" int tpi_op_rowshard_project(int dtype, const void* W, const float* x_
   const int rc = tpi_op_gemv_partials(dtype, W, x_in, rows, Ks, n_shards, scratch, stream);
   if (rc) return rc;
   return tpi_op_reduce_residual(scratch, n_shards, rows, eps, x, xhat, stream);
+}
+
+extern "C" int tpi_op_rowshard_fused_parts(int rows) { return rows < 1 ? TPI_ERR_INVALID_ARG : rowshard_fused_parts(rows); }
+
+extern "C" int tpi_op_rowshard_fused(int dtype, const void* W, const float* x_in, int rows, int Ks, int n_shards,
+                                     float* x, float* ss_part, void* stream) {
+  if (bad_dtype(dtype) || !W || !x_in || !x || !ss_part || rows < 1 || Ks < 1 || n_shards < 1) return TPI_ERR_INVALID_ARG;
+  if (Ks % vec_of(dtype) || Ks % 4 || !rowshard_fused_supported(Ks, n_shards)) return TPI_ERR_SHAPE;
+  return cu(launch_gemv_rowshard_fused(ctx(stream), dtype, W, (size_t)rows * Ks, x_in, rows, Ks, n_shards, x, ss_part, nullptr));
 }
 
 extern "C" size_t tpi_op_attention_scratch_floats(int a, int b, int d, int nsplit) {
@@ -89,7 +98,7 @@ extern "C" int tpi_op_head_argmax(int dtype, const void* Whead, const float* xha
   if (h % vec_of(dtype) || h % 4) return TPI_ERR_SHAPE;
   // the kernel writes tok_hist[*pos + 1]; token_out[0] serves as a zero position, token_out[1] gets the id
   if (cudaMemsetAsync(token_out, 0, 4, (cudaStream_t)stream) != cudaSuccess) return TPI_ERR_CUDA;
-  return cu(launch_head_argmax(ctx(stream), dtype, Whead, xhat, gain, h, vocab, logits, amax_val, amax_idx, ticket,
+  return cu(launch_head_argmax(ctx(stream), dtype, Whead, NormIn{xhat, gain, nullptr, 0, 0.f}, h, vocab, logits, amax_val, amax_idx, ticket,
                                token_out, token_out, 0));
 }
 
@@ -107,3 +116,6 @@ extern "C" int tpi_op_prefill_attention(int dtype, const float* Q, const void* k
   const cudaError_t e = launch_prefill_attention(ctx(stream), dtype, Q, kcache, vcache, T, pos0, a, b, d, max_seq, O);
   return e == cudaErrorInvalidValue ? TPI_ERR_SHAPE : cu(e);
 }
+
+// Internal tuning hook (not part of the public interface): see kernels.h set_tuning.
+extern "C" void tpi_internal_tune(int key, int value) { set_tuning(key, value); }

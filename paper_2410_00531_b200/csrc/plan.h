@@ -39,7 +39,7 @@ struct Plan {
   int nsplit, head_blocks, n_shards_max;
   // device arena offsets
   size_t emb, head, final_gain, rope, inv_freq, kcache, vcache, kv_layer_bytes;
-  size_t x, xhat, q, o, act, partials, logits, attn_scratch, amax_val, amax_idx, tickets, tok_hist, pos, err,
+  size_t x, xhat, ss_part, q, o, act, partials, logits, attn_scratch, amax_val, amax_idx, tickets, tok_hist, pos, err,
       taps;
   size_t pX, pXn, pQKV, pQ, pO, pGU, pACT, pPART;
   size_t blocks;      // start of the weight-block region (resident images or window slots)
@@ -49,8 +49,8 @@ struct Plan {
 };
 
 static inline int attn_nsplit(const tpi_config& c) {
-  int by_len = (c.max_seq + 127) / 128;
-  int by_sm = 296 / c.n_kv_heads;
+  int by_len = (c.max_seq + 31) / 32;   // a split covers at least 32 positions
+  int by_sm = 592 / c.n_kv_heads;       // about four CTAs per SM when every split is active
   if (by_sm < 1) by_sm = 1;
   int n = by_len < by_sm ? by_len : by_sm;
   return n < 1 ? 1 : n;
@@ -83,6 +83,7 @@ static inline void make_plan(const tpi_config& c, int n_shards_max, int window_b
   p->vcache = take(L * p->kv_layer_bytes);
   p->x = take(h * 4);
   p->xhat = take(h * 4);
+  p->ss_part = take(h * 4);
   p->q = take(a * d * 4);
   p->o = take(a * d * 4);
   p->act = take(s * 4);

@@ -17,6 +17,8 @@ OPS_SYMBOLS = {
     "tpi_op_gemv_partials": (_I, [_I, _P, _P, _I, _I, _I, _P, _P]),
     "tpi_op_reduce_residual": (_I, [_P, _I, _I, _F, _P, _P, _P]),
     "tpi_op_rowshard_project": (_I, [_I, _P, _P, _I, _I, _I, _F, _P, _P, _P, _P]),
+    "tpi_op_rowshard_fused_parts": (_I, [_I]),
+    "tpi_op_rowshard_fused": (_I, [_I, _P, _P, _I, _I, _I, _P, _P, _P]),
     "tpi_op_static_scratch_floats": (C.c_size_t, []),
     "tpi_op_rowshard_project_static": (_I, [_I, _P, _P, _I, _I, _I, _F, _P, _P, _P]),
     "tpi_op_attention_scratch_floats": (C.c_size_t, [_I, _I, _I, _I]),
@@ -63,6 +65,14 @@ def reduce_residual(partials, n_shards, h, eps, x, xhat, stream=None):
 
 def rowshard_project(dtype, W, x_in, rows, Ks, n_shards, eps, scratch, x, xhat, stream=None):
     _check(_ops().tpi_op_rowshard_project(dtype, W, x_in, rows, Ks, n_shards, eps, scratch, x, xhat, stream))
+
+
+def rowshard_fused_parts(rows) -> int:
+    return _check(_ops().tpi_op_rowshard_fused_parts(rows))
+
+
+def rowshard_fused(dtype, W, x_in, rows, Ks, n_shards, x, ss_part, stream=None):
+    _check(_ops().tpi_op_rowshard_fused(dtype, W, x_in, rows, Ks, n_shards, x, ss_part, stream))
 
 
 def static_scratch_floats() -> int:

@@ -130,3 +130,13 @@ def test_error_codes():
         with pytest.raises(P.TpiError) as e:
             P.set_window(ses.h, 2)                         # resident load kept no host images
         assert e.value.code in (-9, -3)
+
+
+@pytest.mark.parametrize("cfg,n_shards,T", [("C2", 4, 128), ("C3", 8, 200)])
+def test_full_width_reduced_depth(cfg, n_shards, T):
+    """The benchmarked shapes end to end at full width (bf16, launch configuration of bench.py:
+    graph + PDL), depth reduced to 2 layers and the vocabulary to 32000 so that the fp64 oracle
+    finishes in seconds; teacher-forced, token rule applied at every step."""
+    shape = S.CONFIGS[cfg].with_(n_layers=2, vocab=32000)
+    toks, mism = _run_and_compare(shape, n_shards, n_decode=6, prompt_len=T)
+    assert mism <= 3

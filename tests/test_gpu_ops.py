@@ -247,3 +247,30 @@ def test_prefill_attention(T, dtype, a, b, d, Tq, pos0):
                         max_seq, o.data_ptr())
     want = O.attention(q.astype(np.float64), k[:, :n].astype(np.float64), v[:, :n].astype(np.float64), np.arange(pos0, n))
     assert rel_l2(o.cpu().numpy(), want) < 5e-6
+
+
+@pytest.mark.parametrize("cfg,n_shards,which", [("C2", 4, S.WDOWN), ("C2", 4, S.WO), ("C3", 8, S.WO), ("C1", 2, S.WDOWN),
+                                                ("C2", 1, S.WDOWN), ("C5", 8, S.WDOWN), ("C5", 2, S.WDOWN)])
+def test_rowshard_fused_is_bit_identical_to_partials_then_sum(T, cfg, n_shards, which):
+    """The model driver's fused kernel keeps the N partial sums in registers; the result must be the
+    same bits as partial sums through memory followed by the rank-ordered sum kernel."""
+    import paper_2410_00531_b200.ops as K
+    shape = S.CONFIGS[cfg]
+    w = S.gen_tensor(shape, 3, which)
+    h, Kdim = w.shape
+    cols = Kdim // n_shards
+    Wd = dev(T, pack_rows_sharded(w, n_shards))
+    x_in = dev(T, S.hidden_state(16, Kdim, 0.7))
+    resid = S.hidden_state(17, h, 0.5)
+    x_a, x_b = dev(T, resid.copy()), dev(T, resid.copy())
+    xhat = T.empty(h, dtype=T.float32, device="cuda")
+    scratch = T.empty(n_shards * h, dtype=T.float32, device="cuda")
+    K.rowshard_project(dt_of(shape), Wd.data_ptr(), x_in.data_ptr(), h, cols, n_shards, shape.rms_eps,
+                       scratch.data_ptr(), x_a.data_ptr(), xhat.data_ptr())
+    parts = T.empty(K.rowshard_fused_parts(h), dtype=T.float32, device="cuda")
+    K.rowshard_fused(dt_of(shape), Wd.data_ptr(), x_in.data_ptr(), h, cols, n_shards, x_b.data_ptr(), parts.data_ptr())
+    a, b = x_a.cpu().numpy(), x_b.cpu().numpy()
+    assert np.array_equal(a, b)
+    want = S.as_f64(w) @ S.hidden_state(16, Kdim, 0.7).astype(np.float64) + resid
+    assert rel_l2(b, want) < 2e-6
+    assert abs(float(parts.double().sum()) / float((want * want).sum()) - 1) < 1e-5
