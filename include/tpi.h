@@ -173,8 +173,13 @@ int tpi_get_stats(tpi_model *m, tpi_stats *out);
 /* Options: TPI_OPT_GRAPH (1 = replay the decode step as a CUDA graph when all
  * blocks are resident; default 1), TPI_OPT_PDL (1 = programmatic dependent
  * launch between kernels; default 1), TPI_OPT_PROFILE (1 = CUDA events around
- * each gate/up GEMV launch and each window wait; default 0). */
-enum { TPI_OPT_GRAPH = 0, TPI_OPT_PDL = 1, TPI_OPT_PROFILE = 2 };
+ * each gate/up GEMV launch and each window wait; default 0), TPI_OPT_TENSOR (1 =
+ * bf16 models run the prompt pass's projections on the tensor cores with each
+ * fp32 activation split into two bf16 values, hi + lo, so ~16 mantissa bits
+ * survive; 2 = a single bf16 per activation: twice the tensor throughput, but
+ * the rounding alone costs ~1e-2 relative error on the logits after two
+ * layers of the synthetic workloads; 0 = fp32 SIMT GEMM everywhere; default 1). */
+enum { TPI_OPT_GRAPH = 0, TPI_OPT_PDL = 1, TPI_OPT_PROFILE = 2, TPI_OPT_TENSOR = 3 };
 int tpi_set_option(tpi_model *m, int option, int value);
 
 /* Host-only test hook (needs no GPU): drives the window scheduler's ordering

@@ -103,6 +103,18 @@ int tpi_op_head_argmax(int dtype, const void *Whead, const float *xhat, const fl
 int tpi_op_gemm(int dtype, const float *X, long long x_bs, int ldx, const void *W, long long w_bs, float *Y,
                 long long y_bs, int ldy, int T, int n_out, int K, int n_batch, void *stream);
 
+/* The prompt-pass projection on the tensor cores (bf16 configurations): same contraction with bf16
+ * activations, tcgen05.mma with an fp32 accumulator in tensor memory, operands staged by TMA.
+ * A: bf16 [T][lda]; batch b reads K columns starting at column b * a_col_batch (a multiple of 8).
+ * A_lo: NULL, or a second bf16 tensor like A holding bf16(x - A) so that A + A_lo carries ~16 mantissa
+ * bits of the fp32 activations x (each k-block is then multiplied twice onto one accumulator).
+ * W: bf16 [n_batch * w_row_batch][K], batch b uses rows [b * w_row_batch, b * w_row_batch + n_out).
+ * Y: float, row stride ldy (multiple of 4), batch stride y_bs floats.  K must be a multiple of 64.
+ * err_word: int32 DEVICE word, zero on entry; the kernel's bounded waits write 3 there if one runs out. */
+int tpi_op_gemm_bf16(const void *A, const void *A_lo, int lda, int a_col_batch, const void *W, int w_row_batch, float *Y,
+                     long long y_bs, int ldy, int T, int n_out, int K, int n_batch, int32_t *err_word,
+                     void *stream);
+
 /* Causal attention of T query positions [pos0, pos0+T) over cache positions [0, pos0+T).
  * Q, O: float[T][a][d]. */
 int tpi_op_prefill_attention(int dtype, const float *Q, const void *kcache, const void *vcache, int T, int pos0,

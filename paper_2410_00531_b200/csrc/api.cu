@@ -12,6 +12,8 @@
 #include <thread>
 #include <vector>
 
+#include <cuda_bf16.h>
+
 #include "../../include/tpi.h"
 #include "kernels.h"
 #include "plan.h"
@@ -73,7 +75,7 @@ struct tpi_model {
   char* host = nullptr;
   cudaStream_t cs = nullptr, ps = nullptr;
   bool own_cs = false, own_ps = false;
-  int opt_graph = 1, opt_pdl = 1, opt_profile = 0;
+  int opt_graph = 1, opt_pdl = 1, opt_profile = 0, opt_tensor = 1;
   int position = 0;
   // window ring
   Ring ring;
@@ -583,6 +585,7 @@ extern "C" int tpi_set_option(tpi_model* m, int option, int value) {
   switch (option) {
     case TPI_OPT_GRAPH: m->opt_graph = value != 0; break;
     case TPI_OPT_PDL: m->opt_pdl = value != 0; break;
+    case TPI_OPT_TENSOR: m->opt_tensor = value < 0 ? 0 : (value > 2 ? 2 : value); break;
     case TPI_OPT_PROFILE:
       m->opt_profile = value != 0;
       if (value && m->prof_ev.empty()) {
@@ -793,26 +796,42 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
   float* PART = dptr<float>(m, p.pPART);
   const float2* rope = dptr<float2>(m, p.rope);
   const int qkv_cols = (a + 2 * b) * d;
-  CK(launch_embed_rows(lc, dt, m->dev + p.emb, dptr<int>(m, p.tok_hist), pos0, T, c.vocab, h, X, dptr<int>(m, p.err)));
+  const int Ko = a * d / N, Kd = s / N;
+  // bf16 models run the projections on the tensor cores (activations rounded to bf16, fp32 accumulate);
+  // fp32 models, and shapes the tensor-core kernel does not take, use the fp32 SIMT GEMM.
+  const bool tc = m->opt_tensor && dt == TPI_BF16 && gemm_tc_supported(h, h, qkv_cols) && gemm_tc_supported(Ko, a * d, h) &&
+                  gemm_tc_supported(h, h, 2 * s) && gemm_tc_supported(Kd, s, h);
+  const int act_mode = tc ? (m->opt_tensor == 2 ? 1 : 2) : 0;  // 0 fp32, 1 bf16, 2 split bf16 (default)
+  int* err = dptr<int>(m, p.err);
+  // Y[b] = A[:, b*a_col : b*a_col+K] . W[b]^T for n_batch shards (1 for the column-sharded projections)
+  auto proj = [&](const float* A, int lda, int a_col, const void* W, int w_rows_b, float* Y, long long y_bs, int ldy,
+                  int n_out, int K, int n_batch) -> int {
+    if (tc) {  // split mode: the low halves sit T * lda bf16 elements after the high halves
+      const __nv_bfloat16* hi = reinterpret_cast<const __nv_bfloat16*>(A);
+      CK(launch_gemm_tc(lc, hi, act_mode == 2 ? hi + (size_t)T * lda : nullptr, lda, a_col, W, w_rows_b, Y, y_bs, ldy, T,
+                        n_out, K, n_batch, err));
+    }
+    else CK(launch_gemm_simt(lc, dt, A, a_col, lda, W, (long long)w_rows_b * K, Y, y_bs, ldy, T, n_out, K, n_batch));
+    return TPI_OK;
+  };
+  CK(launch_embed_rows(lc, dt, m->dev + p.emb, dptr<int>(m, p.tok_hist), pos0, T, c.vocab, h, X, err));
   for (int l = 0; l < c.n_layers; ++l) {
     BlockRef br;
     TRY(acquire_block(m, 2 * l, &br));
     void* kc = m->dev + p.kcache + (size_t)l * p.kv_layer_bytes;
     void* vc = m->dev + p.vcache + (size_t)l * p.kv_layer_bytes;
-    CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, 0));
-    CK(launch_gemm_simt(lc, dt, Xn, 0, h, br.base + bl.off_qkv, 0, QKV, 0, qkv_cols, T, qkv_cols, h, 1));
+    CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, act_mode));
+    TRY(proj(Xn, h, 0, br.base + bl.off_qkv, qkv_cols, QKV, 0, qkv_cols, qkv_cols, h, 1));
     CK(launch_rope_kv_rows(lc, dt, QKV, T, pos0, N, a, b, d, c.max_seq, rope, Q, kc, vc));
-    CK(launch_prefill_attention(lc, dt, Q, kc, vc, T, pos0, a, b, d, c.max_seq, O));
-    const int Ko = a * d / N;
-    CK(launch_gemm_simt(lc, dt, O, Ko, a * d, br.base + bl.off_wo, (long long)h * Ko, PART, (long long)T * h, h, T, h, Ko, N));
+    CK(launch_prefill_attention(lc, dt, Q, kc, vc, T, pos0, a, b, d, c.max_seq, O, act_mode));
+    TRY(proj(O, a * d, Ko, br.base + bl.off_wo, h, PART, (long long)T * h, h, h, Ko, N));
     CK(launch_reduce_residual_rows(lc, PART, N, T, h, X, last ? dptr<float>(m, p.taps) + (size_t)(2 * l) * h : nullptr));
     TRY(release_block(m, 2 * l));
     TRY(acquire_block(m, 2 * l + 1, &br));
-    CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, 0));
-    CK(launch_gemm_simt(lc, dt, Xn, 0, h, br.base + bl.off_gu, 0, GU, 0, 2 * s, T, 2 * s, h, 1));
-    CK(launch_swiglu_rows(lc, GU, T, s, ACT));
-    const int Kd = s / N;
-    CK(launch_gemm_simt(lc, dt, ACT, Kd, s, br.base + bl.off_down, (long long)h * Kd, PART, (long long)T * h, h, T, h, Kd, N));
+    CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, act_mode));
+    TRY(proj(Xn, h, 0, br.base + bl.off_gu, 2 * s, GU, 0, 2 * s, 2 * s, h, 1));
+    CK(launch_swiglu_rows(lc, GU, T, s, ACT, act_mode));
+    TRY(proj(ACT, s, Kd, br.base + bl.off_down, h, PART, (long long)T * h, h, h, Kd, N));
     CK(launch_reduce_residual_rows(lc, PART, N, T, h, X, last ? dptr<float>(m, p.taps) + (size_t)(2 * l + 1) * h : nullptr));
     TRY(release_block(m, 2 * l + 1));
   }

@@ -87,7 +87,8 @@ cudaError_t launch_rope_table(const LaunchCtx& c, const double* inv_freq, int ma
 // ---------------------------------------------------------------- prefill (T positions)
 cudaError_t launch_embed_rows(const LaunchCtx& c, int dt, const void* emb, const int* tok_hist, int pos0,
                               int T, int vocab, int h, float* X, int* err);
-// Xn[t] = X[t] * rsqrt(mean + eps) * gain   (Xn fp32, or bf16 when out_bf16)
+// Xn[t] = X[t] * rsqrt(mean + eps) * gain.  out_bf16: 0 = fp32; 1 = bf16; 2 = split bf16 (hi at Xn,
+// lo = bf16(v - hi) at Xn + T*h bf16 elements).  The same convention holds for the attention and SwiGLU outputs.
 cudaError_t launch_rmsnorm_rows(const LaunchCtx& c, const float* X, const float* gain, int T, int h,
                                 float eps, void* Xn, int out_bf16);
 // Y[t][o] = sum_k X[t][k] W[o][k] for a batch of `n_batch` independent problems
@@ -95,6 +96,14 @@ cudaError_t launch_rmsnorm_rows(const LaunchCtx& c, const float* X, const float*
 cudaError_t launch_gemm_simt(const LaunchCtx& c, int dt, const float* X, long long x_batch_stride, int ldx,
                              const void* W, long long w_batch_stride_elems, float* Y,
                              long long y_batch_stride, int ldy, int T, int n_out, int K, int n_batch);
+// The same contraction on the tensor cores (bf16 x bf16 -> fp32, tcgen05 + TMA): A is bf16 [T][lda], batch b
+// reads K columns starting at b * a_col_batch; W is bf16 [n_batch * w_row_batch][K]; Y fp32.
+// Needs gemm_tc_supported(K, lda, ldy).  err: device error word (bounded waits report there).
+bool gemm_tc_supported(int K, int a_cols_total, int ldy);
+// A_lo_bf16 (may be null): second bf16 tensor of the same shape with A = A_bf16 + A_lo_bf16 (split activations).
+cudaError_t launch_gemm_tc(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
+                           const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T,
+                           int n_out, int K, int n_batch, int* err);
 // rotate q and k of T positions, append k, v to the cache. QKV rows: [shard][q | k | v] packed as the GEMV.
 cudaError_t launch_rope_kv_rows(const LaunchCtx& c, int dt, const float* QKV, int T, int pos0, int n_shards,
                                 int a, int b, int d, int max_seq, const float2* rope, float* Q,
@@ -102,9 +111,9 @@ cudaError_t launch_rope_kv_rows(const LaunchCtx& c, int dt, const float* QKV, in
 // causal attention of T query positions [pos0, pos0+T) over cache positions [0, pos0+T)
 cudaError_t launch_prefill_attention(const LaunchCtx& c, int dt, const float* Q, const void* kcache_layer,
                                      const void* vcache_layer, int T, int pos0, int a, int b, int d,
-                                     int max_seq, float* O);
+                                     int max_seq, void* O, int out_bf16);
 // act[t][j] = silu(GU[t][2j]) * GU[t][2j+1] per shard-major interleaved rows
-cudaError_t launch_swiglu_rows(const LaunchCtx& c, const float* GU, int T, int s, float* ACT);
+cudaError_t launch_swiglu_rows(const LaunchCtx& c, const float* GU, int T, int s, void* ACT, int out_bf16);
 // X[t] <- sum_i P_i[t] + X[t]; optional tap of the last row
 cudaError_t launch_reduce_residual_rows(const LaunchCtx& c, const float* partials, int n_shards, int T,
                                         int h, float* X, float* tap_last);

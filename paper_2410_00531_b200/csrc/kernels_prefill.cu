@@ -8,6 +8,17 @@
 
 namespace tpi {
 
+// Activation store for the GEMM that follows: MODE 0 fp32, 1 bf16, 2 split bf16 (hi, and lo = v - hi at +lo_off).
+template <int MODE>
+__device__ __forceinline__ void store_act(void* base, size_t i, size_t lo_off, float v) {
+  if (MODE == 0) reinterpret_cast<float*>(base)[i] = v;
+  else {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    reinterpret_cast<__nv_bfloat16*>(base)[i] = hi;
+    if (MODE == 2) reinterpret_cast<__nv_bfloat16*>(base)[lo_off + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
+  }
+}
+
 // ------------------------------------------------------------------ embedding rows
 template <typename WT>
 __global__ void embed_rows_kernel(const WT* emb, const int* tok_hist, int pos0, int vocab, int h, float* X,
@@ -36,7 +47,7 @@ cudaError_t launch_embed_rows(const LaunchCtx& c, int dt, const void* emb, const
 // ------------------------------------------------------------------ RMSNorm rows
 template <int OUT_BF16>
 __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float* X, const float* gain, int h, float eps,
-                                                          void* Xn) {
+                                                          void* Xn, size_t lo_off) {
   __shared__ float red[32];
   const float* x = X + (size_t)blockIdx.x * h;
   float ss = 0.f;
@@ -44,11 +55,7 @@ __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float* X, const
   ss = block_sum(ss, red);
   const float r = rsqrtf(ss / (float)h + eps);
   for (int k = threadIdx.x; k < h; k += blockDim.x) {
-    const float v = x[k] * r * gain[k];
-    if (OUT_BF16)
-      reinterpret_cast<__nv_bfloat16*>(Xn)[(size_t)blockIdx.x * h + k] = __float2bfloat16_rn(v);
-    else
-      reinterpret_cast<float*>(Xn)[(size_t)blockIdx.x * h + k] = v;
+    store_act<OUT_BF16>(Xn, (size_t)blockIdx.x * h + k, lo_off, x[k] * r * gain[k]);
   }
 }
 
@@ -56,8 +63,10 @@ cudaError_t launch_rmsnorm_rows(const LaunchCtx& c, const float* X, const float*
                                 float eps, void* Xn, int out_bf16) {
   LaunchCtx nc = c;
   nc.pdl = false;
-  if (out_bf16) return launch_kernel(nc, rmsnorm_rows_kernel<1>, dim3(T), dim3(256), 0, X, gain, h, eps, Xn);
-  return launch_kernel(nc, rmsnorm_rows_kernel<0>, dim3(T), dim3(256), 0, X, gain, h, eps, Xn);
+  const size_t lo = (size_t)T * h;
+  if (out_bf16 == 2) return launch_kernel(nc, rmsnorm_rows_kernel<2>, dim3(T), dim3(256), 0, X, gain, h, eps, Xn, lo);
+  if (out_bf16) return launch_kernel(nc, rmsnorm_rows_kernel<1>, dim3(T), dim3(256), 0, X, gain, h, eps, Xn, lo);
+  return launch_kernel(nc, rmsnorm_rows_kernel<0>, dim3(T), dim3(256), 0, X, gain, h, eps, Xn, lo);
 }
 
 __global__ void __launch_bounds__(1024) rmsnorm_stat_row_kernel(const float* xrow, int h, float eps, float* x,
@@ -219,10 +228,10 @@ cudaError_t launch_rope_kv_rows(const LaunchCtx& c, int dt, const float* QKV, in
 // One warp = one (query position, head).  Per tile of 32 cached positions: each lane scores one
 // position (full dot product, q broadcast from shared memory), the tile's softmax statistics go
 // through shuffles, then each lane accumulates its d/32 output dims over the tile's values.
-template <typename KT, int D>
+template <typename KT, int D, int OUT_BF16>
 __global__ void __launch_bounds__(128) prefill_attn_kernel(const float* __restrict__ Q, const KT* kc,
                                                            const KT* vc, int T, int pos0, int a, int b,
-                                                           int max_seq, float* O) {
+                                                           int max_seq, void* O, size_t lo_off) {
   constexpr int VEC = Elem<KT>::VEC, DPL = D / 32;
   __shared__ __align__(16) float qs[4][D];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -266,20 +275,23 @@ __global__ void __launch_bounds__(128) prefill_attn_kernel(const float* __restri
       for (int i = 0; i < DPL; ++i) acc[i] = fmaf(wu, Elem<KT>::load(vr + i), acc[i]);
     }
   }
-  float* o = O + ((size_t)t * a + j) * D + lane * DPL;
+  const size_t off = ((size_t)t * a + j) * D + lane * DPL;
 #pragma unroll
-  for (int i = 0; i < DPL; ++i) o[i] = acc[i] / l;
+  for (int i = 0; i < DPL; ++i) store_act<OUT_BF16>(O, off + i, lo_off, acc[i] / l);
 }
 
 cudaError_t launch_prefill_attention(const LaunchCtx& c, int dt, const float* Q, const void* kcache_layer,
                                      const void* vcache_layer, int T, int pos0, int a, int b, int d,
-                                     int max_seq, float* O) {
+                                     int max_seq, void* O, int out_bf16) {
   LaunchCtx nc = c;
   nc.pdl = false;
   dim3 grid((T + 3) / 4, a);
-#define TPI_PA(KT, DD)                                                                                     \
-  return launch_kernel(nc, prefill_attn_kernel<KT, DD>, grid, dim3(128), 0, Q, (const KT*)kcache_layer,     \
-                       (const KT*)vcache_layer, T, pos0, a, b, max_seq, O)
+  const size_t lo = (size_t)T * a * d;
+#define TPI_PA_M(KT, DD, MM)                                                                           \
+  launch_kernel(nc, prefill_attn_kernel<KT, DD, MM>, grid, dim3(128), 0, Q, (const KT*)kcache_layer,   \
+                (const KT*)vcache_layer, T, pos0, a, b, max_seq, O, lo)
+#define TPI_PA(KT, DD) \
+  return out_bf16 == 2 ? TPI_PA_M(KT, DD, 2) : (out_bf16 ? TPI_PA_M(KT, DD, 1) : TPI_PA_M(KT, DD, 0))
   if (dt == DT_BF16) {
     if (d == 128) TPI_PA(__nv_bfloat16, 128);
     if (d == 64) TPI_PA(__nv_bfloat16, 64);
@@ -290,22 +302,27 @@ cudaError_t launch_prefill_attention(const LaunchCtx& c, int dt, const float* Q,
     if (d == 32) TPI_PA(float, 32);
   }
 #undef TPI_PA
+#undef TPI_PA_M
   return cudaErrorInvalidValue;
 }
 
 // ------------------------------------------------------------------ SwiGLU rows
-__global__ void swiglu_rows_kernel(const float* GU, size_t n_pairs, float* ACT) {
+template <int OUT_BF16>
+__global__ void swiglu_rows_kernel(const float* GU, size_t n_pairs, void* ACT) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_pairs) return;
   const float2 gu = reinterpret_cast<const float2*>(GU)[i];
-  ACT[i] = gu.x / (1.f + expf(-gu.x)) * gu.y;
+  store_act<OUT_BF16>(ACT, i, n_pairs, gu.x / (1.f + expf(-gu.x)) * gu.y);
 }
 
-cudaError_t launch_swiglu_rows(const LaunchCtx& c, const float* GU, int T, int s, float* ACT) {
+cudaError_t launch_swiglu_rows(const LaunchCtx& c, const float* GU, int T, int s, void* ACT, int out_bf16) {
   LaunchCtx nc = c;
   nc.pdl = false;
   const size_t n = (size_t)T * s;
-  return launch_kernel(nc, swiglu_rows_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, GU, n, ACT);
+  const dim3 grid((unsigned)((n + 255) / 256));
+  if (out_bf16 == 2) return launch_kernel(nc, swiglu_rows_kernel<2>, grid, dim3(256), 0, GU, n, ACT);
+  if (out_bf16) return launch_kernel(nc, swiglu_rows_kernel<1>, grid, dim3(256), 0, GU, n, ACT);
+  return launch_kernel(nc, swiglu_rows_kernel<0>, grid, dim3(256), 0, GU, n, ACT);
 }
 
 // ------------------------------------------------------------------ allreduce + shortcut, T rows

@@ -109,11 +109,21 @@ extern "C" int tpi_op_gemm(int dtype, const float* X, long long x_bs, int ldx, c
   return cu(launch_gemm_simt(ctx(stream), dtype, X, x_bs, ldx, W, w_bs, Y, y_bs, ldy, T, n_out, K, n_batch));
 }
 
+extern "C" int tpi_op_gemm_bf16(const void* A, const void* A_lo, int lda, int a_col_batch, const void* W, int w_row_batch, float* Y,
+                                long long y_bs, int ldy, int T, int n_out, int K, int n_batch, int32_t* err_word,
+                                void* stream) {
+  if (!A || !W || !Y || !err_word || T < 1 || n_out < 1 || K < 1 || n_batch < 1) return TPI_ERR_INVALID_ARG;
+  if (!gemm_tc_supported(K, lda, ldy) || a_col_batch % 8) return TPI_ERR_SHAPE;
+  const cudaError_t e = launch_gemm_tc(ctx(stream), A, A_lo, lda, a_col_batch, W, w_row_batch, Y, y_bs, ldy, T, n_out, K,
+                                       n_batch, err_word);
+  return e == cudaErrorInvalidValue ? TPI_ERR_SHAPE : cu(e);
+}
+
 extern "C" int tpi_op_prefill_attention(int dtype, const float* Q, const void* kcache, const void* vcache, int T,
                                         int pos0, int a, int b, int d, int max_seq, float* O, void* stream) {
   if (bad_dtype(dtype) || !Q || !kcache || !vcache || !O || T < 1 || pos0 < 0) return TPI_ERR_INVALID_ARG;
   if (a % b) return TPI_ERR_SHAPE;
-  const cudaError_t e = launch_prefill_attention(ctx(stream), dtype, Q, kcache, vcache, T, pos0, a, b, d, max_seq, O);
+  const cudaError_t e = launch_prefill_attention(ctx(stream), dtype, Q, kcache, vcache, T, pos0, a, b, d, max_seq, O, 0);
   return e == cudaErrorInvalidValue ? TPI_ERR_SHAPE : cu(e);
 }
 

@@ -26,6 +26,7 @@ OPS_SYMBOLS = {
     "tpi_op_head_blocks": (_I, [_I]),
     "tpi_op_head_argmax": (_I, [_I, _P, _P, _P, _I, _I, _P, _P, _P, _P, _P, _P]),
     "tpi_op_gemm": (_I, [_I, _P, _LL, _I, _P, _LL, _P, _LL, _I, _I, _I, _I, _I, _P]),
+    "tpi_op_gemm_bf16": (_I, [_P, _P, _I, _I, _P, _I, _P, _LL, _I, _I, _I, _I, _I, _P, _P]),
     "tpi_op_prefill_attention": (_I, [_I, _P, _P, _P, _I, _I, _I, _I, _I, _I, _P, _P]),
 }
 _BOUND = False
@@ -105,6 +106,10 @@ def head_argmax(dtype, Whead, xhat, gain, h, vocab, logits, amax_val, amax_idx, 
 
 def gemm(dtype, X, x_bs, ldx, W, w_bs, Y, y_bs, ldy, T, n_out, K, n_batch, stream=None):
     _check(_ops().tpi_op_gemm(dtype, X, x_bs, ldx, W, w_bs, Y, y_bs, ldy, T, n_out, K, n_batch, stream))
+
+
+def gemm_bf16(A, lda, a_col_batch, W, w_row_batch, Y, y_bs, ldy, T, n_out, K, n_batch, err_word, stream=None, A_lo=None):
+    _check(_ops().tpi_op_gemm_bf16(A, A_lo, lda, a_col_batch, W, w_row_batch, Y, y_bs, ldy, T, n_out, K, n_batch, err_word, stream))
 
 
 def prefill_attention(dtype, Q, kcache, vcache, T, pos0, a, b, d, max_seq, O, stream=None):

@@ -274,3 +274,33 @@ def test_rowshard_fused_is_bit_identical_to_partials_then_sum(T, cfg, n_shards, 
     want = S.as_f64(w) @ S.hidden_state(16, Kdim, 0.7).astype(np.float64) + resid
     assert rel_l2(b, want) < 2e-6
     assert abs(float(parts.double().sum()) / float((want * want).sum()) - 1) < 1e-5
+
+
+@pytest.mark.parametrize("Tn,K,n_out,nb", [(128, 4096, 12288, 1), (100, 4096, 1024, 1), (300, 1024, 4096, 4),
+                                           (128, 2752, 4096, 4), (37, 64, 200, 2), (512, 3584, 640, 8)])
+@pytest.mark.parametrize("split", [False, True])
+def test_gemm_tensor_core_bf16(T, Tn, K, n_out, nb, split):
+    """Prompt-pass projection on tcgen05: bf16 inputs, fp32 accumulation, against fp64 on the same
+    bf16 values.  Batches model the row-sharded projections (batch b reads A's columns b*K..)."""
+    import paper_2410_00531_b200.ops as KK
+    rng = np.random.default_rng(Tn + K)
+    A32 = rng.standard_normal((Tn, nb * K)).astype(np.float32)
+    A = S.f32_to_bf16_bits(A32).reshape(Tn, nb * K)
+    Alo = S.f32_to_bf16_bits(A32 - S.bf16_bits_to_f32(A).reshape(A32.shape)).reshape(Tn, nb * K) if split else None
+    W = S.f32_to_bf16_bits((rng.standard_normal((nb, n_out, K)) * 0.02).astype(np.float32)).reshape(nb, n_out, K)
+    Y = T.full((nb, Tn, n_out), float("nan"), dtype=T.float32, device="cuda")
+    err = T.zeros(1, dtype=T.int32, device="cuda")
+    KK.gemm_bf16(dev(T, A).data_ptr(), nb * K, K, dev(T, W).data_ptr(), n_out, Y.data_ptr(), Tn * n_out, n_out,
+                 Tn, n_out, K, nb, err.data_ptr(), A_lo=dev(T, Alo).data_ptr() if split else None)
+    T.cuda.synchronize()
+    assert int(err[0]) == 0
+    A64, W64 = S.as_f64(A), S.as_f64(W)
+    if split:                       # hi + lo carries the fp32 activation to ~2^-17
+        assert rel_l2(A64 + S.as_f64(Alo), A32) < 2e-5
+        A64 = A64 + S.as_f64(Alo)
+    want = np.stack([A64[:, b * K:(b + 1) * K] @ W64[b].T for b in range(nb)])
+    got = Y.cpu().numpy()
+    assert np.isfinite(got).all()
+    # products of bf16 pairs are exact in fp32; what is left is the tensor core's fp32 accumulation
+    # over K / 16 (split: K / 8) partial sums, observed <= 1e-5
+    assert rel_l2(got, want) < 2e-5
