@@ -842,15 +842,21 @@ cudaError_t launch_reduce_residual(const LaunchCtx& c, const float* partials, in
 // One CTA = (kv head, split).  A "row group" of LPR lanes owns one cached position at a
 // time (LPR * 16 bytes = one K or V row), keeps online-softmax state (m, l, acc) for the GRP
 // query heads of the kv head, and walks the split's positions in batches of P.
+// The split's K and V rows (contiguous in the cache) are first copied to shared memory with
+// cp.async, all requests in flight at once, so the split costs one DRAM round trip instead of
+// one per batch; splits longer than CH positions are walked CH positions at a time.
 template <typename KT, int GRP, int LPR>
-__global__ void __launch_bounds__(128) decode_attn_kernel(const float* __restrict__ q, const KT* kc,
+__global__ void __launch_bounds__(256) decode_attn_kernel(const float* __restrict__ q, const KT* kc,
                                                           const KT* vc, const int* pos, int max_seq,
                                                           int nsplit, float* scratch, unsigned* tickets,
                                                           float* o) {
   constexpr int VEC = Elem<KT>::VEC;
   constexpr int D = LPR * VEC;
-  constexpr int WARPS = 4, RG = 32 / LPR, G = WARPS * RG, P = 4;
+  constexpr int WARPS = 8, RG = 32 / LPR, G = WARPS * RG, P = 4;  // 8 warps: enough warps per scheduler to hide ALU latency
   extern __shared__ __align__(16) float sm[];
+  constexpr int CH = 256 / (int)sizeof(KT);  // positions staged at a time: 128 (bf16) or 64 (fp32)
+  KT* k_s = reinterpret_cast<KT*>(sm);        // [CH][D], then V [CH][D]; reused by the merge buffers below
+  KT* v_s = k_s + CH * D;
   float* sm_m = sm;                 // [G][GRP]
   float* sm_l = sm + G * GRP;       // [G][GRP]
   float* sm_acc = sm + 2 * G * GRP; // [G][GRP][D]
@@ -877,19 +883,36 @@ __global__ void __launch_bounds__(128) decode_attn_kernel(const float* __restric
     m[hh] = -INFINITY;
     l[hh] = 0.f;
   }
-  const KT* kbase = kc + (size_t)g * max_seq * D + sub * VEC;
-  const KT* vbase = vc + (size_t)g * max_seq * D + sub * VEC;
+  const KT* kg = kc + (size_t)g * max_seq * D;
+  const KT* vg = vc + (size_t)g * max_seq * D;
+  const KT* kbase = k_s + sub * VEC;  // rows are addressed relative to the staged window
+  const KT* vbase = v_s + sub * VEC;
 
   // The trip count is the same for every lane of the warp (the loop variable is the CTA-wide batch
   // base), because the score reduction below shuffles across the whole warp.
-  for (int tb = s0; tb < s1; tb += G * P) {
+  for (int w0 = s0; w0 < s1; w0 += CH) {
+  const int wn = min(CH, s1 - w0);  // positions in this window
+  if (w0 != s0) __syncthreads();    // everyone is done reading the previous window
+  {
+    const int n16 = wn * D * (int)sizeof(KT) / 16;  // 16-byte pieces per tensor
+    const char* ksrc = reinterpret_cast<const char*>(kg + (size_t)w0 * D);
+    const char* vsrc = reinterpret_cast<const char*>(vg + (size_t)w0 * D);
+    for (int i = threadIdx.x; i < n16; i += WARPS * 32) {
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(reinterpret_cast<char*>(k_s) + i * 16)), "l"(ksrc + (size_t)i * 16) : "memory");
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(reinterpret_cast<char*>(v_s) + i * 16)), "l"(vsrc + (size_t)i * 16) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+  }
+  for (int tb = 0; tb < wn; tb += G * P) {
     const int t0 = tb + grp_id;
     // the batch's K and V rows are requested together: one DRAM round trip per batch, not two
     uint4 kv[P], vv[P];
 #pragma unroll
     for (int pp = 0; pp < P; ++pp) {
       const int t = t0 + pp * G;
-      const bool in = t < s1;
+      const bool in = t < wn;
       kv[pp] = in ? *reinterpret_cast<const uint4*>(kbase + (size_t)t * D) : make_uint4(0, 0, 0, 0);
       vv[pp] = in ? *reinterpret_cast<const uint4*>(vbase + (size_t)t * D) : make_uint4(0, 0, 0, 0);
     }
@@ -905,7 +928,7 @@ __global__ void __launch_bounds__(128) decode_attn_kernel(const float* __restric
         for (int v = 0; v < VEC; ++v) s = fmaf(qr[hh][v], kf[v], s);
 #pragma unroll
         for (int off = LPR / 2; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
-        sc[pp][hh] = (t0 + pp * G < s1) ? s : -INFINITY;
+        sc[pp][hh] = (t0 + pp * G < wn) ? s : -INFINITY;
       }
     }
 #pragma unroll
@@ -937,6 +960,8 @@ __global__ void __launch_bounds__(128) decode_attn_kernel(const float* __restric
       }
     }
   }
+  }  // windows
+  __syncthreads();  // the merge buffers alias the staged window
   // ---- merge the G row groups of this CTA (fixed order)
 #pragma unroll
   for (int hh = 0; hh < GRP; ++hh) {
@@ -973,18 +998,34 @@ __global__ void __launch_bounds__(128) decode_attn_kernel(const float* __restric
   __threadfence();
   const int nact = (n + chunk - 1) / chunk;  // splits that saw at least one position
   const float* pg = scratch + (size_t)g * nsplit * GRP * (D + 2);
-  for (int e = threadIdx.x; e < GRP * D; e += blockDim.x) {
-    const int hh = e / D, dd = e - hh * D;
+  // weights of the splits first (one exp2 per head and split, kept in shared memory; the row-group
+  // buffers are free by now), then every thread sums its output elements over the splits in split order
+  float* w_s = sm;                       // [GRP][nact] normalised weights
+  __syncthreads();
+  for (int hh = warp; hh < GRP; hh += WARPS) {
     float M = -INFINITY;
-    for (int s = 0; s < nact; ++s) M = fmaxf(M, __ldcg(pg + (size_t)(s * GRP + hh) * (D + 2)));
-    float A = 0.f, L = 0.f;
-    for (int s = 0; s < nact; ++s) {
+    for (int s = lane; s < nact; s += 32) M = fmaxf(M, __ldcg(pg + (size_t)(s * GRP + hh) * (D + 2)));
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, off));
+    float L = 0.f;  // fixed order: lane-strided partial sums, then the warp tree
+    for (int s = lane; s < nact; s += 32) {
       const float* ps = pg + (size_t)(s * GRP + hh) * (D + 2);
       const float w = exp2f(__ldcg(ps) - M);
-      A = fmaf(w, __ldcg(ps + 2 + dd), A);
+      w_s[hh * nact + s] = w;
       L = fmaf(w, __ldcg(ps + 1), L);
     }
-    o[(size_t)(g * GRP + hh) * D + dd] = A / L;
+    L = warp_sum(L);
+    const float inv = 1.f / L;
+    for (int s = lane; s < nact; s += 32) w_s[hh * nact + s] *= inv;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < GRP * D; e += blockDim.x) {
+    const int hh = e / D, dd = e - hh * D;
+    float A = 0.f;
+#pragma unroll 8
+    for (int s = 0; s < nact; ++s)
+      A = fmaf(w_s[hh * nact + s], __ldcg(pg + (size_t)(s * GRP + hh) * (D + 2) + 2 + dd), A);
+    o[(size_t)(g * GRP + hh) * D + dd] = A;
   }
   if (threadIdx.x == 0) tickets[g] = 0u;
 }
@@ -997,16 +1038,18 @@ template <typename KT, int GRP, int LPR>
 static cudaError_t launch_attn_t(const LaunchCtx& c, const float* q, const void* kc, const void* vc,
                                  const int* pos, int b, int max_seq, int nsplit, float* scratch,
                                  unsigned* tickets, float* o) {
-  constexpr int D = LPR * Elem<KT>::VEC, G = 4 * (32 / LPR);
-  const size_t smem = (size_t)(2 * G * GRP + G * GRP * D) * sizeof(float);
+  constexpr int D = LPR * Elem<KT>::VEC, G = 8 * (32 / LPR);
+  size_t smem = (size_t)(2 * G * GRP + G * GRP * D) * sizeof(float);
+  if (smem < (size_t)GRP * nsplit * sizeof(float)) smem = (size_t)GRP * nsplit * sizeof(float);
+  if (smem < (size_t)2 * 256 * D) smem = (size_t)2 * 256 * D;  // K and V windows: 2 x CH x D x sizeof = 512 D bytes
   auto kern = decode_attn_kernel<KT, GRP, LPR>;
   static bool attr_done = false;
-  if (!attr_done && smem > 48 * 1024) {
+  if (smem > 48 * 1024 && !attr_done) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  return launch_kernel(c, kern, dim3(b, nsplit), dim3(128), smem, q, (const KT*)kc, (const KT*)vc, pos,
+  return launch_kernel(c, kern, dim3(b, nsplit), dim3(256), smem, q, (const KT*)kc, (const KT*)vc, pos,
                        max_seq, nsplit, scratch, tickets, o);
 }
 

@@ -49,10 +49,9 @@ struct Plan {
 };
 
 static inline int attn_nsplit(const tpi_config& c) {
-  int by_len = (c.max_seq + 31) / 32;   // a split covers at least 32 positions
-  int by_sm = 592 / c.n_kv_heads;       // about four CTAs per SM when every split is active
-  if (by_sm < 1) by_sm = 1;
-  int n = by_len < by_sm ? by_len : by_sm;
+  // one split per 128 cached positions (what a CTA stages in shared memory in one go), at most 128 splits
+  int n = (c.max_seq + 127) / 128;
+  if (n > 128) n = 128;
   return n < 1 ? 1 : n;
 }
 
