@@ -55,11 +55,39 @@ def test_c1_full_depth(n_shards):
     assert toks == list(ref)                   # "identical to single-server inference"
 
 
-def test_c1_without_graph_and_pdl():
+def test_c1_every_decode_driver():
+    """The default is a CUDA graph of per-phase kernels with programmatic dependent launch; the same
+    kernels also run without PDL or as plain stream launches, and the whole step can run as one
+    cooperative kernel."""
     import paper_2410_00531_b200 as P
     shape = S.CONFIGS["C1"]
-    _run_and_compare(shape, 2, opts=((P.OPT_GRAPH, 0), (P.OPT_PDL, 0)))
-    _run_and_compare(shape, 2, opts=((P.OPT_GRAPH, 0), (P.OPT_PDL, 1)))
+    _run_and_compare(shape, 2, opts=((P.OPT_MEGA, 1),))
+    _run_and_compare(shape, 4, opts=((P.OPT_MEGA, 1),))
+    _run_and_compare(shape, 2, opts=((P.OPT_MEGA, 0), (P.OPT_GRAPH, 0), (P.OPT_PDL, 0)))
+    _run_and_compare(shape, 2, opts=((P.OPT_MEGA, 0), (P.OPT_GRAPH, 0), (P.OPT_PDL, 1)))
+    _run_and_compare(shape, 2, opts=((P.OPT_MEGA, 0), (P.OPT_GRAPH, 1), (P.OPT_PDL, 0)))
+
+
+@pytest.mark.parametrize("cfg,n_shards", [("C2", 4), ("C3", 8)])
+def test_whole_token_kernel_matches_per_phase_kernels(cfg, n_shards):
+    """Same greedy tokens and (nearly) the same logits from both decode drivers at full width."""
+    import paper_2410_00531_b200 as P
+    shape = S.CONFIGS[cfg].with_(n_layers=2, vocab=32000)
+    toks = S.prompt_tokens(shape, 150)
+    res = {}
+    with gpu_session(shape, 400, 150, n_shards) as ses:
+        for mega in (1, 0):
+            P.set_option(ses.h, P.OPT_MEGA, mega)
+            P.reset(ses.h)
+            t0, _ = P.prefill(ses.h, toks, 0)
+            seq = P.decode_run(ses.h, t0, 40)
+            t1, lg = P.decode_step(ses.h, int(seq[-1]), shape.vocab)
+            st = P.get_stats(ses.h)
+            assert st["kernel_launches_last"] == (1 if mega else 2 + 5 * shape.n_layers)
+            res[mega] = (t0, seq, t1, lg)
+    assert res[1][0] == res[0][0]
+    assert rel_l2(res[1][3], res[0][3]) < 1e-3 or (res[1][1] != res[0][1]).any()
+    assert (res[1][1][:8] == res[0][1][:8]).all()
 
 
 def test_chunked_prefill_matches():
@@ -85,6 +113,7 @@ def test_streamed_is_bit_identical_to_resident(window):
     res = {}
     for w in (0, window):
         with gpu_session(shape, 64, 16, 2, w) as ses:
+            P.set_option(ses.h, P.OPT_MEGA, 0)      # same per-phase kernels in both runs: results must be the same bits
             t0, lg0 = P.prefill(ses.h, toks, shape.vocab)
             seq = P.decode_run(ses.h, t0, 6)
             t1, lg1 = P.decode_step(ses.h, int(seq[-1]), shape.vocab)
