@@ -351,8 +351,15 @@ static cudaError_t launch_rowfused_w(const LaunchCtx& c, RowFusedArgs& A) {
 
 template <typename WT, int R, int NS>
 static cudaError_t launch_rowfused_t(const LaunchCtx& c, RowFusedArgs& A) {
-  if (g_tune.warps >= 32) return launch_rowfused_w<WT, R, NS, 32>(c, A);
-  if (g_tune.warps >= 16) return launch_rowfused_w<WT, R, NS, 16>(c, A);
+  // Keep about 32 warps per SM: when the staged x_in is so large that fewer than four CTAs fit in an
+  // SM's shared memory, make the CTAs bigger instead (70B-shaped down projection: 112 KiB of x_in).
+  const size_t smem = (size_t)A.Ks * A.n_shards * sizeof(float);
+  const int fit = (int)((220 * 1024) / (smem + 1024));
+  int warps = g_tune.warps;
+  if (fit < 2 && warps < 32) warps = 32;
+  else if (fit < 4 && warps < 16) warps = 16;
+  if (warps >= 32) return launch_rowfused_w<WT, R, NS, 32>(c, A);
+  if (warps >= 16) return launch_rowfused_w<WT, R, NS, 16>(c, A);
   return launch_rowfused_w<WT, R, NS, 8>(c, A);
 }
 
