@@ -946,7 +946,7 @@ extern "C" int tpi_prefill(tpi_model* m, const int32_t* tokens, int n_tokens, in
   int* io = (int*)(m->host + p.h_io);
   const auto w0 = std::chrono::steady_clock::now();
   int launches = 0;
-  LaunchCtx lc{m->cs, false, &launches};
+  LaunchCtx lc{m->cs, m->opt_pdl != 0 && !m->opt_profile, &launches};
   const int p_begin = m->position;
   for (int t0 = 0; t0 < n_tokens; t0 += c.max_prefill) {
     const int T = n_tokens - t0 < c.max_prefill ? n_tokens - t0 : c.max_prefill;

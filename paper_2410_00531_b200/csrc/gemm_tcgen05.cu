@@ -130,6 +130,9 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_acc = tmem_base_s;
+  // set-up above overlaps the previous kernel's tail; the activations it wrote are needed from here on
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (warp == 0) {
     if (lane == 0) {  // ---- TMA producer
@@ -249,24 +252,44 @@ static cudaError_t launch_tc_t(const LaunchCtx& c, const CUtensorMap& tmA, const
     attr_done = true;
   }
   if (c.launches) ++*c.launches;
-  dim3 grid((a.n_out + BN - 1) / BN, (a.T + kBM - 1) / kBM, n_batch);
-  kern<<<grid, 192, smem, c.stream>>>(tmA, tmAlo, tmW, a);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((a.n_out + BN - 1) / BN, (a.T + kBM - 1) / kBM, n_batch);
+  cfg.blockDim = dim3(192);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = c.stream;
+  cudaLaunchAttribute attr[1];
+  if (c.pdl) {
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  return cudaLaunchKernelEx(&cfg, kern, tmA, tmAlo, tmW, a);
 }
 
 cudaError_t launch_gemm_tc(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
                            const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T,
                            int n_out, int K, int n_batch, int* err) {
-  constexpr int BN = 128;
+  // 128 x 128 tiles, or 128 x 256 when the narrower tiling would need more CTAs than there are SMs
+  // (a wider tile re-reads the activations half as often per weight byte)
+  int nsm = 148, dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&nsm, cudaDevAttrMultiProcessorCount, dev);
+  const long long tiles128 = (long long)((n_out + 127) / 128) * ((T + kBM - 1) / kBM) * n_batch;
+  const int BN = (tiles128 > nsm && n_out >= 256) ? 256 : 128;
   CUtensorMap tmA, tmAlo, tmW;
   // A: [T][lda] (each batch reads K columns starting at batch * a_col_batch); W: [n_batch * w_row_batch][K]
   if (!make_map(&tmA, A_bf16, (uint64_t)lda, (uint64_t)T, (uint64_t)lda, kBM)) return cudaErrorInvalidValue;
   if (!make_map(&tmAlo, A_lo_bf16 ? A_lo_bf16 : A_bf16, (uint64_t)lda, (uint64_t)T, (uint64_t)lda, kBM)) return cudaErrorInvalidValue;
   const uint64_t w_rows = (uint64_t)(n_batch - 1) * w_row_batch + n_out;
-  if (!make_map(&tmW, W_bf16, (uint64_t)K, w_rows, (uint64_t)K, BN)) return cudaErrorInvalidValue;
+  if (!make_map(&tmW, W_bf16, (uint64_t)K, w_rows, (uint64_t)K, (uint32_t)BN)) return cudaErrorInvalidValue;
   GemmTcArgs a{Y, y_batch_stride, ldy, T, n_out, K, a_col_batch, w_row_batch, err};
-  if (A_lo_bf16) return launch_tc_t<BN, 4, 1>(c, tmA, tmAlo, tmW, a, n_batch);
-  return launch_tc_t<BN, 6, 0>(c, tmA, tmAlo, tmW, a, n_batch);
+  if (BN == 256) {
+    if (A_lo_bf16) return launch_tc_t<256, 3, 1>(c, tmA, tmAlo, tmW, a, n_batch);
+    return launch_tc_t<256, 4, 0>(c, tmA, tmAlo, tmW, a, n_batch);
+  }
+  if (A_lo_bf16) return launch_tc_t<128, 4, 1>(c, tmA, tmAlo, tmW, a, n_batch);
+  return launch_tc_t<128, 6, 0>(c, tmA, tmAlo, tmW, a, n_batch);
 }
 
 }  // namespace tpi

@@ -23,6 +23,8 @@ __device__ __forceinline__ void store_act(void* base, size_t i, size_t lo_off, f
 template <typename WT>
 __global__ void embed_rows_kernel(const WT* emb, const int* tok_hist, int pos0, int vocab, int h, float* X,
                                   int* err) {
+  pdl_launch_dependents();
+  pdl_wait();  // inputs come from the previous kernel in the stream
   const int t = blockIdx.x;
   int tok = tok_hist[pos0 + t];
   if (tok < 0 || tok >= vocab) {
@@ -35,8 +37,7 @@ __global__ void embed_rows_kernel(const WT* emb, const int* tok_hist, int pos0, 
 
 cudaError_t launch_embed_rows(const LaunchCtx& c, int dt, const void* emb, const int* tok_hist, int pos0,
                               int T, int vocab, int h, float* X, int* err) {
-  LaunchCtx nc = c;
-  nc.pdl = false;
+  LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
   if (dt == DT_BF16)
     return launch_kernel(nc, embed_rows_kernel<__nv_bfloat16>, dim3(T), dim3(256), 0,
                          (const __nv_bfloat16*)emb, tok_hist, pos0, vocab, h, X, err);
@@ -48,6 +49,8 @@ cudaError_t launch_embed_rows(const LaunchCtx& c, int dt, const void* emb, const
 template <int OUT_BF16>
 __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float* X, const float* gain, int h, float eps,
                                                           void* Xn, size_t lo_off) {
+  pdl_launch_dependents();
+  pdl_wait();  // inputs come from the previous kernel in the stream
   __shared__ float red[32];
   const float* x = X + (size_t)blockIdx.x * h;
   float ss = 0.f;
@@ -61,8 +64,7 @@ __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float* X, const
 
 cudaError_t launch_rmsnorm_rows(const LaunchCtx& c, const float* X, const float* gain, int T, int h,
                                 float eps, void* Xn, int out_bf16) {
-  LaunchCtx nc = c;
-  nc.pdl = false;
+  LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
   const size_t lo = (size_t)T * h;
   if (out_bf16 == 2) return launch_kernel(nc, rmsnorm_rows_kernel<2>, dim3(T), dim3(256), 0, X, gain, h, eps, Xn, lo);
   if (out_bf16) return launch_kernel(nc, rmsnorm_rows_kernel<1>, dim3(T), dim3(256), 0, X, gain, h, eps, Xn, lo);
@@ -72,6 +74,8 @@ cudaError_t launch_rmsnorm_rows(const LaunchCtx& c, const float* X, const float*
 __global__ void __launch_bounds__(1024) rmsnorm_stat_row_kernel(const float* xrow, int h, float eps, float* x,
                                                                float* xhat, float* ss_part, int n_parts,
                                                                int* pos, int pos_value) {
+  pdl_launch_dependents();
+  pdl_wait();  // inputs come from the previous kernel in the stream
   __shared__ float red[32];
   float ss = 0.f;
   for (int k = threadIdx.x; k < h; k += blockDim.x) {
@@ -88,8 +92,7 @@ __global__ void __launch_bounds__(1024) rmsnorm_stat_row_kernel(const float* xro
 
 cudaError_t launch_rmsnorm_stat_row(const LaunchCtx& c, const float* xrow, int h, float eps, float* x,
                                     float* xhat, float* ss_part, int n_parts, int* pos, int pos_value) {
-  LaunchCtx nc = c;
-  nc.pdl = false;
+  LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
   return launch_kernel(nc, rmsnorm_stat_row_kernel, dim3(1), dim3(1024), 0, xrow, h, eps, x, xhat, ss_part,
                        n_parts, pos, pos_value);
 }
@@ -101,6 +104,8 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const float* __restrict_
                                                         const WT* __restrict__ W, long long wbs,
                                                         float* __restrict__ Y, long long ybs, int ldy, int T,
                                                         int n_out, int K) {
+  pdl_launch_dependents();
+  pdl_wait();  // inputs come from the previous kernel in the stream
   constexpr int BM = 64, BN = 64, BK = 16;
   __shared__ __align__(16) float Xs[BK][BM + 4];
   __shared__ __align__(16) float Ws[BK][BN + 4];
@@ -162,8 +167,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const float* __restrict_
 cudaError_t launch_gemm_simt(const LaunchCtx& c, int dt, const float* X, long long x_batch_stride, int ldx,
                              const void* W, long long w_batch_stride_elems, float* Y,
                              long long y_batch_stride, int ldy, int T, int n_out, int K, int n_batch) {
-  LaunchCtx nc = c;
-  nc.pdl = false;
+  LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
   dim3 grid((n_out + 63) / 64, (T + 63) / 64, n_batch);
   if (dt == DT_BF16)
     return launch_kernel(nc, gemm_simt_kernel<__nv_bfloat16>, grid, dim3(256), 0, X, x_batch_stride, ldx,
@@ -177,6 +181,8 @@ cudaError_t launch_gemm_simt(const LaunchCtx& c, int dt, const float* X, long lo
 template <typename WT>
 __global__ void rope_kv_rows_kernel(const float* QKV, int pos0, int n_shards, int a, int b, int d, int max_seq,
                                     const float2* rope, float* Q, WT* kc, WT* vc) {
+  pdl_launch_dependents();
+  pdl_wait();  // inputs come from the previous kernel in the stream
   const int t = blockIdx.x, half = d >> 1;
   const int hps = a / n_shards, kps = b / n_shards;
   const int per_shard = (hps + 2 * kps) * d;
@@ -215,8 +221,7 @@ __global__ void rope_kv_rows_kernel(const float* QKV, int pos0, int n_shards, in
 cudaError_t launch_rope_kv_rows(const LaunchCtx& c, int dt, const float* QKV, int T, int pos0, int n_shards,
                                 int a, int b, int d, int max_seq, const float2* rope, float* Q,
                                 void* kcache_layer, void* vcache_layer) {
-  LaunchCtx nc = c;
-  nc.pdl = false;
+  LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
   if (dt == DT_BF16)
     return launch_kernel(nc, rope_kv_rows_kernel<__nv_bfloat16>, dim3(T), dim3(256), 0, QKV, pos0, n_shards, a,
                          b, d, max_seq, rope, Q, (__nv_bfloat16*)kcache_layer, (__nv_bfloat16*)vcache_layer);
@@ -232,6 +237,8 @@ template <typename KT, int D, int OUT_BF16>
 __global__ void __launch_bounds__(128) prefill_attn_kernel(const float* __restrict__ Q, const KT* kc,
                                                            const KT* vc, int T, int pos0, int a, int b,
                                                            int max_seq, void* O, size_t lo_off) {
+  pdl_launch_dependents();
+  pdl_wait();  // inputs come from the previous kernel in the stream
   constexpr int VEC = Elem<KT>::VEC, DPL = D / 32;
   __shared__ __align__(16) float qs[4][D];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -283,8 +290,7 @@ __global__ void __launch_bounds__(128) prefill_attn_kernel(const float* __restri
 cudaError_t launch_prefill_attention(const LaunchCtx& c, int dt, const float* Q, const void* kcache_layer,
                                      const void* vcache_layer, int T, int pos0, int a, int b, int d,
                                      int max_seq, void* O, int out_bf16) {
-  LaunchCtx nc = c;
-  nc.pdl = false;
+  LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
   dim3 grid((T + 3) / 4, a);
   const size_t lo = (size_t)T * a * d;
 #define TPI_PA_M(KT, DD, MM)                                                                           \
@@ -309,6 +315,8 @@ cudaError_t launch_prefill_attention(const LaunchCtx& c, int dt, const float* Q,
 // ------------------------------------------------------------------ SwiGLU rows
 template <int OUT_BF16>
 __global__ void swiglu_rows_kernel(const float* GU, size_t n_pairs, void* ACT) {
+  pdl_launch_dependents();
+  pdl_wait();  // inputs come from the previous kernel in the stream
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_pairs) return;
   const float2 gu = reinterpret_cast<const float2*>(GU)[i];
@@ -316,8 +324,7 @@ __global__ void swiglu_rows_kernel(const float* GU, size_t n_pairs, void* ACT) {
 }
 
 cudaError_t launch_swiglu_rows(const LaunchCtx& c, const float* GU, int T, int s, void* ACT, int out_bf16) {
-  LaunchCtx nc = c;
-  nc.pdl = false;
+  LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
   const size_t n = (size_t)T * s;
   const dim3 grid((unsigned)((n + 255) / 256));
   if (out_bf16 == 2) return launch_kernel(nc, swiglu_rows_kernel<2>, grid, dim3(256), 0, GU, n, ACT);
@@ -328,6 +335,8 @@ cudaError_t launch_swiglu_rows(const LaunchCtx& c, const float* GU, int T, int s
 // ------------------------------------------------------------------ allreduce + shortcut, T rows
 __global__ void reduce_residual_rows_kernel(const float* __restrict__ partials, int n_shards, int T, int h,
                                             float* X, float* tap_last) {
+  pdl_launch_dependents();
+  pdl_wait();  // inputs come from the previous kernel in the stream
   const size_t n = (size_t)T * h;
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
@@ -340,8 +349,7 @@ __global__ void reduce_residual_rows_kernel(const float* __restrict__ partials, 
 
 cudaError_t launch_reduce_residual_rows(const LaunchCtx& c, const float* partials, int n_shards, int T,
                                         int h, float* X, float* tap_last) {
-  LaunchCtx nc = c;
-  nc.pdl = false;
+  LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
   const size_t n = (size_t)T * h;
   return launch_kernel(nc, reduce_residual_rows_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0,
                        partials, n_shards, T, h, X, tap_last);
@@ -349,18 +357,21 @@ cudaError_t launch_reduce_residual_rows(const LaunchCtx& c, const float* partial
 
 // ------------------------------------------------------------------ misc
 __global__ void fill_u32_kernel(uint32_t* p, size_t n, uint32_t v) {
+  pdl_launch_dependents();
+  pdl_wait();  // inputs come from the previous kernel in the stream
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
     p[i] = v;
 }
 cudaError_t launch_fill_u32(const LaunchCtx& c, uint32_t* p, size_t n, uint32_t v) {
-  LaunchCtx nc = c;
-  nc.pdl = false;
+  LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
   const unsigned blocks = (unsigned)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184);
   return launch_kernel(nc, fill_u32_kernel, dim3(blocks ? blocks : 1), dim3(256), 0, p, n, v);
 }
 
 template <typename WT, int TO_FLOAT>
 __global__ void kv_convert_kernel(WT* cache, float* f, size_t n) {
+  pdl_launch_dependents();
+  pdl_wait();  // inputs come from the previous kernel in the stream
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   if (TO_FLOAT) f[i] = Elem<WT>::load(cache + i);
@@ -368,8 +379,7 @@ __global__ void kv_convert_kernel(WT* cache, float* f, size_t n) {
 }
 cudaError_t launch_kv_convert(const LaunchCtx& c, int dt, void* cache_rows, float* f32_rows, size_t n,
                               int to_float) {
-  LaunchCtx nc = c;
-  nc.pdl = false;
+  LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
   dim3 grid((unsigned)((n + 255) / 256));
   if (dt == DT_BF16) {
     if (to_float) return launch_kernel(nc, kv_convert_kernel<__nv_bfloat16, 1>, grid, dim3(256), 0, (__nv_bfloat16*)cache_rows, f32_rows, n);
