@@ -909,7 +909,10 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
     CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, act_mode));
     TRY(proj(Xn, h, 0, br.base + bl.off_qkv, qkv_cols, QKV, 0, qkv_cols, qkv_cols, h, 1));
     CK(launch_rope_kv_rows(lc, dt, QKV, T, pos0, N, a, b, d, c.max_seq, rope, Q, kc, vc));
-    CK(launch_prefill_attention(lc, dt, Q, kc, vc, T, pos0, a, b, d, c.max_seq, O, act_mode));
+    if (m->opt_tensor && prefill_attention_mma_supported(dt, d))
+      CK(launch_prefill_attention_mma(lc, Q, kc, vc, T, pos0, a, b, d, c.max_seq, O, act_mode));
+    else
+      CK(launch_prefill_attention(lc, dt, Q, kc, vc, T, pos0, a, b, d, c.max_seq, O, act_mode));
     TRY(proj(O, a * d, Ko, br.base + bl.off_wo, h, PART, (long long)T * h, h, h, Ko, N));
     CK(launch_reduce_residual_rows(lc, PART, N, T, h, X, last ? dptr<float>(m, p.taps) + (size_t)(2 * l) * h : nullptr));
     TRY(release_block(m, 2 * l));

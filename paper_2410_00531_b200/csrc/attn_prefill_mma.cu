@@ -1,0 +1,253 @@
+// Causal attention of the prompt pass on tensor cores (bf16 KV cache): Eq. 1's softmax(QK^T/sqrt d)V for
+// T query positions at once.  One CTA = 64 queries of one head (4 warps x 16 rows); keys are walked in
+// tiles of 64 staged in shared memory (cp.async, two stages, XOR-swizzled 16-byte chunks); S = QK^T and
+// O += PV run on mma.sync m16n8k16 (bf16 inputs, fp32 accumulate) with an online softmax in between.
+// K and V are exact bf16 (the cache's storage type); the fp32 queries and the softmax weights are each
+// split into bf16 hi + lo and multiplied twice, so the result keeps fp32-level accuracy.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "kernels.h"
+#include "launch.cuh"
+
+namespace tpi {
+
+namespace {
+
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// (x, y) -> packed bf16 pair of the rounded values, and the pair of the remainders
+__device__ __forceinline__ void split_pack(float x, float y, uint32_t& hi, uint32_t& lo) {
+  const __nv_bfloat16 hx = __float2bfloat16_rn(x), hy = __float2bfloat16_rn(y);
+  const __nv_bfloat162 h = __halves2bfloat162(hx, hy);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(x - __bfloat162float(hx), y - __bfloat162float(hy));
+  hi = *reinterpret_cast<const uint32_t*>(&h);
+  lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+
+template <int MODE>
+__device__ __forceinline__ void store_out(void* base, size_t i, size_t lo_off, float v) {
+  if (MODE == 0) reinterpret_cast<float*>(base)[i] = v;
+  else {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    reinterpret_cast<__nv_bfloat16*>(base)[i] = hi;
+    if (MODE == 2) reinterpret_cast<__nv_bfloat16*>(base)[lo_off + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
+  }
+}
+
+constexpr int QB = 64, KB = 64;
+
+// byte offset of 16-byte chunk c of row r in a tile whose rows hold D bf16 (chunks XOR-swizzled in groups of 8)
+template <int D>
+__device__ __forceinline__ uint32_t tile_off(int r, int c) {
+  return (uint32_t)(r * (D * 2) + (((c & ~7) | ((c ^ r) & 7)) << 4));
+}
+
+template <int D, int MODE>
+__global__ void __launch_bounds__(128) prefill_attn_mma_kernel(const float* __restrict__ Q, const __nv_bfloat16* kc,
+                                                               const __nv_bfloat16* vc, int T, int pos0, int a, int b,
+                                                               int max_seq, void* O, size_t lo_off) {
+  constexpr int KS = D / 16;       // k-steps of the QK^T contraction
+  constexpr int ND = D / 8;        // 8-wide output blocks of O
+  constexpr int CPR = D / 8;       // 16-byte chunks per row
+  constexpr int TILE = KB * D * 2; // bytes of one K (or V) tile
+  extern __shared__ __align__(128) uint8_t smem[];  // [2 stages][K tile | V tile]
+  pdl_launch_dependents();
+  pdl_wait();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  const int j = blockIdx.y, kvh = j / (a / b);
+  const int q0 = blockIdx.x * QB;                      // first query row of the CTA
+  const int row_lo = q0 + warp * 16 + g, row_hi = row_lo + 8;
+  const int n_keys = min(pos0 + min(q0 + QB, T), pos0 + T);  // keys any row of this CTA may see
+  const __nv_bfloat16* kg = kc + (size_t)kvh * max_seq * D;
+  const __nv_bfloat16* vg = vc + (size_t)kvh * max_seq * D;
+  const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
+
+  auto stage_tile = [&](int stage, int k0) {
+    // 64 rows x CPR chunks for K and for V; rows beyond the cache's valid range are zero-filled
+    for (int i = threadIdx.x; i < KB * CPR; i += 128) {
+      const int r = i / CPR, c = i - r * CPR;
+      const uint32_t dk = smem_base + stage * 2 * TILE + tile_off<D>(r, c);
+      const uint32_t dv = dk + TILE;
+      if (k0 + r < n_keys) {
+        const size_t src = (size_t)(k0 + r) * D + c * 8;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dk), "l"(kg + src) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dv), "l"(vg + src) : "memory");
+      } else {
+        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(dk), "r"(0u) : "memory");
+        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(dv), "r"(0u) : "memory");
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+
+  // ---- Q fragments (scaled into the log2 domain, split hi/lo)
+  const float qscale = 1.4426950408889634f * rsqrtf((float)D);
+  uint32_t qh[KS][4], ql[KS][4];
+  {
+    const float* q_lo = Q + ((size_t)min(row_lo, T - 1) * a + j) * D;
+    const float* q_hi = Q + ((size_t)min(row_hi, T - 1) * a + j) * D;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      const float2 v0 = *reinterpret_cast<const float2*>(q_lo + ks * 16 + 2 * t);
+      const float2 v1 = *reinterpret_cast<const float2*>(q_hi + ks * 16 + 2 * t);
+      const float2 v2 = *reinterpret_cast<const float2*>(q_lo + ks * 16 + 8 + 2 * t);
+      const float2 v3 = *reinterpret_cast<const float2*>(q_hi + ks * 16 + 8 + 2 * t);
+      split_pack(v0.x * qscale, v0.y * qscale, qh[ks][0], ql[ks][0]);
+      split_pack(v1.x * qscale, v1.y * qscale, qh[ks][1], ql[ks][1]);
+      split_pack(v2.x * qscale, v2.y * qscale, qh[ks][2], ql[ks][2]);
+      split_pack(v3.x * qscale, v3.y * qscale, qh[ks][3], ql[ks][3]);
+    }
+  }
+  float o[ND][4];
+#pragma unroll
+  for (int nd = 0; nd < ND; ++nd) { o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f; }
+  float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+  const int qpos_lo = pos0 + row_lo, qpos_hi = pos0 + row_hi;
+
+  const int n_tiles = (n_keys + KB - 1) / KB;
+  stage_tile(0, 0);
+  for (int kt = 0; kt < n_tiles; ++kt) {
+    const int k0 = kt * KB, stage = kt & 1;
+    if (kt + 1 < n_tiles) {
+      stage_tile(stage ^ 1, k0 + KB);  // next tile streams in while this one is used
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();
+    const uint32_t ks_base = smem_base + stage * 2 * TILE, vs_base = ks_base + TILE;
+
+    // ---- S = Q K^T for this warp's 16 rows x 64 keys
+    float s[KB / 8][4];
+#pragma unroll
+    for (int nb = 0; nb < KB / 8; ++nb) {
+      s[nb][0] = s[nb][1] = s[nb][2] = s[nb][3] = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < KS; ks += 2) {
+        uint32_t kb[4];
+        ldsm_x4(kb, ks_base + tile_off<D>(nb * 8 + (lane & 7), ks * 2 + (lane >> 3)));
+        mma_bf16(s[nb], qh[ks], kb[0], kb[1]);
+        mma_bf16(s[nb], ql[ks], kb[0], kb[1]);
+        mma_bf16(s[nb], qh[ks + 1], kb[2], kb[3]);
+        mma_bf16(s[nb], ql[ks + 1], kb[2], kb[3]);
+      }
+    }
+    // ---- causal mask + online softmax (rows g and g + 8 of the warp's block)
+    float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+    for (int nb = 0; nb < KB / 8; ++nb) {
+      const int key = k0 + nb * 8 + 2 * t;
+      if (key > qpos_lo) s[nb][0] = -INFINITY;
+      if (key + 1 > qpos_lo) s[nb][1] = -INFINITY;
+      if (key > qpos_hi) s[nb][2] = -INFINITY;
+      if (key + 1 > qpos_hi) s[nb][3] = -INFINITY;
+      mx_lo = fmaxf(mx_lo, fmaxf(s[nb][0], s[nb][1]));
+      mx_hi = fmaxf(mx_hi, fmaxf(s[nb][2], s[nb][3]));
+    }
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xFFFFFFFFu, mx_lo, 1));
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xFFFFFFFFu, mx_lo, 2));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xFFFFFFFFu, mx_hi, 1));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xFFFFFFFFu, mx_hi, 2));
+    const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+    const float ref_lo = (mn_lo == -INFINITY) ? 0.f : mn_lo, ref_hi = (mn_hi == -INFINITY) ? 0.f : mn_hi;
+    const float sc_lo = exp2f(m_lo - ref_lo), sc_hi = exp2f(m_hi - ref_hi);
+    m_lo = mn_lo;
+    m_hi = mn_hi;
+    l_lo *= sc_lo;
+    l_hi *= sc_hi;
+#pragma unroll
+    for (int nd = 0; nd < ND; ++nd) { o[nd][0] *= sc_lo; o[nd][1] *= sc_lo; o[nd][2] *= sc_hi; o[nd][3] *= sc_hi; }
+    uint32_t ph[KB / 16][4], pl[KB / 16][4];  // P as A-operand fragments: k-step kk covers key blocks 2kk, 2kk+1
+#pragma unroll
+    for (int nb = 0; nb < KB / 8; ++nb) {
+      const float p0 = exp2f(s[nb][0] - ref_lo), p1 = exp2f(s[nb][1] - ref_lo);
+      const float p2 = exp2f(s[nb][2] - ref_hi), p3 = exp2f(s[nb][3] - ref_hi);
+      l_lo += p0 + p1;
+      l_hi += p2 + p3;
+      const int kk = nb >> 1, half = nb & 1;
+      split_pack(p0, p1, ph[kk][half * 2 + 0], pl[kk][half * 2 + 0]);
+      split_pack(p2, p3, ph[kk][half * 2 + 1], pl[kk][half * 2 + 1]);
+    }
+    // ---- O += P V
+#pragma unroll
+    for (int kk = 0; kk < KB / 16; ++kk) {
+#pragma unroll
+      for (int nd = 0; nd < ND; nd += 2) {
+        uint32_t vb[4];
+        ldsm_x4_trans(vb, vs_base + tile_off<D>(kk * 16 + ((lane >> 3) & 1) * 8 + (lane & 7), nd + (lane >> 4)));
+        mma_bf16(o[nd], ph[kk], vb[0], vb[1]);
+        mma_bf16(o[nd], pl[kk], vb[0], vb[1]);
+        mma_bf16(o[nd + 1], ph[kk], vb[2], vb[3]);
+        mma_bf16(o[nd + 1], pl[kk], vb[2], vb[3]);
+      }
+    }
+    __syncthreads();  // the stage is overwritten two iterations from now
+  }
+  // ---- normalise and store
+  l_lo += __shfl_xor_sync(0xFFFFFFFFu, l_lo, 1);
+  l_lo += __shfl_xor_sync(0xFFFFFFFFu, l_lo, 2);
+  l_hi += __shfl_xor_sync(0xFFFFFFFFu, l_hi, 1);
+  l_hi += __shfl_xor_sync(0xFFFFFFFFu, l_hi, 2);
+  const float inv_lo = 1.f / l_lo, inv_hi = 1.f / l_hi;
+#pragma unroll
+  for (int nd = 0; nd < ND; ++nd) {
+    const int col = nd * 8 + 2 * t;
+    if (row_lo < T) {
+      const size_t i = ((size_t)row_lo * a + j) * D + col;
+      store_out<MODE>(O, i, lo_off, o[nd][0] * inv_lo);
+      store_out<MODE>(O, i + 1, lo_off, o[nd][1] * inv_lo);
+    }
+    if (row_hi < T) {
+      const size_t i = ((size_t)row_hi * a + j) * D + col;
+      store_out<MODE>(O, i, lo_off, o[nd][2] * inv_hi);
+      store_out<MODE>(O, i + 1, lo_off, o[nd][3] * inv_hi);
+    }
+  }
+}
+
+template <int D, int MODE>
+cudaError_t launch_t(const LaunchCtx& c, const float* Q, const void* kc, const void* vc, int T, int pos0, int a, int b,
+                     int max_seq, void* O) {
+  auto kern = prefill_attn_mma_kernel<D, MODE>;
+  const size_t smem = (size_t)2 * 2 * KB * D * 2;
+  static bool attr_done = false;
+  if (!attr_done && smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  return launch_kernel(c, kern, dim3((T + QB - 1) / QB, a), dim3(128), smem, Q, (const __nv_bfloat16*)kc,
+                       (const __nv_bfloat16*)vc, T, pos0, a, b, max_seq, O, (size_t)T * a * D);
+}
+
+}  // namespace
+
+bool prefill_attention_mma_supported(int dt, int d) { return dt == DT_BF16 && (d == 128 || d == 64); }
+
+cudaError_t launch_prefill_attention_mma(const LaunchCtx& c, const float* Q, const void* kcache_layer,
+                                         const void* vcache_layer, int T, int pos0, int a, int b, int d, int max_seq,
+                                         void* O, int out_mode) {
+#define TPI_AM(DD)                                                                                         \
+  return out_mode == 2 ? launch_t<DD, 2>(c, Q, kcache_layer, vcache_layer, T, pos0, a, b, max_seq, O)       \
+         : out_mode == 1 ? launch_t<DD, 1>(c, Q, kcache_layer, vcache_layer, T, pos0, a, b, max_seq, O)     \
+                         : launch_t<DD, 0>(c, Q, kcache_layer, vcache_layer, T, pos0, a, b, max_seq, O)
+  if (d == 128) TPI_AM(128);
+  if (d == 64) TPI_AM(64);
+#undef TPI_AM
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace tpi

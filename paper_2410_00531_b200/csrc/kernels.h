@@ -112,6 +112,11 @@ cudaError_t launch_rope_kv_rows(const LaunchCtx& c, int dt, const float* QKV, in
 cudaError_t launch_prefill_attention(const LaunchCtx& c, int dt, const float* Q, const void* kcache_layer,
                                      const void* vcache_layer, int T, int pos0, int a, int b, int d,
                                      int max_seq, void* O, int out_bf16);
+// the same on tensor cores (mma.sync m16n8k16) for a bf16 cache with head dim 64 or 128; out_mode as out_bf16 above
+bool prefill_attention_mma_supported(int dt, int d);
+cudaError_t launch_prefill_attention_mma(const LaunchCtx& c, const float* Q, const void* kcache_layer,
+                                         const void* vcache_layer, int T, int pos0, int a, int b, int d, int max_seq,
+                                         void* O, int out_mode);
 // act[t][j] = silu(GU[t][2j]) * GU[t][2j+1] per shard-major interleaved rows
 cudaError_t launch_swiglu_rows(const LaunchCtx& c, const float* GU, int T, int s, void* ACT, int out_bf16);
 // X[t] <- sum_i P_i[t] + X[t]; optional tap of the last row

@@ -231,7 +231,9 @@ def test_gemm_batched_ragged(T, dtype):
     assert rel_l2(Y.cpu().numpy(), want) < 2e-6
 
 
-@pytest.mark.parametrize("dtype,a,b,d,Tq,pos0", [("f32", 4, 4, 64, 16, 0), ("bf16", 8, 2, 128, 37, 20), ("bf16", 8, 1, 32, 5, 0)])
+@pytest.mark.parametrize("dtype,a,b,d,Tq,pos0", [("f32", 4, 4, 64, 16, 0), ("bf16", 8, 2, 128, 37, 20), ("bf16", 8, 1, 32, 5, 0),
+                                                    ("bf16", 4, 4, 128, 200, 0), ("bf16", 8, 2, 64, 130, 77), ("bf16", 2, 1, 128, 64, 64),
+                                                    ("bf16", 4, 2, 128, 1, 300)])
 def test_prefill_attention(T, dtype, a, b, d, Tq, pos0):
     import paper_2410_00531_b200.ops as K
     n = pos0 + Tq
@@ -246,7 +248,8 @@ def test_prefill_attention(T, dtype, a, b, d, Tq, pos0):
     K.prefill_attention(1 if dtype == "bf16" else 0, dev(T, q).data_ptr(), kc.data_ptr(), vc.data_ptr(), Tq, pos0, a, b, d,
                         max_seq, o.data_ptr())
     want = O.attention(q.astype(np.float64), k[:, :n].astype(np.float64), v[:, :n].astype(np.float64), np.arange(pos0, n))
-    assert rel_l2(o.cpu().numpy(), want) < 5e-6
+    # bf16 caches with d = 64 / 128 run on tensor cores with split-bf16 queries and weights (~2^-17 per operand)
+    assert rel_l2(o.cpu().numpy(), want) < (2e-5 if dtype == "bf16" else 5e-6)
 
 
 @pytest.mark.parametrize("cfg,n_shards,which", [("C2", 4, S.WDOWN), ("C2", 4, S.WO), ("C3", 8, S.WO), ("C1", 2, S.WDOWN),
