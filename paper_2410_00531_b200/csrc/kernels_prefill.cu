@@ -47,7 +47,7 @@ cudaError_t launch_embed_rows(const LaunchCtx& c, int dt, const void* emb, const
 
 // ------------------------------------------------------------------ RMSNorm rows
 template <int OUT_BF16>
-__global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float* X, const float* gain, int h, float eps,
+__global__ void __launch_bounds__(1024) rmsnorm_rows_kernel(const float* X, const float* gain, int h, float eps,
                                                           void* Xn, size_t lo_off) {
   pdl_launch_dependents();
   pdl_wait();  // inputs come from the previous kernel in the stream
@@ -66,9 +66,9 @@ cudaError_t launch_rmsnorm_rows(const LaunchCtx& c, const float* X, const float*
                                 float eps, void* Xn, int out_bf16) {
   LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
   const size_t lo = (size_t)T * h;
-  if (out_bf16 == 2) return launch_kernel(nc, rmsnorm_rows_kernel<2>, dim3(T), dim3(256), 0, X, gain, h, eps, Xn, lo);
-  if (out_bf16) return launch_kernel(nc, rmsnorm_rows_kernel<1>, dim3(T), dim3(256), 0, X, gain, h, eps, Xn, lo);
-  return launch_kernel(nc, rmsnorm_rows_kernel<0>, dim3(T), dim3(256), 0, X, gain, h, eps, Xn, lo);
+  if (out_bf16 == 2) return launch_kernel(nc, rmsnorm_rows_kernel<2>, dim3(T), dim3(h >= 4096 ? 1024 : 256), 0, X, gain, h, eps, Xn, lo);
+  if (out_bf16) return launch_kernel(nc, rmsnorm_rows_kernel<1>, dim3(T), dim3(h >= 4096 ? 1024 : 256), 0, X, gain, h, eps, Xn, lo);
+  return launch_kernel(nc, rmsnorm_rows_kernel<0>, dim3(T), dim3(h >= 4096 ? 1024 : 256), 0, X, gain, h, eps, Xn, lo);
 }
 
 __global__ void __launch_bounds__(1024) rmsnorm_stat_row_kernel(const float* xrow, int h, float eps, float* x,
@@ -189,7 +189,7 @@ __global__ void rope_kv_rows_kernel(const float* QKV, int pos0, int n_shards, in
   const float* row = QKV + (size_t)t * per_shard * n_shards;
   const int p = pos0 + t;
   const int pairs = (a + b) * half;  // rotary pairs of q and k
-  for (int e = threadIdx.x; e < pairs + b * d; e += blockDim.x) {
+  for (int e = blockIdx.y * blockDim.x + threadIdx.x; e < pairs + b * d; e += gridDim.y * blockDim.x) {
     if (e < pairs) {
       const int head = e / half, ii = e - head * half;  // heads 0..a-1 are q, a..a+b-1 are k
       const bool is_q = head < a;
@@ -222,10 +222,12 @@ cudaError_t launch_rope_kv_rows(const LaunchCtx& c, int dt, const float* QKV, in
                                 int a, int b, int d, int max_seq, const float2* rope, float* Q,
                                 void* kcache_layer, void* vcache_layer) {
   LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
+  const int work = (a + b) * (d / 2) + b * d;  // elements per position; two per thread and slice
+  const dim3 grid(T, (work + 511) / 512);
   if (dt == DT_BF16)
-    return launch_kernel(nc, rope_kv_rows_kernel<__nv_bfloat16>, dim3(T), dim3(256), 0, QKV, pos0, n_shards, a,
+    return launch_kernel(nc, rope_kv_rows_kernel<__nv_bfloat16>, grid, dim3(256), 0, QKV, pos0, n_shards, a,
                          b, d, max_seq, rope, Q, (__nv_bfloat16*)kcache_layer, (__nv_bfloat16*)vcache_layer);
-  return launch_kernel(nc, rope_kv_rows_kernel<float>, dim3(T), dim3(256), 0, QKV, pos0, n_shards, a, b, d,
+  return launch_kernel(nc, rope_kv_rows_kernel<float>, grid, dim3(256), 0, QKV, pos0, n_shards, a, b, d,
                        max_seq, rope, Q, (float*)kcache_layer, (float*)vcache_layer);
 }
 
