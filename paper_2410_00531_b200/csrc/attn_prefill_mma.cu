@@ -235,6 +235,231 @@ cudaError_t launch_t(const LaunchCtx& c, const float* Q, const void* kc, const v
 
 }  // namespace
 
+// =====================================================================================================
+// Decode attention on tensor cores: one query position, the GRP query heads of a kv head are the rows
+// (padded to 16) of the same m16n8k16 tiles.  Grid (kv head, split); the 4 warps of a CTA take 64-key
+// tiles of the split in turn (each stages its own K/V tile in shared memory), then the CTA folds the
+// warps' partial results, and the last split of a kv head to finish merges the splits in split order.
+// =====================================================================================================
+namespace {
+
+template <int D>
+__global__ void __launch_bounds__(128) decode_attn_mma_kernel(const float* __restrict__ q, const __nv_bfloat16* kc,
+                                                              const __nv_bfloat16* vc, const int* pos, int grp,
+                                                              int max_seq, int nsplit, float* scratch,
+                                                              unsigned* tickets, float* o_out) {
+  constexpr int KS = D / 16, ND = D / 8, CPR = D / 8, TILE = KB * D * 2;
+  extern __shared__ __align__(128) uint8_t smem[];  // [4 warps][K tile | V tile], reused by the merge buffers
+  __shared__ bool s_last;
+  pdl_launch_dependents();
+  pdl_wait();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  const int kvh = blockIdx.x, split = blockIdx.y;
+  const int n = *pos + 1;
+  int chunk = (n + nsplit - 1) / nsplit;
+  chunk = max(256, (chunk + 63) & ~63);
+  const int nact = (n + chunk - 1) / chunk;
+  if (split >= nact) return;  // this split sees no position (its ticket is not counted)
+  const int s0 = split * chunk, s1 = min(n, s0 + chunk);
+  const __nv_bfloat16* kg = kc + (size_t)kvh * max_seq * D;
+  const __nv_bfloat16* vg = vc + (size_t)kvh * max_seq * D;
+  const uint32_t my_k = (uint32_t)__cvta_generic_to_shared(smem) + warp * 2 * TILE, my_v = my_k + TILE;
+
+  // Q fragments: row g = head g of the group (rows >= grp and rows 8..15 are zero)
+  const float qscale = 1.4426950408889634f * rsqrtf((float)D);
+  uint32_t qh[KS][4], ql[KS][4];
+  {
+    const float* qrow = q + (size_t)(kvh * grp + min(g, grp - 1)) * D;
+    const float on = g < grp ? qscale : 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      const float2 v0 = *reinterpret_cast<const float2*>(qrow + ks * 16 + 2 * t);
+      const float2 v2 = *reinterpret_cast<const float2*>(qrow + ks * 16 + 8 + 2 * t);
+      split_pack(v0.x * on, v0.y * on, qh[ks][0], ql[ks][0]);
+      split_pack(v2.x * on, v2.y * on, qh[ks][2], ql[ks][2]);
+      qh[ks][1] = ql[ks][1] = qh[ks][3] = ql[ks][3] = 0u;
+    }
+  }
+  float o[ND][4];
+#pragma unroll
+  for (int nd = 0; nd < ND; ++nd) { o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f; }
+  float m_r = -INFINITY, l_r = 0.f;
+
+  for (int k0 = s0 + warp * KB; k0 < s1; k0 += 4 * KB) {  // this warp's tiles of the split
+    __syncwarp();
+    for (int i = lane; i < KB * CPR; i += 32) {
+      const int r = i / CPR, c = i - r * CPR;
+      const uint32_t off = tile_off<D>(r, c);
+      if (k0 + r < s1) {
+        const size_t src = (size_t)(k0 + r) * D + c * 8;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(my_k + off), "l"(kg + src) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(my_v + off), "l"(vg + src) : "memory");
+      } else {
+        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(my_k + off), "r"(0u) : "memory");
+        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(my_v + off), "r"(0u) : "memory");
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncwarp();
+    float s[KB / 8][4];
+#pragma unroll
+    for (int nb = 0; nb < KB / 8; ++nb) {
+      s[nb][0] = s[nb][1] = s[nb][2] = s[nb][3] = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < KS; ks += 2) {
+        uint32_t kb[4];
+        ldsm_x4(kb, my_k + tile_off<D>(nb * 8 + (lane & 7), ks * 2 + (lane >> 3)));
+        mma_bf16(s[nb], qh[ks], kb[0], kb[1]);
+        mma_bf16(s[nb], ql[ks], kb[0], kb[1]);
+        mma_bf16(s[nb], qh[ks + 1], kb[2], kb[3]);
+        mma_bf16(s[nb], ql[ks + 1], kb[2], kb[3]);
+      }
+    }
+    float mx = -INFINITY;
+#pragma unroll
+    for (int nb = 0; nb < KB / 8; ++nb) {
+      const int key = k0 + nb * 8 + 2 * t;
+      if (key >= s1) s[nb][0] = -INFINITY;
+      if (key + 1 >= s1) s[nb][1] = -INFINITY;
+      mx = fmaxf(mx, fmaxf(s[nb][0], s[nb][1]));
+    }
+    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
+    const float mn = fmaxf(m_r, mx);  // finite: the tile's first key is valid
+    const float sc = exp2f(m_r - mn);
+    m_r = mn;
+    l_r *= sc;
+#pragma unroll
+    for (int nd = 0; nd < ND; ++nd) { o[nd][0] *= sc; o[nd][1] *= sc; }
+    uint32_t ph[KB / 16][4], pl[KB / 16][4];
+#pragma unroll
+    for (int nb = 0; nb < KB / 8; ++nb) {
+      const float p0 = exp2f(s[nb][0] - mn), p1 = exp2f(s[nb][1] - mn);
+      l_r += p0 + p1;
+      const int kk = nb >> 1, half = nb & 1;
+      split_pack(p0, p1, ph[kk][half * 2], pl[kk][half * 2]);
+      ph[kk][half * 2 + 1] = pl[kk][half * 2 + 1] = 0u;
+    }
+#pragma unroll
+    for (int kk = 0; kk < KB / 16; ++kk) {
+#pragma unroll
+      for (int nd = 0; nd < ND; nd += 2) {
+        uint32_t vb[4];
+        ldsm_x4_trans(vb, my_v + tile_off<D>(kk * 16 + ((lane >> 3) & 1) * 8 + (lane & 7), nd + (lane >> 4)));
+        mma_bf16(o[nd], ph[kk], vb[0], vb[1]);
+        mma_bf16(o[nd], pl[kk], vb[0], vb[1]);
+        mma_bf16(o[nd + 1], ph[kk], vb[2], vb[3]);
+        mma_bf16(o[nd + 1], pl[kk], vb[2], vb[3]);
+      }
+    }
+  }
+  l_r += __shfl_xor_sync(0xFFFFFFFFu, l_r, 1);
+  l_r += __shfl_xor_sync(0xFFFFFFFFu, l_r, 2);
+
+  // ---- fold the 4 warps (fixed order).  Buffers alias the tiles, so everyone must be done reading them.
+  __syncthreads();
+  float* w_m = reinterpret_cast<float*>(smem);  // [4][8]
+  float* w_l = w_m + 32;                        // [4][8]
+  float* w_o = w_l + 32;                        // [4][8][D]
+  float* mw = w_o + 4 * 8 * D;                  // [grp][nsplit] weights of the final merge
+  if (t == 0) { w_m[warp * 8 + g] = m_r; w_l[warp * 8 + g] = l_r; }
+#pragma unroll
+  for (int nd = 0; nd < ND; ++nd) {
+    w_o[(warp * 8 + g) * D + nd * 8 + 2 * t] = o[nd][0];
+    w_o[(warp * 8 + g) * D + nd * 8 + 2 * t + 1] = o[nd][1];
+  }
+  __syncthreads();
+  float* part = scratch + ((size_t)kvh * nsplit + split) * grp * (D + 2);
+  for (int e = threadIdx.x; e < grp * D; e += 128) {
+    const int hh = e / D, dd = e - hh * D;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) M = fmaxf(M, w_m[w * 8 + hh]);
+    float A = 0.f, L = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float sc = exp2f(w_m[w * 8 + hh] - M);  // a warp that saw no tile has m = -inf, weight 0
+      A = fmaf(sc, w_o[(w * 8 + hh) * D + dd], A);
+      L = fmaf(sc, w_l[w * 8 + hh], L);
+    }
+    if (nact == 1) {
+      o_out[(size_t)(kvh * grp + hh) * D + dd] = A / L;  // a single split is the answer
+    } else {
+      part[hh * (D + 2) + 2 + dd] = A;
+      if (dd == 0) { part[hh * (D + 2)] = M; part[hh * (D + 2) + 1] = L; }
+    }
+  }
+  if (nact == 1) return;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned tk = atomicAdd(tickets + kvh, 1u);
+    s_last = (tk == (unsigned)nact - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const float* pg = scratch + (size_t)kvh * nsplit * grp * (D + 2);
+  for (int hh = warp; hh < grp; hh += 4) {
+    float M = -INFINITY;
+    for (int sI = lane; sI < nact; sI += 32) M = fmaxf(M, __ldcg(pg + (size_t)(sI * grp + hh) * (D + 2)));
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, off));
+    float L = 0.f;
+    for (int sI = lane; sI < nact; sI += 32) {
+      const float* ps = pg + (size_t)(sI * grp + hh) * (D + 2);
+      const float w = exp2f(__ldcg(ps) - M);
+      mw[hh * nact + sI] = w;
+      L = fmaf(w, __ldcg(ps + 1), L);
+    }
+    L = warp_sum(L);
+    const float inv = 1.f / L;
+    for (int sI = lane; sI < nact; sI += 32) mw[hh * nact + sI] *= inv;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < grp * D; e += 128) {
+    const int hh = e / D, dd = e - hh * D;
+    float A = 0.f;
+#pragma unroll 8
+    for (int sI = 0; sI < nact; ++sI)
+      A = fmaf(mw[hh * nact + sI], __ldcg(pg + (size_t)(sI * grp + hh) * (D + 2) + 2 + dd), A);
+    o_out[(size_t)(kvh * grp + hh) * D + dd] = A;
+  }
+  if (threadIdx.x == 0) tickets[kvh] = 0u;
+}
+
+template <int D>
+cudaError_t launch_dec_t(const LaunchCtx& c, const float* q, const void* kc, const void* vc, const int* pos, int a,
+                         int b, int max_seq, int nsplit, float* scratch, unsigned* tickets, float* o) {
+  auto kern = decode_attn_mma_kernel<D>;
+  const size_t smem = (size_t)4 * 2 * KB * D * 2;  // >= merge buffers (64 + 32 D + grp * nsplit floats)
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  return launch_kernel(c, kern, dim3(b, nsplit), dim3(128), smem, q, (const __nv_bfloat16*)kc,
+                       (const __nv_bfloat16*)vc, pos, a / b, max_seq, nsplit, scratch, tickets, o);
+}
+
+}  // namespace
+
+bool decode_attention_mma_supported(int dt, int a, int b, int d, int nsplit) {
+  const int grp = a / b;
+  return dt == DT_BF16 && (d == 128 || d == 64) && grp <= 8 && (size_t)(64 + 32 * d + grp * nsplit) * 4 <= (size_t)4 * 2 * KB * d * 2;
+}
+
+cudaError_t launch_decode_attention_mma(const LaunchCtx& c, const float* q, const void* kcache_layer,
+                                        const void* vcache_layer, const int* pos, int a, int b, int d, int max_seq,
+                                        int nsplit, float* scratch, unsigned* tickets, float* o) {
+  if (d == 128) return launch_dec_t<128>(c, q, kcache_layer, vcache_layer, pos, a, b, max_seq, nsplit, scratch, tickets, o);
+  if (d == 64) return launch_dec_t<64>(c, q, kcache_layer, vcache_layer, pos, a, b, max_seq, nsplit, scratch, tickets, o);
+  return cudaErrorInvalidValue;
+}
+
 bool prefill_attention_mma_supported(int dt, int d) { return dt == DT_BF16 && (d == 128 || d == 64); }
 
 cudaError_t launch_prefill_attention_mma(const LaunchCtx& c, const float* Q, const void* kcache_layer,

@@ -72,6 +72,11 @@ cudaError_t launch_decode_attention(const LaunchCtx& c, int dt, const float* q, 
                                     int max_seq, int nsplit, float* scratch, unsigned* tickets,
                                     float* o);
 size_t decode_attention_scratch_floats(int a, int b, int d, int nsplit);
+// tensor-core form (bf16 cache, head dim 64 / 128, up to 8 query heads per kv head); launch_decode_attention uses it when it applies
+bool decode_attention_mma_supported(int dt, int a, int b, int d, int nsplit);
+cudaError_t launch_decode_attention_mma(const LaunchCtx& c, const float* q, const void* kcache_layer,
+                                        const void* vcache_layer, const int* pos, int a, int b, int d, int max_seq,
+                                        int nsplit, float* scratch, unsigned* tickets, float* o);
 
 // Task head (Step 4): logits = W_head . (xhat * gain), greedy argmax (lowest index on ties);
 // writes tok_hist[*pos + 1] and advances *pos.  amax scratch: >= grid blocks entries.

@@ -697,6 +697,8 @@ cudaError_t launch_decode_attention(const LaunchCtx& c, int dt, const float* q, 
                                     const void* vcache_layer, const int* pos, int a, int b, int d,
                                     int max_seq, int nsplit, float* scratch, unsigned* tickets,
                                     float* o) {
+  if (decode_attention_mma_supported(dt, a, b, d, nsplit))
+    return launch_decode_attention_mma(c, q, kcache_layer, vcache_layer, pos, a, b, d, max_seq, nsplit, scratch, tickets, o);
   const int grp = a / b;
   const int lpr = (int)(d * dt_size(dt) / 16);
   if (dt == DT_BF16) {

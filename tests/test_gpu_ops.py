@@ -157,6 +157,9 @@ def test_qkv_rope_kv_append(T, cfg, n_shards, p):
     ("f32", 4, 4, 64, 24, 1),            # C1
     ("f32", 64, 8, 128, 577, 5),         # C4, ragged split
     ("bf16", 8, 2, 32, 1, 3),            # a single cached position, empty splits
+    ("bf16", 8, 2, 128, 1, 3),           # the same on the tensor-core path
+    ("bf16", 16, 2, 64, 700, 4),         # 8 heads per kv head, d = 64, three active splits
+    ("bf16", 32, 8, 128, 257, 33),       # just past one split
     ("f32", 8, 4, 64, 33, 8),
 ])
 def test_decode_attention(T, dtype, a, b, d, n, nsplit):
@@ -179,7 +182,8 @@ def test_decode_attention(T, dtype, a, b, d, n, nsplit):
                            a, b, d, max_seq, nsplit, scratch.data_ptr(), tickets.data_ptr(), o.data_ptr())
     want = O.attention(q.astype(np.float64).reshape(1, a, d), k[:, :n].astype(np.float64), v[:, :n].astype(np.float64),
                        np.array([n - 1]))[0]
-    assert rel_l2(o.cpu().numpy(), want) < 5e-6
+    # bf16 caches with d = 64 / 128 run on tensor cores with split-bf16 queries and weights (~2^-17 per operand)
+    assert rel_l2(o.cpu().numpy(), want) < (2e-5 if dtype == "bf16" and d >= 64 else 5e-6)
     assert not tickets.cpu().numpy().any()
 
 
