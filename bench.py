@@ -187,7 +187,12 @@ def run_gpu(args, shape):
     max_seq = T + W + K + 8
     cfg = tpi_config(shape, max_seq, min(T, 512))
     t_load = time.perf_counter()
-    ses = P.Session(cfg, S.synth_fill(shape), shape.n_shards, args.window, device=local)
+    extra = 0
+    if args.window > 0 and args.retain > 0:      # room for the kept FFN blocks beside the window (Prop. 6)
+        extra = len(range(0, shape.n_layers, args.retain)) * P.block_bytes(cfg)[1]
+    ses = P.Session(cfg, S.synth_fill(shape), shape.n_shards, args.window, device=local, extra_dev_bytes=extra)
+    if extra:
+        P.set_retention(ses.h, args.retain)
     t_load = time.perf_counter() - t_load
     if args.window > 0:
         return run_streamed(args, shape, ses, t_load, local, rank)
@@ -354,6 +359,8 @@ def run_streamed(args, shape, ses, t_load, local, rank):
         "config": {"workload": workload_name(shape, args).replace("all weights resident", f"layer blocks streamed from pinned host memory, window {args.window} blocks"),
                    "l2": "inputs larger than L2 (every block is copied from host memory each token)",
                    "window_blocks": args.window, "window_device_bytes": st["window_peak_bytes"],
+                   "retain_ffn_every": args.retain, "retained_blocks": st["retained_blocks"],
+                   "retained_device_bytes": st["retained_bytes"],
                    "block_bytes": {"attention": attn_b, "ffn": ffn_b}, "load_s": round(t_load, 1)},
         "clocks": clocks,
         "e2e": {"value": K / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(link_bytes) + 4, "d2h_bytes_per_step": 8},
@@ -377,6 +384,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C2", choices=sorted(S.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--retain", type=int, default=0,
+                    help="with --window: keep one FFN block in every T resident beside the window (0 = none)")
     ap.add_argument("--window", type=int, default=0,
                     help="stream the layer blocks through a window of this many blocks (0 = all resident)")
     ap.add_argument("--prompt", type=int, default=0, help="override the prompt length")

@@ -117,6 +117,15 @@ int tpi_set_shards(tpi_model *m, int n_shards);
  * Needs host images unless going 0 -> 0. */
 int tpi_set_window(tpi_model *m, int window_blocks);
 
+/* Block retention (Sec. 3.3, Prop. 6 / Appendix A.6): when the link is the bottleneck, keep ONE FFN
+ * block in every `ffn_every_T` FFN blocks resident (layers 0, T, 2T, ...) beside the window and stream
+ * only the rest; 0 turns retention off, 1 keeps every FFN block.  Only for a streamed model
+ * (window >= 1).  The retained blocks live in the device arena after the window slots: the arena must
+ * have room for them (TPI_ERR_NOMEM otherwise, and the previous setting stays in force).  Keeps the KV
+ * cache and the position; results are bit-identical with and without retention.  tpi_set_window turns
+ * retention off again (it is chosen per window size). */
+int tpi_set_retention(tpi_model *m, int ffn_every_T);
+
 /* One pass of Algorithm 1's loop body over n_tokens prompt positions starting
  * at the current position (usually 0): fills the KV cache and returns the
  * greedy next token.  tokens: HOST int32[n_tokens].  first_token: HOST int32*.
@@ -167,6 +176,8 @@ typedef struct {
   int32_t kernel_launches_last; /* kernels launched by the last prefill/decode call      */
   int32_t window_blocks, n_shards, position, graph_active;
   uint64_t window_peak_bytes;  /* device bytes held by window slots                      */
+  uint64_t retained_bytes;     /* device bytes held by retained blocks (block retention) */
+  int32_t retained_blocks, reserved_;
 } tpi_stats;
 int tpi_get_stats(tpi_model *m, tpi_stats *out);
 
@@ -195,6 +206,9 @@ int tpi_set_option(tpi_model *m, int option, int value);
  * `slot`, 4 = compute queue releases `slot`.  Returns the number of operations
  * (which may exceed max_ops) or a negative tpi_status. */
 int tpi_ring_trace(int n_blocks, int w, int n_exec, int *ops, int max_ops);
+/* The same with block retention: the FFN block of layers 0, T, 2T, ... is retained; executing a
+ * retained block is recorded as op 5 (slot -1) and touches neither queue. */
+int tpi_ring_trace_retained(int n_blocks, int w, int n_exec, int ffn_every_T, int *ops, int max_ops);
 
 void tpi_free(tpi_model *m);
 const char *tpi_strerror(int code);

@@ -98,3 +98,56 @@ def loose_condition(t_attn, t_ffn, t_ar, tau_attn, tau_ffn, L: int) -> bool:
 def tight_condition(t_attn, t_ffn, t_ar, tau_attn, tau_ffn) -> bool:
     """Prop. 4."""
     return t_attn + t_ar >= tau_ffn and t_ffn + t_ar >= tau_attn
+
+
+def retained_ffn_layers(L: int, T: int):
+    """Appendix A.6's indicator: with one FFN block kept in every T, the kept ones are those of
+    layers l = 1 + kT (1-based), i.e. 0, T, 2T, ... (0-based).  T = 0: none."""
+    return set() if T <= 0 else set(range(0, L, T))
+
+
+def timeline_retained(t_attn, t_ffn, t_ar, tau_attn, tau_ffn, n_blocks: int, w: int, T: int, L: int):
+    """The time-slot model with block retention (Prop. 6 / Appendix A.6).
+
+    As ``timeline`` (blocks alternate attention, FFN; execution wraps around after 2L blocks), except
+    that the FFN blocks of the retained layers are always in memory: the loader skips them and they
+    never wait.  The window's w places are split as Prop. 5 counts them, floor(w/2) attention and
+    ceil(w/2) FFN blocks (w = 1: a single shared place), so a streamed block may start loading only
+    after the streamed block of its kind that many places earlier has been released.
+    """
+    keep = retained_ffn_layers(L, T)
+    n_slots = {0: w // 2, 1: (w + 1) // 2} if w > 1 else None
+    stall = [0.0] * n_blocks
+    slack = [0.0] * n_blocks
+    released_of_kind = {0: [], 1: [], 2: []}      # release times of streamed blocks, per kind (2: shared, w = 1)
+    loader_free = 0.0
+    prev_done = 0.0
+    for k in range(n_blocks):
+        kind = k % 2
+        layer = (k // 2) % L
+        t = t_ffn if kind else t_attn
+        if kind == 1 and layer in keep:
+            prev_done += t + t_ar
+            continue
+        tau = tau_ffn if kind else tau_attn
+        hist = released_of_kind[kind if n_slots else 2]
+        places = n_slots[kind] if n_slots else 1
+        start_load = loader_free if len(hist) < places else max(loader_free, hist[len(hist) - places])
+        load_done = start_load + tau
+        loader_free = load_done
+        stall[k] = max(0.0, load_done - prev_done)
+        slack[k] = max(0.0, prev_done - load_done)
+        prev_done = max(prev_done, load_done) + t + t_ar
+        hist.append(prev_done)
+    return stall, slack, prev_done
+
+
+def retention_condition(t_attn, t_ffn, t_ar, tau_attn, tau_ffn, L: int, T: int) -> bool:
+    """Prop. 6 as printed: both families of inequalities for l = 1..L."""
+    def kept(l):
+        return -(-l // T)                      # ceil(l / T)
+    first = all(l * t_attn + l * t_ffn + 2 * l * t_ar >= (l - kept(l)) * tau_ffn + l * tau_attn
+                for l in range(1, L + 1))
+    second = all(l * t_attn + (l - 1) * t_ffn + (2 * l - 1) * t_ar >= (l - kept(l)) * tau_ffn + (l - 1) * tau_attn
+                 for l in range(1, L + 1))
+    return first and second

@@ -49,7 +49,8 @@ class TpiStats(C.Structure):
                 ("dominant_kernel_bytes", C.c_uint64), ("dominant_kernel_samples", C.c_uint32),
                 ("kernel_launches_last", C.c_int32), ("window_blocks", C.c_int32),
                 ("n_shards", C.c_int32), ("position", C.c_int32), ("graph_active", C.c_int32),
-                ("window_peak_bytes", C.c_uint64)]
+                ("window_peak_bytes", C.c_uint64), ("retained_bytes", C.c_uint64),
+                ("retained_blocks", C.c_int32), ("reserved_", C.c_int32)]
 
     def as_dict(self) -> dict:
         return {k: getattr(self, k) for k, _ in self._fields_}
@@ -81,6 +82,8 @@ SYMBOLS = {
     "tpi_get_stats": (C.c_int, [C.c_void_p, C.POINTER(TpiStats)]),
     "tpi_set_option": (C.c_int, [C.c_void_p, C.c_int, C.c_int]),
     "tpi_ring_trace": (C.c_int, [C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.c_int]),
+    "tpi_ring_trace_retained": (C.c_int, [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.c_int]),
+    "tpi_set_retention": (C.c_int, [C.c_void_p, C.c_int]),
     "tpi_free": (None, [C.c_void_p]),
     "tpi_strerror": (C.c_char_p, [C.c_int]),
     "tpi_last_error": (C.c_char_p, []),
@@ -206,9 +209,14 @@ def set_option(h, option: int, value: int) -> None:
     _check(lib().tpi_set_option(h, option, value))
 
 
-def ring_trace(n_blocks: int, w: int, n_exec: int, max_ops: int = 1 << 16) -> np.ndarray:
+def set_retention(h, ffn_every_T: int) -> None:
+    _check(lib().tpi_set_retention(h, ffn_every_T))
+
+
+def ring_trace(n_blocks: int, w: int, n_exec: int, max_ops: int = 1 << 16, ffn_every_T: int = 0) -> np.ndarray:
     ops = np.zeros((max_ops, 3), np.int32)
-    n = _check(lib().tpi_ring_trace(n_blocks, w, n_exec, ops.ctypes.data_as(C.POINTER(C.c_int)), max_ops))
+    n = _check(lib().tpi_ring_trace_retained(n_blocks, w, n_exec, ffn_every_T,
+                                             ops.ctypes.data_as(C.POINTER(C.c_int)), max_ops))
     if n > max_ops:
         raise ValueError("trace buffer too small")
     return ops[:n]
@@ -233,7 +241,8 @@ class Session:
     """Owns the arenas (torch tensors), the streams and the model handle."""
 
     def __init__(self, cfg: TpiConfig, fill: FillFn, n_shards: int, window_blocks: int = 0,
-                 keep_host_images: Optional[bool] = None, device: int = 0, other_windows=()):
+                 keep_host_images: Optional[bool] = None, device: int = 0, other_windows=(),
+                 extra_dev_bytes: int = 0):
         """other_windows: window sizes this session may later switch to with set_window
         (the device arena is sized for the largest of them; 0 means fully resident)."""
         import torch
@@ -250,6 +259,7 @@ class Session:
             d_need = max(d_need, query_arena(cfg, n_shards, w, True)[0])
         if keep_host_images:
             h_need = query_arena(cfg, n_shards, window_blocks, True)[1]
+        d_need += int(extra_dev_bytes)      # e.g. room for retained blocks (tpi_set_retention)
         self.dev = torch.empty(d_need, dtype=torch.uint8, device=f"cuda:{device}")
         self.host = torch.empty(h_need, dtype=torch.uint8, pin_memory=True)
         self.compute = torch.cuda.Stream(device=device)

@@ -80,6 +80,10 @@ struct tpi_model {
   int position = 0;
   // window ring
   Ring ring;
+  int retain_T = 0;                  // keep the FFN block of every T-th layer resident beside the window (0: none)
+  std::vector<char> retained;        // per block
+  std::vector<size_t> retained_off;  // byte offset of a retained block after the window slots
+  size_t retained_bytes = 0;
   std::vector<cudaEvent_t> ev_loaded, ev_released;
   uint64_t link_bytes = 0;
   // graph of one resident decode step
@@ -471,7 +475,33 @@ static int start_window(tpi_model* m) {
   be.copy_record_loaded = be_copy_record_loaded;
   be.compute_wait_loaded = be_compute_wait_loaded;
   be.compute_record_released = be_compute_record_released;
-  m->ring.configure(2 * m->cfg.n_layers, m->window, be);
+  // Block retention (Prop. 6): the FFN block of every T-th layer stays resident after the window slots.
+  const int nb = 2 * m->cfg.n_layers;
+  m->retained.assign(nb, 0);
+  m->retained_off.assign(nb, 0);
+  m->retained_bytes = 0;
+  {
+    int nA, nF;
+    window_slots(m->window, &nA, &nF);
+    const size_t slots = (size_t)nA * m->plan.bl.attn_bytes + (size_t)nF * m->plan.bl.ffn_bytes;
+    size_t off = slots;
+    if (m->retain_T > 0)
+      for (int l = 0; l < m->cfg.n_layers; l += m->retain_T) {
+        m->retained[2 * l + 1] = 1;
+        m->retained_off[2 * l + 1] = off;
+        off += m->plan.bl.ffn_bytes;
+      }
+    m->retained_bytes = off - slots;
+    if (m->plan.blocks + off > m->res.dev_bytes)
+      return fail(TPI_ERR_NOMEM, "device arena too small for the window plus retained blocks: need %zu bytes, have %zu",
+                  m->plan.blocks + off, m->res.dev_bytes);
+    for (int b = 0; b < nb; ++b)
+      if (m->retained[b])
+        CK(cudaMemcpyAsync(m->dev + m->plan.blocks + m->retained_off[b], host_image(m, b), block_size(m, b),
+                           cudaMemcpyHostToDevice, m->cs));
+    CK(cudaStreamSynchronize(m->cs));
+  }
+  m->ring.configure(nb, m->window, be, m->retained.data());
   for (int i = 0; i < m->ring.n_slots(); ++i) {
     cudaEvent_t a, b;
     CK(cudaEventCreateWithFlags(&a, cudaEventDisableTiming));
@@ -641,12 +671,28 @@ extern "C" int tpi_set_window(tpi_model* m, int window_blocks) {
   drop_graph(m);
   m->plan = np;
   m->window = window_blocks;
+  m->retain_T = 0;  // retention is chosen per window size: set it again after this call
   if (window_blocks == 0) {
     for (int b = 0; b < 2 * m->cfg.n_layers; ++b)
       CK(cudaMemcpyAsync(resident_block(m, b), host_image(m, b), block_size(m, b), cudaMemcpyHostToDevice, m->cs));
     CK(cudaStreamSynchronize(m->cs));
   }
   return start_window(m);
+}
+
+extern "C" int tpi_set_retention(tpi_model* m, int ffn_every_T) {
+  if (!m || ffn_every_T < 0) return fail(TPI_ERR_INVALID_ARG, "bad argument");
+  if (m->window <= 0) return fail(TPI_ERR_STATE, "block retention applies to a streamed model (window >= 1)");
+  TRY(quiesce(m));
+  drop_graph(m);
+  const int old = m->retain_T;
+  m->retain_T = ffn_every_T;
+  const int rc = start_window(m);
+  if (rc) {  // put the previous setting back so that the model stays usable
+    m->retain_T = old;
+    start_window(m);
+  }
+  return rc;
 }
 
 extern "C" int tpi_reset(tpi_model* m) {
@@ -696,6 +742,7 @@ struct BlockRef {
 };
 static int acquire_block(tpi_model* m, int block, BlockRef* r) {
   if (m->window <= 0) { r->base = resident_block(m, block); r->slot = -1; return TPI_OK; }
+  if (m->retained[block]) { r->base = m->dev + m->plan.blocks + m->retained_off[block]; r->slot = -1; return TPI_OK; }
   const int s = m->ring.acquire(block);
   if (s < 0) return s == -1000 || s == -1001 ? fail(TPI_ERR_STATE, "window ring out of order (%d)", s) : s;
   r->base = slot_ptr(m, s);
@@ -703,7 +750,7 @@ static int acquire_block(tpi_model* m, int block, BlockRef* r) {
   return TPI_OK;
 }
 static int release_block(tpi_model* m, int block) {
-  if (m->window <= 0) return TPI_OK;
+  if (m->window <= 0 || m->retained[block]) return TPI_OK;
   const int rc = m->ring.release(block);
   if (rc == -1000) return fail(TPI_ERR_STATE, "window ring out of order");
   return rc;
@@ -1045,6 +1092,10 @@ extern "C" int tpi_get_stats(tpi_model* m, tpi_stats* out) {
     s.window_peak_bytes = (uint64_t)m->ring.n_attn_slots() * m->plan.bl.attn_bytes +
                           (uint64_t)m->ring.n_ffn_slots() * m->plan.bl.ffn_bytes;
   } else s.window_peak_bytes = 0;
+  s.retained_bytes = m->window > 0 ? m->retained_bytes : 0;
+  s.retained_blocks = 0;
+  if (m->window > 0)
+    for (char r : m->retained) s.retained_blocks += r != 0;
   *out = s;
   return TPI_OK;
 }
@@ -1074,8 +1125,15 @@ int tr_xrr(void* c, int s) { return tr_push(c, 4, s, -1); }
 // 2 copy-queue marks slot loaded, 3 compute-queue waits for slot, 4 compute-queue releases slot.
 // Returns the number of operations (may exceed max_ops) or a negative status.
 extern "C" int tpi_ring_trace(int n_blocks, int w, int n_exec, int* ops, int max_ops) {
-  if (n_blocks < 2 || n_blocks % 2 || w < 1 || n_exec < 0 || (!ops && max_ops > 0))
+  return tpi_ring_trace_retained(n_blocks, w, n_exec, 0, ops, max_ops);
+}
+
+extern "C" int tpi_ring_trace_retained(int n_blocks, int w, int n_exec, int ffn_every_T, int* ops, int max_ops) {
+  if (n_blocks < 2 || n_blocks % 2 || w < 1 || n_exec < 0 || ffn_every_T < 0 || (!ops && max_ops > 0))
     return fail(TPI_ERR_INVALID_ARG, "bad argument");
+  std::vector<char> keep(n_blocks, 0);
+  if (ffn_every_T > 0)
+    for (int l = 0; l < n_blocks / 2; l += ffn_every_T) keep[2 * l + 1] = 1;
   TraceCtx t{ops, max_ops, 0};
   RingBackend be;
   be.ctx = &t;
@@ -1085,10 +1143,11 @@ extern "C" int tpi_ring_trace(int n_blocks, int w, int n_exec, int* ops, int max
   be.compute_wait_loaded = tr_xwl;
   be.compute_record_released = tr_xrr;
   Ring r;
-  r.configure(n_blocks, w, be);
+  r.configure(n_blocks, w, be, keep.data());
   if (r.pump()) return TPI_ERR_STATE;
   for (int i = 0; i < n_exec; ++i) {
     const int blk = i % n_blocks;
+    if (keep[blk]) { tr_push(&t, 5, -1, blk); continue; }  // a retained block runs without any window operation
     if (r.acquire(blk) < 0) return TPI_ERR_STATE;
     if (r.release(blk)) return TPI_ERR_STATE;
   }

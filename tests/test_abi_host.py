@@ -117,6 +117,10 @@ def replay(ops, t_exec, t_ar, tau, n_blocks):
             comp_t += t_exec[k % 2] + t_ar
             released[slot] = comp_t
             k += 1
+        elif op == 5:                                           # a retained block: no window operation
+            stalls.append(0.0)
+            comp_t += t_exec[k % 2] + t_ar
+            k += 1
     return stalls, comp_t
 
 
@@ -127,6 +131,20 @@ def test_ring_reproduces_the_oracle_timeline(w):
     ops = P.ring_trace(n_blocks, w, n_exec)
     stalls, end = replay(ops, (ta, tf), tr, (la, lf), n_blocks)
     want, _, want_end = W.timeline(ta, tf, tr, la, lf, n_exec, w)
+    assert len(stalls) == n_exec
+    assert np.allclose(stalls, want) and np.isclose(end, want_end)
+
+
+@pytest.mark.parametrize("w,T", [(1, 2), (2, 1), (2, 3), (4, 2), (6, 4), (8, 5)])
+def test_ring_with_block_retention_reproduces_the_oracle_timeline(w, T):
+    ta, tf, tr, la, lf = 11.0, 17.0, 14.0, 18.0, 60.0           # a link too slow for Prop. 3
+    L, n_exec = 16, 100                                         # crosses the token boundary (cyclic)
+    ops = P.ring_trace(2 * L, w, n_exec, ffn_every_T=T)
+    keep = {2 * l + 1 for l in W.retained_ffn_layers(L, T)}
+    assert {int(b) for op, _, b in ops if op == 5} == keep     # exactly the kept blocks run without a load
+    assert not any(int(b) in keep for op, _, b in ops if op == 1)
+    stalls, end = replay(ops, (ta, tf), tr, (la, lf), 2 * L)
+    want, _, want_end = W.timeline_retained(ta, tf, tr, la, lf, n_exec, w, T, L)
     assert len(stalls) == n_exec
     assert np.allclose(stalls, want) and np.isclose(end, want_end)
 

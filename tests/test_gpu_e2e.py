@@ -126,6 +126,46 @@ def test_streamed_is_bit_identical_to_resident(window):
     assert np.array_equal(a[1], b[1]) and np.array_equal(a[4], b[4])
 
 
+@pytest.mark.parametrize("window,T", [(1, 2), (2, 1), (4, 3)])
+def test_block_retention_is_bit_identical_and_loads_less(window, T):
+    """Prop. 6's retention: the kept FFN blocks never cross the link again, the rest stream as before,
+    and the tokens and logits are the same bits as the resident run's."""
+    import paper_2410_00531_b200 as P
+    from helpers import tpi_config
+    shape = S.CONFIGS["C1"].with_(n_layers=6)
+    toks = S.prompt_tokens(shape)
+    _, ffn_bytes = P.block_bytes(tpi_config(shape, 64, 16))
+    n_keep = len(range(0, shape.n_layers, T))
+    res, loads = {}, {}
+    for mode in ("resident", "streamed", "retained"):
+        extra = n_keep * ffn_bytes if mode == "retained" else 0
+        with gpu_session(shape, 64, 16, 2, 0 if mode == "resident" else window, extra_dev_bytes=extra) as ses:
+            P.set_option(ses.h, P.OPT_MEGA, 0)
+            if mode == "retained":
+                P.set_retention(ses.h, T)
+            t0, lg0 = P.prefill(ses.h, toks, shape.vocab)
+            seq = P.decode_run(ses.h, t0, 5)
+            t1, lg1 = P.decode_step(ses.h, int(seq[-1]), shape.vocab)
+            res[mode] = (t0, lg0, seq, t1, lg1)
+            st = P.get_stats(ses.h)
+            loads[mode] = st["link_bytes_total"]
+            if mode == "retained":
+                assert st["retained_blocks"] == n_keep and st["retained_bytes"] == n_keep * ffn_bytes
+            elif mode == "streamed":
+                assert st["retained_blocks"] == 0
+                with pytest.raises(P.TpiError) as e:           # no room was given for kept blocks
+                    P.set_retention(ses.h, T)
+                assert e.value.code == -3
+                t2, _ = P.prefill(ses.h, toks, 0)               # ... and the model still works as before
+                assert t2 == t0
+    a = res["resident"]
+    for mode in ("streamed", "retained"):
+        b = res[mode]
+        assert a[0] == b[0] and a[3] == b[3] and (a[2] == b[2]).all()
+        assert np.array_equal(a[1], b[1]) and np.array_equal(a[4], b[4])
+    assert loads["retained"] < loads["streamed"]
+
+
 def test_set_shards_and_set_window_roundtrip():
     import paper_2410_00531_b200 as P
     shape = S.CONFIGS["C1"]

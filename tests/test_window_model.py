@@ -73,3 +73,37 @@ def test_prop5_worker_peak_counts_blocks():
     assert W.master_peak(4, h, v, a, b, s, p) == 2 * h * v + h + attn + ffn
     # the attention block of Table 5 and the one of Prop. 5 are the same count
     assert W.block_params("attn", h, v, a, b, s, p) == attn
+
+
+def test_retention_slot_expressions_and_prop6():
+    """Appendix A.6's time-slot expressions evaluated by hand on the paper's measured latencies
+    (t_attn 11, t_ffn 17, tau_attn 18, tau_ffn 30; allreduce 14 as in the worked example) with T = 2."""
+    ta, tf, tr, la, lf = 11.0, 17.0, 14.0, 18.0, 30.0
+    stall, slack, _ = W.timeline_retained(ta, tf, tr, la, lf, n_blocks=64, w=10**6, T=2, L=32)
+    assert stall[0] == la and all(s == 0 for s in stall[1:])
+    assert slack[1] == 0                                                   # slot 3: layer 1's FFN block is kept
+    assert slack[2] == ta + tf + 2 * tr - la == 38                         # slot 5 with the indicator = 1
+    assert slack[3] == 2 * ta + tf + 3 * tr - lf - la == 33                # slot 7: one FFN load so far
+    assert slack[4] == 2 * ta + 2 * tf + 4 * tr - lf - 2 * la == 46        # slot 9
+    assert W.retained_ffn_layers(7, 3) == {0, 3, 6} and W.retained_ffn_layers(7, 0) == set()
+    # no retention: the same model as the plain timeline, at every window size
+    for w in (1, 2, 4, 6, 10**6):
+        assert W.timeline_retained(ta, tf, tr, la, lf, 64, w, 0, 32) == W.timeline(ta, tf, tr, la, lf, 64, w)
+
+
+def test_prop6_decides_the_steady_state_of_the_timeline():
+    """A link twice as slow for FFN blocks (tau_ffn 60) breaks Prop. 3; Prop. 6 says which T repairs it,
+    and the event model with an unbounded window stalls exactly when Prop. 6 fails."""
+    ta, tf, tr, la, lf = 11.0, 17.0, 14.0, 18.0, 60.0
+    assert not W.loose_condition(ta, tf, tr, la, lf, L=32)
+    verdicts = {}
+    for T in (1, 2, 3, 4, 8):
+        stall, _, end = W.timeline_retained(ta, tf, tr, la, lf, n_blocks=64, w=10**6, T=T, L=32)
+        steady = all(s == 0 for s in stall[1:])
+        verdicts[T] = steady
+        assert steady == W.retention_condition(ta, tf, tr, la, lf, L=32, T=T), T
+        if steady:
+            assert end == la + 32 * (ta + tf + 2 * tr)
+    assert verdicts == {1: True, 2: True, 3: False, 4: False, 8: False}
+    # by hand for T = 3 at l = 3: 3*56 = 168 < (3 - 1)*60 + 3*18 = 174
+    assert 3 * (ta + tf + 2 * tr) < 2 * lf + 3 * la
