@@ -184,7 +184,7 @@ def run_gpu(args, shape):
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     torch.cuda.set_device(local)
     K, W, T = args.steps, args.warmup, shape.prompt_len
-    max_seq = T + W + K + 8
+    max_seq = T + W + K + 8 + (K + 8 if args.window > 0 else 0)   # the streamed leg also decodes its e2e and diagnostic tokens
     cfg = tpi_config(shape, max_seq, min(T, 512))
     t_load = time.perf_counter()
     extra = 0
@@ -345,6 +345,12 @@ def run_streamed(args, shape, ses, t_load, local, rank):
         tok, _ = P.decode_step(h, int(out[-1]) if _ == 0 else tok, 0)
     e2e_s = time.perf_counter() - t0
     attn_b, ffn_b = P.block_bytes(ses.cfg)
+    # the paper's scheduler diagnostics on a few extra tokens (event-timed per block: outside every timed region)
+    P.set_option(h, P.OPT_PROFILE, 1)
+    P.scheduler_reset(h)
+    P.decode_run(h, tok, min(K, 4))
+    torch.cuda.synchronize()
+    sched = P.scheduler_report(h)
     ses.close()
     peak = host_link_peak(torch, local)
     # The window is full when the timed region starts (the loader ran ahead while the host was idle) and the
@@ -370,6 +376,7 @@ def run_streamed(args, shape, ses, t_load, local, rank):
                      "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                      "traffic": link_bytes, "bytes_in_timed_region": timed_bytes,
                      "peak_kind": "pinned H2D copy (1 GiB, best of 4) measured in this run"},
+        "scheduler": sched,
         "cpu_baseline": None, "tokens_tail": [int(x) for x in out[-4:]],
     }
     if rank == 0:

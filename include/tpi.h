@@ -181,6 +181,31 @@ typedef struct {
 } tpi_stats;
 int tpi_get_stats(tpi_model *m, tpi_stats *out);
 
+/* The paper's scheduler diagnostics (Sec. 3.3): the latencies that Prop. 3-6 are stated in, measured
+ * on this run, and the propositions evaluated on them.  Samples are taken by decode calls while
+ * TPI_OPT_PROFILE is 1 (CUDA events around every block's kernels on the compute stream and around
+ * every block copy on the copy stream; means over all samples since load or tpi_scheduler_reset).
+ * The emulated allreduce (the rank-ordered sum) runs inside each block's last kernel, so it is part
+ * of t_attn / t_ffn and t_all_reduce is reported as 0; every proposition only uses the sums
+ * t + t_all_reduce, so the verdicts are unaffected.  tight_holds / loose_holds: Prop. 4 / Prop. 3
+ * (1 or 0); retention_T: 0 if Prop. 3 holds without retention, else the largest T for which Prop. 6
+ * holds, -1 if none does; all three are -2 while a needed sample is missing (e.g. a resident model
+ * has no loads).  m_worker_bytes: Prop. 5's M_worker for the current window without the empirical
+ * factor; window_device_bytes: what the window slots plus retained blocks occupy. */
+typedef struct {
+  double t_attn_ms, t_ffn_ms, t_all_reduce_ms, tau_attn_ms, tau_ffn_ms, stall_ms_total;
+  uint32_t n_t_attn, n_t_ffn, n_tau_attn, n_tau_ffn;
+  int32_t tight_holds, loose_holds, retention_T, window_blocks, retain_every_T, reserved_;
+  uint64_t m_worker_bytes, window_device_bytes;
+} tpi_sched_report;
+int tpi_scheduler_report(tpi_model *m, tpi_sched_report *out);
+int tpi_scheduler_reset(tpi_model *m);
+
+/* Prop. 3 (loose), Prop. 4 (tight) and Prop. 6 (retention) on given latencies; host arithmetic only,
+ * any consistent time unit.  Outputs may be null.  *retention_T as in tpi_sched_report. */
+int tpi_steady_conditions(double t_attn, double t_ffn, double t_all_reduce, double tau_attn, double tau_ffn,
+                          int n_layers, int *tight, int *loose, int *retention_T);
+
 /* Options: TPI_OPT_GRAPH (1 = replay the decode step as a CUDA graph when all
  * blocks are resident; default 1), TPI_OPT_PDL (1 = programmatic dependent
  * launch between kernels; default 1), TPI_OPT_PROFILE (1 = CUDA events around

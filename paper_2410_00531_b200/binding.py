@@ -84,6 +84,9 @@ SYMBOLS = {
     "tpi_ring_trace": (C.c_int, [C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.c_int]),
     "tpi_ring_trace_retained": (C.c_int, [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.c_int]),
     "tpi_set_retention": (C.c_int, [C.c_void_p, C.c_int]),
+    "tpi_scheduler_report": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "tpi_scheduler_reset": (C.c_int, [C.c_void_p]),
+    "tpi_steady_conditions": (C.c_int, [C.c_double] * 5 + [C.c_int] + [C.POINTER(C.c_int)] * 3),
     "tpi_free": (None, [C.c_void_p]),
     "tpi_strerror": (C.c_char_p, [C.c_int]),
     "tpi_last_error": (C.c_char_p, []),
@@ -207,6 +210,33 @@ def get_stats(h) -> dict:
 
 def set_option(h, option: int, value: int) -> None:
     _check(lib().tpi_set_option(h, option, value))
+
+
+class TpiSchedReport(C.Structure):
+    _fields_ = [(n, C.c_double) for n in ("t_attn_ms", "t_ffn_ms", "t_all_reduce_ms", "tau_attn_ms", "tau_ffn_ms",
+                                          "stall_ms_total")] + \
+               [(n, C.c_uint32) for n in ("n_t_attn", "n_t_ffn", "n_tau_attn", "n_tau_ffn")] + \
+               [(n, C.c_int32) for n in ("tight_holds", "loose_holds", "retention_T", "window_blocks",
+                                         "retain_every_T", "reserved_")] + \
+               [("m_worker_bytes", C.c_uint64), ("window_device_bytes", C.c_uint64)]
+
+
+def scheduler_report(h) -> dict:
+    r = TpiSchedReport()
+    _check(lib().tpi_scheduler_report(h, C.byref(r)))
+    return {n: getattr(r, n) for n, _ in r._fields_ if n != "reserved_"}
+
+
+def scheduler_reset(h) -> None:
+    _check(lib().tpi_scheduler_reset(h))
+
+
+def steady_conditions(t_attn, t_ffn, t_all_reduce, tau_attn, tau_ffn, n_layers: int):
+    """Returns (tight, loose, retention_T)."""
+    a, b, c = C.c_int(), C.c_int(), C.c_int()
+    _check(lib().tpi_steady_conditions(t_attn, t_ffn, t_all_reduce, tau_attn, tau_ffn, n_layers,
+                                       C.byref(a), C.byref(b), C.byref(c)))
+    return bool(a.value), bool(b.value), c.value
 
 
 def set_retention(h, ffn_every_T: int) -> None:

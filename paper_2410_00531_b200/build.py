@@ -39,7 +39,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     for src, p in procs:
         if p.wait():
             raise RuntimeError(f"nvcc failed on {src}")
-    subprocess.check_call([nvcc, "-shared", "-o", OUT, *objs, "-Xcompiler", "-fopenmp", "-lgomp"])
+    subprocess.check_call([nvcc, *NVCC_FLAGS[:2], "-shared", "-o", OUT, *objs, "-Xcompiler", "-fopenmp", "-lgomp"])
     return OUT
 
 

@@ -95,6 +95,15 @@ struct tpi_model {
   size_t prof_used = 0;
   double prof_ms_sum = 0;
   uint32_t prof_samples = 0;
+  // scheduler diagnostics (profile mode, decode only): event pairs around each block's kernels on the
+  // compute stream (kinds 0 attention, 1 FFN) and around each block copy on the copy stream (kinds 2, 3)
+  struct TimedPair { cudaEvent_t a, b; int kind; };
+  std::vector<TimedPair> sched_pending;
+  std::vector<cudaEvent_t> sched_free;
+  cudaEvent_t sched_open = nullptr;
+  bool sched_rec = false;
+  double sched_sum[4] = {0, 0, 0, 0};
+  uint32_t sched_n[4] = {0, 0, 0, 0};
   std::vector<cudaEvent_t> stall_ev;  // pairs around window waits (profile mode)
   size_t stall_used = 0;
   double stall_ms = 0;
@@ -342,6 +351,32 @@ static int load_layers(tpi_model* m) {
   return TPI_OK;
 }
 
+// ------------------------------------------------------------------------------ scheduler diagnostics
+static cudaEvent_t sched_event(tpi_model* m) {
+  if (!m->sched_free.empty()) { cudaEvent_t e = m->sched_free.back(); m->sched_free.pop_back(); return e; }
+  if (m->sched_pending.size() >= 8192) return nullptr;  // bounded: further samples are dropped until a harvest
+  cudaEvent_t e = nullptr;
+  return cudaEventCreate(&e) == cudaSuccess ? e : nullptr;
+}
+// completed pairs go into the running means; pairs still in flight (the loader runs ahead) stay for the next call
+static void sched_harvest(tpi_model* m) {
+  size_t keep = 0;
+  for (size_t i = 0; i < m->sched_pending.size(); ++i) {
+    tpi_model::TimedPair tp = m->sched_pending[i];
+    float ms = 0;
+    if (cudaEventQuery(tp.b) == cudaSuccess && cudaEventElapsedTime(&ms, tp.a, tp.b) == cudaSuccess) {
+      m->sched_sum[tp.kind] += ms;
+      ++m->sched_n[tp.kind];
+      m->sched_free.push_back(tp.a);
+      m->sched_free.push_back(tp.b);
+    } else {
+      cudaGetLastError();  // cudaErrorNotReady is expected here
+      m->sched_pending[keep++] = tp;
+    }
+  }
+  m->sched_pending.resize(keep);
+}
+
 // ------------------------------------------------------------------------------ ring back end (CUDA)
 static int be_copy_wait_released(void* ctx, int slot) {
   tpi_model* m = (tpi_model*)ctx;
@@ -351,7 +386,13 @@ static int be_copy_wait_released(void* ctx, int slot) {
 static int be_copy_block(void* ctx, int slot, int block) {
   tpi_model* m = (tpi_model*)ctx;
   const size_t n = block_size(m, block);
+  cudaEvent_t a = nullptr, b = nullptr;
+  if (m->sched_rec && (a = sched_event(m)) && (b = sched_event(m))) CK(cudaEventRecord(a, m->ps));
   CK(cudaMemcpyAsync(slot_ptr(m, slot), host_image(m, block), n, cudaMemcpyHostToDevice, m->ps));
+  if (a && b) {
+    CK(cudaEventRecord(b, m->ps));
+    m->sched_pending.push_back({a, b, 2 + (block & 1)});
+  } else if (a) m->sched_free.push_back(a);
   m->link_bytes += n;
   return 0;
 }
@@ -626,6 +667,9 @@ extern "C" void tpi_free(tpi_model* m) {
   for (auto e : m->ev_released) cudaEventDestroy(e);
   for (auto e : m->prof_ev) cudaEventDestroy(e);
   for (auto e : m->stall_ev) cudaEventDestroy(e);
+  for (auto& tp : m->sched_pending) { cudaEventDestroy(tp.a); cudaEventDestroy(tp.b); }
+  for (auto e : m->sched_free) cudaEventDestroy(e);
+  if (m->sched_open) cudaEventDestroy(m->sched_open);
   if (m->ev_t0) cudaEventDestroy(m->ev_t0);
   if (m->ev_t1) cudaEventDestroy(m->ev_t1);
   if (m->ev_done) cudaEventDestroy(m->ev_done);
@@ -741,15 +785,26 @@ struct BlockRef {
   int slot;
 };
 static int acquire_block(tpi_model* m, int block, BlockRef* r) {
-  if (m->window <= 0) { r->base = resident_block(m, block); r->slot = -1; return TPI_OK; }
-  if (m->retained[block]) { r->base = m->dev + m->plan.blocks + m->retained_off[block]; r->slot = -1; return TPI_OK; }
-  const int s = m->ring.acquire(block);
-  if (s < 0) return s == -1000 || s == -1001 ? fail(TPI_ERR_STATE, "window ring out of order (%d)", s) : s;
-  r->base = slot_ptr(m, s);
-  r->slot = s;
+  if (m->window <= 0) { r->base = resident_block(m, block); r->slot = -1; }
+  else if (m->retained[block]) { r->base = m->dev + m->plan.blocks + m->retained_off[block]; r->slot = -1; }
+  else {
+    const int s = m->ring.acquire(block);
+    if (s < 0) return s == -1000 || s == -1001 ? fail(TPI_ERR_STATE, "window ring out of order (%d)", s) : s;
+    r->base = slot_ptr(m, s);
+    r->slot = s;
+  }
+  if (m->sched_rec && (m->sched_open = sched_event(m))) CK(cudaEventRecord(m->sched_open, m->cs));  // after the wait
   return TPI_OK;
 }
 static int release_block(tpi_model* m, int block) {
+  if (m->sched_open) {
+    cudaEvent_t b = sched_event(m);
+    if (b) {
+      CK(cudaEventRecord(b, m->cs));
+      m->sched_pending.push_back({m->sched_open, b, block & 1});
+    } else m->sched_free.push_back(m->sched_open);
+    m->sched_open = nullptr;
+  }
   if (m->window <= 0 || m->retained[block]) return TPI_OK;
   const int rc = m->ring.release(block);
   if (rc == -1000) return fail(TPI_ERR_STATE, "window ring out of order");
@@ -849,6 +904,7 @@ static void harvest_profile(tpi_model* m) {
     if (cudaEventElapsedTime(&ms, m->stall_ev[i], m->stall_ev[i + 1]) == cudaSuccess) m->stall_ms += ms;
   }
   m->stall_used = 0;
+  sched_harvest(m);
 }
 
 static int check_device_error(tpi_model* m, const int* io_err) {
@@ -884,7 +940,10 @@ static int run_decode(tpi_model* m, int32_t token_in, int n_steps, int32_t* toke
     } else if (use_graph) { CK(cudaGraphLaunch(m->graph_exec, m->cs)); launches += m->graph_launches; }
     else {
       LaunchCtx lc{m->cs, m->opt_pdl != 0 && !m->opt_profile, &launches};
-      TRY(enqueue_decode(m, lc));
+      m->sched_rec = m->opt_profile != 0;
+      const int rc = enqueue_decode(m, lc);
+      m->sched_rec = false;
+      TRY(rc);
     }
   }
   CK(cudaEventRecord(m->ev_t1, m->cs));
@@ -1124,6 +1183,81 @@ int tr_xrr(void* c, int s) { return tr_push(c, 4, s, -1); }
 // triples (op, slot, block): op 0 copy-queue waits for release of slot, 1 copy block into slot,
 // 2 copy-queue marks slot loaded, 3 compute-queue waits for slot, 4 compute-queue releases slot.
 // Returns the number of operations (may exceed max_ops) or a negative status.
+// ------------------------------------------------------------------------------ steady-state diagnostics
+// Prop. 3, Prop. 4 and Prop. 6 evaluated on given latencies (host arithmetic only).
+extern "C" int tpi_steady_conditions(double t_attn, double t_ffn, double t_all_reduce, double tau_attn, double tau_ffn,
+                                     int n_layers, int* tight, int* loose, int* retention_T) {
+  if (n_layers < 1 || !(t_attn >= 0) || !(t_ffn >= 0) || !(t_all_reduce >= 0) || !(tau_attn >= 0) || !(tau_ffn >= 0))
+    return fail(TPI_ERR_INVALID_ARG, "bad argument");
+  const double ca = t_attn + t_all_reduce, cf = t_ffn + t_all_reduce;  // a block's compute with its allreduce
+  if (tight) *tight = ca >= tau_ffn && cf >= tau_attn;
+  // Prop. 3: one layer's compute covers one layer's loads, and one of the two prefix families holds for every l
+  bool fam_a = true, fam_b = true;
+  for (int l = 1; l <= n_layers; ++l) {
+    if (l * ca + (l - 1) * cf < l * tau_ffn + (l - 1) * tau_attn) fam_a = false;
+    if ((l - 1) * ca + l * cf < (l - 1) * tau_ffn + l * tau_attn) fam_b = false;
+  }
+  const bool loose_ok = ca + cf >= tau_ffn + tau_attn && (fam_a || fam_b);
+  if (loose) *loose = loose_ok;
+  if (retention_T) {
+    // Prop. 6: with one FFN block in every T kept, ceil(l/T) of the first l FFN loads disappear; both prefix
+    // families must hold.  Fewer kept blocks (larger T) only add loads, so scan from the cheapest setting down.
+    int best = -1;
+    for (int T = n_layers; T >= 1 && best < 0; --T) {
+      bool ok = true;
+      for (int l = 1; l <= n_layers && ok; ++l) {
+        const double ffn_loads = (double)(l - (l + T - 1) / T) * tau_ffn;
+        if (l * ca + l * cf < ffn_loads + l * tau_attn) ok = false;
+        if (l * ca + (l - 1) * cf < ffn_loads + (l - 1) * tau_attn) ok = false;
+      }
+      if (ok) best = T;
+    }
+    *retention_T = loose_ok ? 0 : best;
+  }
+  return TPI_OK;
+}
+
+extern "C" int tpi_scheduler_report(tpi_model* m, tpi_sched_report* out) {
+  if (!m || !out) return fail(TPI_ERR_INVALID_ARG, "null argument");
+  sched_harvest(m);
+  tpi_sched_report r;
+  memset(&r, 0, sizeof r);
+  double mean[4];
+  for (int k = 0; k < 4; ++k) mean[k] = m->sched_n[k] ? m->sched_sum[k] / m->sched_n[k] : 0.0;
+  r.t_attn_ms = mean[0]; r.t_ffn_ms = mean[1]; r.tau_attn_ms = mean[2]; r.tau_ffn_ms = mean[3];
+  r.n_t_attn = m->sched_n[0]; r.n_t_ffn = m->sched_n[1]; r.n_tau_attn = m->sched_n[2]; r.n_tau_ffn = m->sched_n[3];
+  r.t_all_reduce_ms = 0.0;  // the rank-ordered sum runs inside the block's last kernel: it is part of t_attn / t_ffn
+  r.stall_ms_total = m->stall_ms;
+  r.tight_holds = r.loose_holds = r.retention_T = -2;
+  const bool have_t = r.n_t_attn && r.n_t_ffn;
+  // a retained or resident block has no load: its tau counts as 0 only when nothing of that kind is streamed
+  const bool streams_ffn = m->window > 0 && m->retain_T != 1;
+  const bool have_tau = m->window > 0 && r.n_tau_attn && (r.n_tau_ffn || !streams_ffn);
+  if (have_t && have_tau)
+    TRY(tpi_steady_conditions(r.t_attn_ms, r.t_ffn_ms, 0.0, r.tau_attn_ms, r.tau_ffn_ms, m->cfg.n_layers, &r.tight_holds,
+                              &r.loose_holds, &r.retention_T));
+  r.window_blocks = m->window;
+  r.retain_every_T = m->window > 0 ? m->retain_T : 0;
+  if (m->window > 0) {
+    int nA, nF;
+    window_slots(m->window, &nA, &nF);
+    // Prop. 5 without the empirical factor: floor(w/2) attention blocks + ceil(w/2) FFN blocks
+    r.m_worker_bytes = (uint64_t)(m->window / 2) * m->plan.bl.attn_bytes + (uint64_t)((m->window + 1) / 2) * m->plan.bl.ffn_bytes;
+    r.window_device_bytes = (uint64_t)nA * m->plan.bl.attn_bytes + (uint64_t)nF * m->plan.bl.ffn_bytes + m->retained_bytes;
+  }
+  *out = r;
+  return TPI_OK;
+}
+
+extern "C" int tpi_scheduler_reset(tpi_model* m) {
+  if (!m) return fail(TPI_ERR_INVALID_ARG, "null model");
+  TRY(quiesce(m));
+  sched_harvest(m);
+  for (int k = 0; k < 4; ++k) { m->sched_sum[k] = 0; m->sched_n[k] = 0; }
+  m->stall_ms = 0;
+  return TPI_OK;
+}
+
 extern "C" int tpi_ring_trace(int n_blocks, int w, int n_exec, int* ops, int max_ops) {
   return tpi_ring_trace_retained(n_blocks, w, n_exec, 0, ops, max_ops);
 }

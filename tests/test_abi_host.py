@@ -177,3 +177,27 @@ def test_ring_invariants():
             assert all(len(k) == 1 for k in kinds.values())
             n_attn = sum(1 for k in kinds.values() if k == {0})
             assert n_attn == w // 2 and len(kinds) - n_attn == (w + 1) // 2
+
+
+# ----------------------------------------------------------------- steady-state diagnostics (Prop. 3, 4, 6)
+def test_steady_conditions_match_the_oracle_and_the_worked_example():
+    # the paper's worked example: tight fails, loose holds, so no retention is needed
+    assert P.steady_conditions(11, 17, 14, 18, 30, 32) == (False, True, 0)
+    rng = np.random.default_rng(7)
+    seen = set()
+    for _ in range(400):
+        ta, tf, la, lf = rng.integers(1, 40, 4).astype(float)
+        tr = float(rng.integers(0, 12))
+        L = int(rng.integers(1, 20))
+        tight, loose, T = P.steady_conditions(ta, tf, tr, la, lf, L)
+        assert tight == W.tight_condition(ta, tf, tr, la, lf)
+        assert loose == W.loose_condition(ta, tf, tr, la, lf, L)
+        ok = [t for t in range(1, L + 1) if W.retention_condition(ta, tf, tr, la, lf, L, t)]
+        want = 0 if loose else (max(ok) if ok else -1)
+        assert T == want, (ta, tf, tr, la, lf, L)
+        seen.add(min(T, 1))
+    assert seen == {-1, 0, 1}                                   # every outcome occurred
+    # the allreduce term only ever appears added to a block's compute time
+    assert P.steady_conditions(11, 17, 14, 18, 30, 32) == P.steady_conditions(25, 31, 0, 18, 30, 32)
+    with pytest.raises(P.TpiError):
+        P.steady_conditions(-1, 1, 1, 1, 1, 4)

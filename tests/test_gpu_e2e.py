@@ -1,6 +1,7 @@
 """End-to-end parity of the CUDA library against the CPU oracle through the C ABI
 (tiny fp32 workload C1, full depth; small bf16 / grouped-head variants)."""
 import numpy as np
+import torch
 import pytest
 
 import tpi_synth as S
@@ -131,7 +132,7 @@ def test_block_retention_is_bit_identical_and_loads_less(window, T):
     """Prop. 6's retention: the kept FFN blocks never cross the link again, the rest stream as before,
     and the tokens and logits are the same bits as the resident run's."""
     import paper_2410_00531_b200 as P
-    from helpers import tpi_config
+    from tests.helpers import tpi_config
     shape = S.CONFIGS["C1"].with_(n_layers=6)
     toks = S.prompt_tokens(shape)
     _, ffn_bytes = P.block_bytes(tpi_config(shape, 64, 16))
@@ -164,6 +165,37 @@ def test_block_retention_is_bit_identical_and_loads_less(window, T):
         assert a[0] == b[0] and a[3] == b[3] and (a[2] == b[2]).all()
         assert np.array_equal(a[1], b[1]) and np.array_equal(a[4], b[4])
     assert loads["retained"] < loads["streamed"]
+
+
+def test_scheduler_report_measures_the_propositions_inputs():
+    """Sec. 3.3's diagnostics: block compute and load latencies measured on the run, Prop. 3/4/6 evaluated on them."""
+    import paper_2410_00531_b200 as P
+    from tests.helpers import tpi_config
+    shape = S.CONFIGS["C1"].with_(n_layers=4)
+    toks = S.prompt_tokens(shape)
+    attn_b, ffn_b = P.block_bytes(tpi_config(shape, 64, 16))
+    with gpu_session(shape, 64, 16, 2, 3) as ses:
+        P.set_option(ses.h, P.OPT_PROFILE, 1)
+        t0, _ = P.prefill(ses.h, toks, 0)
+        assert P.scheduler_report(ses.h)["n_t_attn"] == 0          # the prompt pass is not sampled
+        P.decode_run(ses.h, t0, 5)
+        torch.cuda.synchronize()
+        r = P.scheduler_report(ses.h)
+        assert r["n_t_attn"] == r["n_t_ffn"] == 5 * shape.n_layers
+        assert r["n_tau_attn"] >= 5 * shape.n_layers - 2 and r["n_tau_ffn"] >= 5 * shape.n_layers - 2
+        assert min(r["t_attn_ms"], r["t_ffn_ms"], r["tau_attn_ms"], r["tau_ffn_ms"]) > 0 and r["t_all_reduce_ms"] == 0
+        want = P.steady_conditions(r["t_attn_ms"], r["t_ffn_ms"], 0.0, r["tau_attn_ms"], r["tau_ffn_ms"], shape.n_layers)
+        assert (bool(r["tight_holds"]), bool(r["loose_holds"]), r["retention_T"]) == want
+        assert r["window_blocks"] == 3 and r["m_worker_bytes"] == attn_b + 2 * ffn_b == r["window_device_bytes"]
+        P.scheduler_reset(ses.h)
+        assert P.scheduler_report(ses.h)["n_t_ffn"] == 0
+    with gpu_session(shape, 64, 16, 2, 0) as ses:                  # resident: compute samples only, no verdicts
+        P.set_option(ses.h, P.OPT_PROFILE, 1)
+        t0, _ = P.prefill(ses.h, toks, 0)
+        P.decode_run(ses.h, t0, 3)
+        r = P.scheduler_report(ses.h)
+        assert r["n_t_attn"] == 3 * shape.n_layers and r["n_tau_attn"] == 0
+        assert r["tight_holds"] == r["loose_holds"] == r["retention_T"] == -2 and r["m_worker_bytes"] == 0
 
 
 def test_set_shards_and_set_window_roundtrip():
