@@ -109,6 +109,7 @@ __device__ __forceinline__ void cols_body(const GemvArgs& A, float* xs, const in
   constexpr int R = 2, XR = 4;
   __shared__ float red[32];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nw = WARPS > 0 ? WARPS : (int)(blockDim.x >> 5);  // WARPS == 0: the launch decides (up to 32 warps)
   const long long total = (long long)A.items_per_shard * A.n_shards;
   const int lo = (int)(total * cta / ncta), hi = (int)(total * (cta + 1) / ncta);
   const uint32_t row_bytes = (uint32_t)(A.K * sizeof(WT));
@@ -143,11 +144,11 @@ __device__ __forceinline__ void cols_body(const GemvArgs& A, float* xs, const in
   // ---- prologue: one round trip to L2 for the statistics, x and the gain together
   float ss = 0.f;
   if (A.ss_part)
-    for (int i = threadIdx.x; i < A.n_parts; i += WARPS * 32) ss += A.ss_part[i];
+    for (int i = threadIdx.x; i < A.n_parts; i += nw * 32) ss += A.ss_part[i];
   float4 xr[XR], gr[XR];
 #pragma unroll
   for (int j = 0; j < XR; ++j) {
-    const int k = (threadIdx.x + j * WARPS * 32) * 4;
+    const int k = (threadIdx.x + j * nw * 32) * 4;
     if (k < A.K) {
       xr[j] = *reinterpret_cast<const float4*>(A.x + k);
       gr[j] = A.gain ? *reinterpret_cast<const float4*>(A.gain + k) : make_float4(1.f, 1.f, 1.f, 1.f);
@@ -160,7 +161,7 @@ __device__ __forceinline__ void cols_body(const GemvArgs& A, float* xs, const in
   }
 #pragma unroll
   for (int j = 0; j < XR; ++j) {
-    const int k = (threadIdx.x + j * WARPS * 32) * 4;
+    const int k = (threadIdx.x + j * nw * 32) * 4;
     if (k < A.K) {
       float4 v = xr[j];
       if (A.ss_part) { v.x *= rnorm; v.y *= rnorm; v.z *= rnorm; v.w *= rnorm; }
@@ -168,7 +169,7 @@ __device__ __forceinline__ void cols_body(const GemvArgs& A, float* xs, const in
       *reinterpret_cast<float4*>(xs + k) = v;
     }
   }
-  for (int k = (threadIdx.x + XR * WARPS * 32) * 4; k < A.K; k += WARPS * 32 * 4) {
+  for (int k = (threadIdx.x + XR * nw * 32) * 4; k < A.K; k += nw * 32 * 4) {
     float4 v = *reinterpret_cast<const float4*>(A.x + k);
     if (A.ss_part) { v.x *= rnorm; v.y *= rnorm; v.z *= rnorm; v.w *= rnorm; }
     if (A.gain) {
@@ -183,7 +184,7 @@ __device__ __forceinline__ void cols_body(const GemvArgs& A, float* xs, const in
   const int nvec = A.K / Elem<WT>::VEC;
   float bv = -INFINITY;  // EPI_LOGITS: this warp's running best
   int bi = 0x7FFFFFFF;
-  for (int it = lo + warp; it < hi; it += WARPS) {
+  for (int it = lo + warp; it < hi; it += nw) {
     int shard, item;
     const uint4* wp[R];
     row_ptrs(it, shard, item, wp);
@@ -235,13 +236,13 @@ __device__ __forceinline__ void cols_body(const GemvArgs& A, float* xs, const in
     }
   }
   if constexpr (EPI == EPI_LOGITS) {
-    __shared__ float s_val[WARPS];
-    __shared__ int s_idx[WARPS];
+    __shared__ float s_val[WARPS > 0 ? WARPS : 32];
+    __shared__ int s_idx[WARPS > 0 ? WARPS : 32];
     __shared__ bool s_last;
     if (lane == 0) { s_val[warp] = bv; s_idx[warp] = bi; }
     __syncthreads();
     if (threadIdx.x == 0) {
-      for (int w = 1; w < WARPS; ++w)
+      for (int w = 1; w < nw; ++w)
         if (s_val[w] > bv || (s_val[w] == bv && s_idx[w] < bi)) { bv = s_val[w]; bi = s_idx[w]; }
       A.amax_val[cta] = bv;
       A.amax_idx[cta] = bi;
@@ -297,8 +298,9 @@ struct RowFusedArgs {
 // NS > 0: the shard count is a compile-time constant (1, 2, 4, 8); NS == 0: any N, shard by shard.
 template <typename WT, int R, int NS, int WARPS>
 __device__ __forceinline__ void rowfused_body(const RowFusedArgs& A, float* xs, const int cta, const int ncta) {
-  __shared__ float s_sq[WARPS];
+  __shared__ float s_sq[WARPS > 0 ? WARPS : 32];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nw = WARPS > 0 ? WARPS : (int)(blockDim.x >> 5);
   const int groups = A.rows / R;
   const int lo = (int)((long long)groups * cta / ncta);
   const int hi = (int)((long long)groups * (cta + 1) / ncta);
@@ -312,14 +314,14 @@ __device__ __forceinline__ void rowfused_body(const RowFusedArgs& A, float* xs, 
   pdl_wait();
 
   const int ktot = A.n_shards * A.Ks;
-  for (int k = threadIdx.x * 4; k < ktot; k += WARPS * 32 * 4)
+  for (int k = threadIdx.x * 4; k < ktot; k += nw * 32 * 4)
     *reinterpret_cast<float4*>(xs + k) = *reinterpret_cast<const float4*>(A.x_in + k);
   __syncthreads();
 
   constexpr int VEC = Elem<WT>::VEC;
   const int nvec = A.Ks / VEC;
   float sq = 0.f;
-  for (int g = lo + warp; g < hi; g += WARPS) {
+  for (int g = lo + warp; g < hi; g += nw) {
     const int row0 = g * R;
     float sum[R], res[R];
 #pragma unroll
@@ -394,7 +396,7 @@ __device__ __forceinline__ void rowfused_body(const RowFusedArgs& A, float* xs, 
   __syncthreads();
   if (threadIdx.x == 0) {
     float t = s_sq[0];
-    for (int w = 1; w < WARPS; ++w) t += s_sq[w];
+    for (int w = 1; w < nw; ++w) t += s_sq[w];
     A.ss_part[cta] = t;
     for (int i = cta + ncta; i < A.n_parts; i += ncta) A.ss_part[i] = 0.f;
   }

@@ -20,7 +20,7 @@ struct Tuning {
   int cps_cols = 4;          // CTAs per SM, column-sharded GEMVs
   int cps_rows = 4;          // CTAs per SM, fused row-sharded GEMVs
   int prefetch_bytes = 4096; // L2 prefetch per row issued before the dependency wait
-  int warps = 8;             // warps per CTA of the persistent GEMVs (8, 16 or 32)
+  int warps = 0;             // 0: one CTA per SM with a balanced warp count; 8, 16, 32: that many warps, cps CTAs per SM
   int mega_prefetch = 2048;  // whole-token kernel: bytes per row requested from L2 ahead of a barrier
 };
 static Tuning g_tune;
@@ -42,6 +42,29 @@ static int sm_count() {
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
   }
   return n;
+}
+
+// Work split of the persistent GEMVs.  `items` equal work items go to one CTA per SM as contiguous ranges, and
+// inside a CTA warp w takes items w, w + W, ...: the kernel ends when the fullest warp ends, so W is chosen so
+// that the busiest CTA's items fill its warps' rounds with little left over (a 7B-shaped gate/up projection has
+// 74.4 row pairs per SM: 32 warps would need 3 rounds for 2.3 rounds of work, 25 warps fill 3 rounds exactly).
+// Fewer warps keep fewer loads in flight, hence the weight below 20 warps.
+constexpr int lb_threads(int w) { return w > 0 ? w * 32 : 1024; }
+constexpr int lb_blocks(int w) { return w > 0 ? 32 / w : 1; }
+static void balance_split(long long items, int* grid, int* warps) {
+  const int sms = sm_count();
+  const int g = (int)(items < sms ? (items < 1 ? 1 : items) : sms);
+  const long long per = (items + g - 1) / g;  // items of the busiest CTA
+  double best = -1.0;
+  int bw = 8;
+  for (int w = 32; w >= 4; --w) {
+    const long long rounds = (per + w - 1) / w;
+    const double fill = (double)items / g / (double)(rounds * w);
+    const double score = fill * (w >= 20 ? 1.0 : w / 20.0);
+    if (score > best + 1e-9) { best = score; bw = w; }
+  }
+  *grid = g;
+  *warps = bw;
 }
 
 template <typename WT, int R, int EPI, int WARPS>
@@ -193,7 +216,7 @@ __global__ void __launch_bounds__(WARPS * 32) gemv_kernel(const GemvArgs A) {
 
 
 template <typename WT, int EPI, int WARPS>
-__global__ void __launch_bounds__(WARPS * 32, 32 / WARPS) gemv_cols_kernel(const GemvArgs A) {
+__global__ void __launch_bounds__(lb_threads(WARPS), lb_blocks(WARPS)) gemv_cols_kernel(const GemvArgs A) {
   extern __shared__ __align__(16) float xs[];
   cols_body<WT, EPI, WARPS>(A, xs, blockIdx.x, gridDim.x);
 }
@@ -203,8 +226,15 @@ static cudaError_t launch_gemv_cols_w(const LaunchCtx& c, GemvArgs& A) {
   A.prefetch_bytes = g_tune.prefetch_bytes;
   const long long total = (long long)A.items_per_shard * A.n_shards;
   long long grid = (long long)sm_count() * g_tune.cps_cols;
-  if (grid > (total + WARPS - 1) / WARPS) grid = (total + WARPS - 1) / WARPS;
-  if (grid < 1) grid = 1;
+  int warps = WARPS;
+  if (WARPS > 0) {
+    if (grid > (total + WARPS - 1) / WARPS) grid = (total + WARPS - 1) / WARPS;
+    if (grid < 1) grid = 1;
+  } else {
+    int g;
+    balance_split(total, &g, &warps);
+    grid = g;
+  }
   auto kern = gemv_cols_kernel<WT, EPI, WARPS>;
   static bool attr_done = false;
   if (!attr_done) {
@@ -212,10 +242,11 @@ static cudaError_t launch_gemv_cols_w(const LaunchCtx& c, GemvArgs& A) {
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  return launch_kernel(c, kern, dim3((unsigned)grid), dim3(WARPS * 32), (size_t)A.K * sizeof(float), A);
+  return launch_kernel(c, kern, dim3((unsigned)grid), dim3(warps * 32), (size_t)A.K * sizeof(float), A);
 }
 template <typename WT, int EPI>
 static cudaError_t launch_gemv_cols_t(const LaunchCtx& c, GemvArgs& A) {
+  if (g_tune.warps <= 0) return launch_gemv_cols_w<WT, EPI, 0>(c, A);
   if (g_tune.warps >= 32) return launch_gemv_cols_w<WT, EPI, 32>(c, A);
   if (g_tune.warps >= 16) return launch_gemv_cols_w<WT, EPI, 16>(c, A);
   return launch_gemv_cols_w<WT, EPI, 8>(c, A);
@@ -299,7 +330,8 @@ cudaError_t launch_gemv_partials(const LaunchCtx& c, int dt, const void* W, size
 static int head_rows_per_warp(int vocab) { return vocab % 2 == 0 ? 2 : 1; }
 int head_argmax_blocks(int vocab) {
   const int R = head_rows_per_warp(vocab);
-  return (vocab / R + 7) / 8;
+  const int per_item = (vocab / R + 7) / 8, per_sm = sm_count() * 4;  // an upper bound of every grid the head kernel uses
+  return per_item > per_sm ? per_item : per_sm;
 }
 
 cudaError_t launch_head_argmax(const LaunchCtx& c, int dt, const void* Whead, const NormIn& in,
@@ -321,7 +353,8 @@ cudaError_t launch_head_argmax(const LaunchCtx& c, int dt, const void* Whead, co
 }
 
 template <typename WT, int R, int NS, int WARPS>
-__global__ void __launch_bounds__(WARPS * 32, 32 / WARPS) gemv_rowshard_fused_kernel(const RowFusedArgs A) {
+__global__ void __launch_bounds__(lb_threads(WARPS), lb_blocks(WARPS))
+    gemv_rowshard_fused_kernel(const RowFusedArgs A) {
   extern __shared__ __align__(16) float xs[];
   rowfused_body<WT, R, NS, WARPS>(A, xs, blockIdx.x, gridDim.x);
 }
@@ -343,16 +376,21 @@ static cudaError_t launch_rowfused_w(const LaunchCtx& c, RowFusedArgs& A) {
   const int fit = (int)((220 * 1024) / (smem + 1024));
   if (cps > fit) cps = fit < 1 ? 1 : fit;
   const int groups = A.rows / R;
-  int grid = sm_count() * cps;
-  if (grid > (groups + WARPS - 1) / WARPS) grid = (groups + WARPS - 1) / WARPS;
-  if (grid < 1) grid = 1;
-  return launch_kernel(c, kern, dim3(grid), dim3(WARPS * 32), smem, A);
+  int grid = sm_count() * cps, warps = WARPS;
+  if (WARPS > 0) {
+    if (grid > (groups + WARPS - 1) / WARPS) grid = (groups + WARPS - 1) / WARPS;
+    if (grid < 1) grid = 1;
+  } else {
+    balance_split(groups, &grid, &warps);
+  }
+  return launch_kernel(c, kern, dim3(grid), dim3(warps * 32), smem, A);
 }
 
 template <typename WT, int R, int NS>
 static cudaError_t launch_rowfused_t(const LaunchCtx& c, RowFusedArgs& A) {
   // Keep about 32 warps per SM: when the staged x_in is so large that fewer than four CTAs fit in an
   // SM's shared memory, make the CTAs bigger instead (70B-shaped down projection: 112 KiB of x_in).
+  if (g_tune.warps <= 0) return launch_rowfused_w<WT, R, NS, 0>(c, A);
   const size_t smem = (size_t)A.Ks * A.n_shards * sizeof(float);
   const int fit = (int)((220 * 1024) / (smem + 1024));
   int warps = g_tune.warps;
