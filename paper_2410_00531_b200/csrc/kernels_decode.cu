@@ -227,7 +227,7 @@ static cudaError_t launch_gemv_cols_w(const LaunchCtx& c, GemvArgs& A) {
   const long long total = (long long)A.items_per_shard * A.n_shards;
   long long grid = (long long)sm_count() * g_tune.cps_cols;
   int warps = WARPS;
-  if (WARPS > 0) {
+  if constexpr (WARPS > 0) {
     if (grid > (total + WARPS - 1) / WARPS) grid = (total + WARPS - 1) / WARPS;
     if (grid < 1) grid = 1;
   } else {
@@ -377,7 +377,7 @@ static cudaError_t launch_rowfused_w(const LaunchCtx& c, RowFusedArgs& A) {
   if (cps > fit) cps = fit < 1 ? 1 : fit;
   const int groups = A.rows / R;
   int grid = sm_count() * cps, warps = WARPS;
-  if (WARPS > 0) {
+  if constexpr (WARPS > 0) {
     if (grid > (groups + WARPS - 1) / WARPS) grid = (groups + WARPS - 1) / WARPS;
     if (grid < 1) grid = 1;
   } else {
