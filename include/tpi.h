@@ -178,6 +178,8 @@ typedef struct {
   uint64_t window_peak_bytes;  /* device bytes held by window slots                      */
   uint64_t retained_bytes;     /* device bytes held by retained blocks (block retention) */
   int32_t retained_blocks, reserved_;
+  double last_prefill_dev_ms;     /* the last tpi_prefill's kernels timed with CUDA events             */
+  double last_prefill_enqueue_ms; /* host time that call spent enqueueing them (before it waited)      */
 } tpi_stats;
 int tpi_get_stats(tpi_model *m, tpi_stats *out);
 

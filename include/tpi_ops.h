@@ -115,6 +115,19 @@ int tpi_op_gemm_bf16(const void *A, const void *A_lo, int lda, int a_col_batch, 
                      long long y_bs, int ldy, int T, int n_out, int K, int n_batch, int32_t *err_word,
                      void *stream);
 
+/* The gate/up projection of Eq. 2 for T positions with SwiGLU applied in the GEMM's epilogue:
+ * ACT[t][j] = silu(y[t][2j]) * y[t][2j+1], y = A . Wgu^T, Wgu bf16 [2 s][K] with rows interleaved
+ * gate_j, up_j (all shards, shard-major).  A, A_lo as tpi_op_gemm_bf16 (one batch).  ACT: bf16 [T][s];
+ * with split_out != 0 a second bf16 tensor bf16(v - hi) follows T*s elements later.  s % 16 == 0. */
+int tpi_op_gemm_bf16_swiglu(const void *A, const void *A_lo, int lda, const void *Wgu, void *ACT, int split_out, int T,
+                            int s, int K, int32_t *err_word, void *stream);
+
+/* Eq. 1-2's star sum and shortcut for T positions followed by the next block's RMSNorm:
+ * X[t] <- ((P_0[t] + P_1[t]) + ...) + X[t];  Xn[t] = X[t] * rsqrt(mean(X[t]^2) + rms_eps) * gain.
+ * partials: float[n_shards][T][h]; X in/out float[T][h]; gain float[h]; Xn float[T][h]. */
+int tpi_op_reduce_residual_norm_rows(const float *partials, int n_shards, int T, int h, float *X, const float *gain,
+                                     float rms_eps, float *Xn, void *stream);
+
 /* Causal attention of T query positions [pos0, pos0+T) over cache positions [0, pos0+T).
  * Q, O: float[T][a][d]. */
 int tpi_op_prefill_attention(int dtype, const float *Q, const void *kcache, const void *vcache, int T, int pos0,

@@ -50,7 +50,8 @@ class TpiStats(C.Structure):
                 ("kernel_launches_last", C.c_int32), ("window_blocks", C.c_int32),
                 ("n_shards", C.c_int32), ("position", C.c_int32), ("graph_active", C.c_int32),
                 ("window_peak_bytes", C.c_uint64), ("retained_bytes", C.c_uint64),
-                ("retained_blocks", C.c_int32), ("reserved_", C.c_int32)]
+                ("retained_blocks", C.c_int32), ("reserved_", C.c_int32),
+                ("last_prefill_dev_ms", C.c_double), ("last_prefill_enqueue_ms", C.c_double)]
 
     def as_dict(self) -> dict:
         return {k: getattr(self, k) for k, _ in self._fields_}

@@ -1007,12 +1007,16 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
     return TPI_OK;
   };
   CK(launch_embed_rows(lc, dt, m->dev + p.emb, dptr<int>(m, p.tok_hist), pos0, T, c.vocab, h, X, err));
+  // With every block resident, the kernel that ends a block (star sum + shortcut) also applies the next block's
+  // RMSNorm, whose gain lives in that next block's image; a streamed model may not hold the next block yet.
+  const bool fuse_norm = m->window <= 0;
+  bool normed = false;  // Xn already holds the input of the block about to start
   for (int l = 0; l < c.n_layers; ++l) {
     BlockRef br;
     TRY(acquire_block(m, 2 * l, &br));
     void* kc = m->dev + p.kcache + (size_t)l * p.kv_layer_bytes;
     void* vc = m->dev + p.vcache + (size_t)l * p.kv_layer_bytes;
-    CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, act_mode));
+    if (!normed) CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, act_mode));
     TRY(proj(Xn, h, 0, br.base + bl.off_qkv, qkv_cols, QKV, 0, qkv_cols, qkv_cols, h, 1));
     CK(launch_rope_kv_rows(lc, dt, QKV, T, pos0, N, a, b, d, c.max_seq, rope, Q, kc, vc));
     if (m->opt_tensor && prefill_attention_mma_supported(dt, d))
@@ -1020,14 +1024,28 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
     else
       CK(launch_prefill_attention(lc, dt, Q, kc, vc, T, pos0, a, b, d, c.max_seq, O, act_mode));
     TRY(proj(O, a * d, Ko, br.base + bl.off_wo, h, PART, (long long)T * h, h, h, Ko, N));
-    CK(launch_reduce_residual_rows(lc, PART, N, T, h, X, last ? dptr<float>(m, p.taps) + (size_t)(2 * l) * h : nullptr));
+    float* tap_a = last ? dptr<float>(m, p.taps) + (size_t)(2 * l) * h : nullptr;
+    if (fuse_norm)
+      CK(launch_reduce_residual_norm_rows(lc, PART, N, T, h, X, tap_a, (const float*)resident_block(m, 2 * l + 1), c.rms_eps, Xn, act_mode));
+    else
+      CK(launch_reduce_residual_rows(lc, PART, N, T, h, X, tap_a));
     TRY(release_block(m, 2 * l));
     TRY(acquire_block(m, 2 * l + 1, &br));
-    CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, act_mode));
-    TRY(proj(Xn, h, 0, br.base + bl.off_gu, 2 * s, GU, 0, 2 * s, 2 * s, h, 1));
-    CK(launch_swiglu_rows(lc, GU, T, s, ACT, act_mode));
+    if (!fuse_norm) CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, act_mode));
+    if (tc && gemm_tc_swiglu_supported(h, h, s)) {  // SwiGLU in the GEMM's epilogue: the fp32 gate/up rows never reach memory
+      const __nv_bfloat16* hi = reinterpret_cast<const __nv_bfloat16*>(Xn);
+      CK(launch_gemm_tc_swiglu(lc, hi, act_mode == 2 ? hi + (size_t)T * h : nullptr, h, br.base + bl.off_gu, ACT, act_mode, T, s, h, err));
+    } else {
+      TRY(proj(Xn, h, 0, br.base + bl.off_gu, 2 * s, GU, 0, 2 * s, 2 * s, h, 1));
+      CK(launch_swiglu_rows(lc, GU, T, s, ACT, act_mode));
+    }
     TRY(proj(ACT, s, Kd, br.base + bl.off_down, h, PART, (long long)T * h, h, h, Kd, N));
-    CK(launch_reduce_residual_rows(lc, PART, N, T, h, X, last ? dptr<float>(m, p.taps) + (size_t)(2 * l + 1) * h : nullptr));
+    float* tap_f = last ? dptr<float>(m, p.taps) + (size_t)(2 * l + 1) * h : nullptr;
+    normed = fuse_norm && l + 1 < c.n_layers;
+    if (normed)
+      CK(launch_reduce_residual_norm_rows(lc, PART, N, T, h, X, tap_f, (const float*)resident_block(m, 2 * l + 2), c.rms_eps, Xn, act_mode));
+    else
+      CK(launch_reduce_residual_rows(lc, PART, N, T, h, X, tap_f));
     TRY(release_block(m, 2 * l + 1));
   }
   if (last) {
@@ -1057,6 +1075,7 @@ extern "C" int tpi_prefill(tpi_model* m, const int32_t* tokens, int n_tokens, in
   int launches = 0;
   LaunchCtx lc{m->cs, m->opt_pdl != 0 && !m->opt_profile, &launches};
   const int p_begin = m->position;
+  CK(cudaEventRecord(m->ev_t0, m->cs));
   for (int t0 = 0; t0 < n_tokens; t0 += c.max_prefill) {
     const int T = n_tokens - t0 < c.max_prefill ? n_tokens - t0 : c.max_prefill;
     // token ids go through the pinned io area, one chunk at a time
@@ -1066,6 +1085,8 @@ extern "C" int tpi_prefill(tpi_model* m, const int32_t* tokens, int n_tokens, in
     CK(cudaEventRecord(m->ev_done, m->cs));
     TRY(enqueue_prefill_chunk(m, lc, p_begin + t0, T, t0 + T == n_tokens));
   }
+  CK(cudaEventRecord(m->ev_t1, m->cs));
+  m->st.last_prefill_enqueue_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - w0).count();
   CK(cudaMemcpyAsync(io + 2, dptr<int>(m, p.tok_hist) + p_begin + n_tokens, 4, cudaMemcpyDeviceToHost, m->cs));
   CK(cudaMemcpyAsync(io + 1, m->dev + p.err, 4, cudaMemcpyDeviceToHost, m->cs));
   if (logits_or_null) CK(cudaMemcpyAsync(m->host + p.h_logits, m->dev + p.logits, (size_t)c.vocab * 4, cudaMemcpyDeviceToHost, m->cs));
@@ -1075,6 +1096,10 @@ extern "C" int tpi_prefill(tpi_model* m, const int32_t* tokens, int n_tokens, in
   *first_token = io[2];
   if (logits_or_null) memcpy(logits_or_null, m->host + p.h_logits, (size_t)c.vocab * 4);
   m->st.last_prefill_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - w0).count();
+  {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, m->ev_t0, m->ev_t1) == cudaSuccess) m->st.last_prefill_dev_ms = ms;
+  }
   m->st.kernel_launches_last = launches;
   if (m->opt_profile) harvest_profile(m);
   return check_device_error(m, io + 1);

@@ -96,9 +96,34 @@ struct GemmTcArgs {
   int a_col_batch;  // A's column offset per batch (elements)
   int w_row_batch;  // W's row offset per batch
   int* err;
+  // SwiGLU epilogue (gate/up projection whose output columns are interleaved gate_j, up_j): when act != nullptr
+  // nothing is written to Y; act[t][c / 2] = silu(y[t][c]) * y[t][c + 1] goes out as bf16 (hi, and in split mode
+  // lo = bf16(v - hi) act_lo_off elements further), row stride act_ld.
+  __nv_bfloat16* act;
+  long long act_lo_off;
+  int act_ld, act_split;
 };
 
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[32]) {  // columns [0, 16) of r
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 constexpr int kBM = 128, kBK = 64;
+// tensor-memory columns are allocated in powers of two
+__host__ __device__ constexpr uint32_t tmem_cols(int bn) { return bn <= 32 ? 32u : bn <= 64 ? 64u : bn <= 128 ? 128u : 256u; }
+// pipeline depth that fits one SM's shared memory
+constexpr int stages_for(int bn, int split) {
+  const int stage = (1 + split) * kBM * kBK * 2 + bn * kBK * 2;
+  const int n = (226 * 1024 - 1024) / stage;
+  return n > 8 ? 8 : n;
+}
 
 // SPLIT = 1: the activations come as two bf16 tensors, A = A_hi + A_lo (A_lo = bf16(A - A_hi)), and every
 // k-block issues the MMAs twice onto the same accumulator.  That keeps ~16 mantissa bits of the fp32
@@ -110,6 +135,7 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES], acc_ready;
   __shared__ uint32_t tmem_base_s;
+  constexpr uint32_t TCOLS = tmem_cols(BN);
   constexpr uint32_t A_BYTES = kBM * kBK * 2, B_BYTES = BN * kBK * 2, STAGE_BYTES = (1 + SPLIT) * A_BYTES + B_BYTES;
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -123,7 +149,7 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {  // one warp allocates BN columns of tensor memory for the fp32 accumulator
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)BN) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(TCOLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -182,8 +208,46 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         uint32_t r[32];
+        if (BN - c0 < 32) {  // a tile width that is an odd multiple of 16: the last 16 columns (plain output only)
+          tmem_ld16(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+          if (row < a.T && !a.act)
+            for (int j = 0; j < 16; ++j)
+              if (n0 + c0 + j < a.n_out) yrow[c0 + j] = __uint_as_float(r[j]);
+          break;
+        }
         tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
-        if (row < a.T) {
+        if (row < a.T && a.act) {
+          __nv_bfloat16* arow = a.act + (size_t)row * a.act_ld + ((n0 + c0) >> 1);
+          uint32_t hi[8], lo[8];
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {  // two (gate, up) pairs -> two activations packed in one word
+            float v[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const float g = __uint_as_float(r[j + 2 * e]), u = __uint_as_float(r[j + 2 * e + 1]);
+              v[e] = g / (1.f + expf(-g)) * u;
+            }
+            const __nv_bfloat16 h0 = __float2bfloat16_rn(v[0]), h1 = __float2bfloat16_rn(v[1]);
+            hi[j >> 2] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+            const __nv_bfloat16 l0 = __float2bfloat16_rn(v[0] - __bfloat162float(h0)),
+                                l1 = __float2bfloat16_rn(v[1] - __bfloat162float(h1));
+            lo[j >> 2] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+          }
+          if (n0 + c0 + 32 <= a.n_out) {
+            *reinterpret_cast<uint4*>(arow) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4*>(arow + 8) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+            if (a.act_split) {
+              *reinterpret_cast<uint4*>(arow + a.act_lo_off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+              *reinterpret_cast<uint4*>(arow + a.act_lo_off + 8) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+            }
+          } else {
+            for (int j = 0; j < 16; ++j)
+              if (n0 + c0 + 2 * j + 1 < a.n_out) {
+                arow[j] = __ushort_as_bfloat16((unsigned short)(hi[j >> 1] >> ((j & 1) * 16)));
+                if (a.act_split) arow[a.act_lo_off + j] = __ushort_as_bfloat16((unsigned short)(lo[j >> 1] >> ((j & 1) * 16)));
+              }
+          }
+        } else if (row < a.T) {
           if (n0 + c0 + 32 <= a.n_out) {
 #pragma unroll
             for (int j = 0; j < 32; j += 4)
@@ -201,7 +265,7 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(TCOLS) : "memory");
   }
 }
 
@@ -267,29 +331,62 @@ static cudaError_t launch_tc_t(const LaunchCtx& c, const CUtensorMap& tmA, const
   return cudaLaunchKernelEx(&cfg, kern, tmA, tmAlo, tmW, a);
 }
 
-cudaError_t launch_gemm_tc(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
-                           const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T,
-                           int n_out, int K, int n_batch, int* err) {
-  // 128 x 128 tiles, or 128 x 256 when the narrower tiling would need more CTAs than there are SMs
-  // (a wider tile re-reads the activations half as often per weight byte)
+static cudaError_t launch_gemm_tc_any(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
+                                      const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T,
+                                      int n_out, int K, int n_batch, int* err, void* act, int act_ld, long long act_lo_off,
+                                      int act_split) {
+  // Tile width: one CTA computes 128 positions x BN outputs and, per 64-wide k-block, pulls the activation tile(s)
+  // plus BN weight rows through shared memory; a CTA's ingest rate is what bounds it, so the cost of a choice is
+  // (waves of CTAs over the SMs) x (bytes per k-block), and widths that leave SMs idle or spill into another wave lose.
   int nsm = 148, dev = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&nsm, cudaDevAttrMultiProcessorCount, dev);
-  const long long tiles128 = (long long)((n_out + 127) / 128) * ((T + kBM - 1) / kBM) * n_batch;
-  const int BN = (tiles128 > nsm && n_out >= 256) ? 256 : 128;
+  static const int cand[4] = {256, 160, 128, 96};  // 112 (148 CTAs for a 4096-wide output x 4 shards) measured slower than 128
+  const long long mt = (T + kBM - 1) / kBM;
+  int BN = 128;
+  double best = 1e30;
+  for (int i = 0; i < 4; ++i) {
+    const int bn = cand[i];
+    if (act && bn % 32) continue;                 // the SwiGLU epilogue works on 32-column groups
+    if (bn > 128 && n_out < bn) continue;
+    const long long tiles = (long long)((n_out + bn - 1) / bn) * mt * n_batch;
+    const long long waves = (tiles + nsm - 1) / nsm;
+    const double cost = (double)waves * ((A_lo_bf16 ? 2 : 1) * kBM * kBK * 2 + bn * kBK * 2);
+    if (cost < best - 1e-9) { best = cost; BN = bn; }
+  }
   CUtensorMap tmA, tmAlo, tmW;
   // A: [T][lda] (each batch reads K columns starting at batch * a_col_batch); W: [n_batch * w_row_batch][K]
   if (!make_map(&tmA, A_bf16, (uint64_t)lda, (uint64_t)T, (uint64_t)lda, kBM)) return cudaErrorInvalidValue;
   if (!make_map(&tmAlo, A_lo_bf16 ? A_lo_bf16 : A_bf16, (uint64_t)lda, (uint64_t)T, (uint64_t)lda, kBM)) return cudaErrorInvalidValue;
   const uint64_t w_rows = (uint64_t)(n_batch - 1) * w_row_batch + n_out;
   if (!make_map(&tmW, W_bf16, (uint64_t)K, w_rows, (uint64_t)K, (uint32_t)BN)) return cudaErrorInvalidValue;
-  GemmTcArgs a{Y, y_batch_stride, ldy, T, n_out, K, a_col_batch, w_row_batch, err};
-  if (BN == 256) {
-    if (A_lo_bf16) return launch_tc_t<256, 3, 1>(c, tmA, tmAlo, tmW, a, n_batch);
-    return launch_tc_t<256, 4, 0>(c, tmA, tmAlo, tmW, a, n_batch);
+  GemmTcArgs a{Y, y_batch_stride, ldy, T, n_out, K, a_col_batch, w_row_batch, err, (__nv_bfloat16*)act, act_lo_off, act_ld, act_split};
+#define TPI_TC(BNV) \
+  return A_lo_bf16 ? launch_tc_t<BNV, stages_for(BNV, 1), 1>(c, tmA, tmAlo, tmW, a, n_batch) \
+                   : launch_tc_t<BNV, stages_for(BNV, 0), 0>(c, tmA, tmAlo, tmW, a, n_batch)
+  switch (BN) {
+    case 256: TPI_TC(256);
+    case 160: TPI_TC(160);
+    case 96: TPI_TC(96);
+    default: TPI_TC(128);
   }
-  if (A_lo_bf16) return launch_tc_t<128, 4, 1>(c, tmA, tmAlo, tmW, a, n_batch);
-  return launch_tc_t<128, 6, 0>(c, tmA, tmAlo, tmW, a, n_batch);
+#undef TPI_TC
+}
+
+cudaError_t launch_gemm_tc(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
+                           const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T,
+                           int n_out, int K, int n_batch, int* err) {
+  return launch_gemm_tc_any(c, A_bf16, A_lo_bf16, lda, a_col_batch, W_bf16, w_row_batch, Y, y_batch_stride, ldy, T, n_out, K,
+                            n_batch, err, nullptr, 0, 0, 0);
+}
+
+bool gemm_tc_swiglu_supported(int K, int lda, int s) { return gemm_tc_supported(K, lda, 2 * s) && s % 16 == 0; }
+
+cudaError_t launch_gemm_tc_swiglu(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, const void* Wgu_bf16,
+                                  void* ACT, int out_mode, int T, int s, int K, int* err) {
+  if (out_mode != 1 && out_mode != 2) return cudaErrorInvalidValue;
+  return launch_gemm_tc_any(c, A_bf16, A_lo_bf16, lda, 0, Wgu_bf16, 2 * s, nullptr, 0, 2 * s, T, 2 * s, K, 1, err, ACT, s,
+                            (long long)T * s, out_mode == 2);
 }
 
 }  // namespace tpi

@@ -109,6 +109,11 @@ bool gemm_tc_supported(int K, int a_cols_total, int ldy);
 cudaError_t launch_gemm_tc(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
                            const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T,
                            int n_out, int K, int n_batch, int* err);
+// Gate/up projection with the SwiGLU of launch_swiglu_rows applied in the epilogue (same arithmetic, same bits):
+// Wgu rows interleaved gate_j, up_j; ACT [T][s] bf16 (out_mode 1) or split bf16 (2: lo at + T*s elements).
+bool gemm_tc_swiglu_supported(int K, int lda, int s);
+cudaError_t launch_gemm_tc_swiglu(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, const void* Wgu_bf16,
+                                  void* ACT, int out_mode, int T, int s, int K, int* err);
 // rotate q and k of T positions, append k, v to the cache. QKV rows: [shard][q | k | v] packed as the GEMV.
 cudaError_t launch_rope_kv_rows(const LaunchCtx& c, int dt, const float* QKV, int T, int pos0, int n_shards,
                                 int a, int b, int d, int max_seq, const float2* rope, float* Q,
@@ -127,6 +132,11 @@ cudaError_t launch_swiglu_rows(const LaunchCtx& c, const float* GU, int T, int s
 // X[t] <- sum_i P_i[t] + X[t]; optional tap of the last row
 cudaError_t launch_reduce_residual_rows(const LaunchCtx& c, const float* partials, int n_shards, int T,
                                         int h, float* X, float* tap_last);
+// The same followed by the next block's RMSNorm (gain: that block's norm gain): Xn as launch_rmsnorm_rows writes it.
+// Bit-identical to launch_reduce_residual_rows + launch_rmsnorm_rows.
+cudaError_t launch_reduce_residual_norm_rows(const LaunchCtx& c, const float* partials, int n_shards, int T, int h,
+                                             float* X, float* tap_last, const float* gain, float eps, void* Xn,
+                                             int out_bf16);
 // xhat of one row of X (to hand the last position to the decode-style head)
 // (also sets *pos = pos_value when pos is not null)
 cudaError_t launch_rmsnorm_stat_row(const LaunchCtx& c, const float* xrow, int h, float eps, float* x,

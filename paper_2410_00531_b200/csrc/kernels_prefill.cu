@@ -46,6 +46,95 @@ cudaError_t launch_embed_rows(const LaunchCtx& c, int dt, const void* emb, const
 }
 
 // ------------------------------------------------------------------ RMSNorm rows
+// Row kernels below share one mapping so that their sums agree to the bit: thread tid owns the float4 groups
+// tid, tid + B, ... of the row (B threads), adds the squares of its elements in index order, then block_sum.
+constexpr int ROW_KEEP = 8;  // float4 groups a thread keeps in registers (rows up to 32 * B elements)
+__device__ __forceinline__ float sq4(float4 v, float ss) {
+  ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
+  return ss;
+}
+template <int MODE>
+__device__ __forceinline__ void store_act4(void* base, size_t i, size_t lo_off, float4 v) {
+  if (MODE == 0) *reinterpret_cast<float4*>(reinterpret_cast<float*>(base) + i) = v;
+  else {
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(v.x), h1 = __float2bfloat16_rn(v.y), h2 = __float2bfloat16_rn(v.z),
+                        h3 = __float2bfloat16_rn(v.w);
+    __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(base) + i;
+    *reinterpret_cast<uint2*>(o) = make_uint2((uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16),
+                                              (uint32_t)__bfloat16_as_ushort(h2) | ((uint32_t)__bfloat16_as_ushort(h3) << 16));
+    if (MODE == 2) {
+      const __nv_bfloat16 l0 = __float2bfloat16_rn(v.x - __bfloat162float(h0)), l1 = __float2bfloat16_rn(v.y - __bfloat162float(h1)),
+                          l2 = __float2bfloat16_rn(v.z - __bfloat162float(h2)), l3 = __float2bfloat16_rn(v.w - __bfloat162float(h3));
+      *reinterpret_cast<uint2*>(o + lo_off) =
+          make_uint2((uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16),
+                     (uint32_t)__bfloat16_as_ushort(l2) | ((uint32_t)__bfloat16_as_ushort(l3) << 16));
+    }
+  }
+}
+// threads per row: enough float4 groups per thread to keep many loads in flight, few enough to stay in registers
+static inline int row_threads(int h) { return h / 4 <= 8 * 256 ? 256 : 1024; }
+
+// PARTS: 0 = plain RMSNorm of X; 1 = first X <- ((P_0 + P_1) + ...) + X (star sum in rank order + shortcut), then the norm.
+template <int MODE, int PARTS, int THREADS>
+__global__ void __launch_bounds__(THREADS) norm_rows_kernel(const float* __restrict__ partials, int n_shards, int T, int h,
+                                                        float* X, float* tap_last, const float* __restrict__ gain,
+                                                        float eps, void* Xn, size_t lo_off) {
+  pdl_launch_dependents();
+  pdl_wait();  // inputs come from the previous kernel in the stream
+  __shared__ float red[32];
+  const int B = blockDim.x, ng = h >> 2;
+  const size_t n = (size_t)T * h, row = (size_t)blockIdx.x * h;
+  float4 v[ROW_KEEP];
+#pragma unroll
+  for (int j = 0; j < ROW_KEEP; ++j) {
+    const int g = threadIdx.x + j * B;
+    if (g < ng) v[j] = *reinterpret_cast<const float4*>(X + row + 4 * g);
+  }
+  if (PARTS) {
+    float4 acc[ROW_KEEP];
+    for (int sh = 0; sh < n_shards; ++sh) {
+#pragma unroll
+      for (int j = 0; j < ROW_KEEP; ++j) {
+        const int g = threadIdx.x + j * B;
+        if (g < ng) {
+          const float4 p = *reinterpret_cast<const float4*>(partials + (size_t)sh * n + row + 4 * g);
+          if (sh == 0) acc[j] = p;
+          else { acc[j].x += p.x; acc[j].y += p.y; acc[j].z += p.z; acc[j].w += p.w; }
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < ROW_KEEP; ++j) {
+      const int g = threadIdx.x + j * B;
+      if (g < ng) {
+        v[j].x = acc[j].x + v[j].x; v[j].y = acc[j].y + v[j].y; v[j].z = acc[j].z + v[j].z; v[j].w = acc[j].w + v[j].w;
+        *reinterpret_cast<float4*>(X + row + 4 * g) = v[j];
+        if (tap_last && blockIdx.x == T - 1) *reinterpret_cast<float4*>(tap_last + 4 * g) = v[j];
+      }
+    }
+  }
+  if (!gain) return;  // sum and shortcut only
+  float ss = 0.f;
+#pragma unroll
+  for (int j = 0; j < ROW_KEEP; ++j) {
+    const int g = threadIdx.x + j * B;
+    if (g < ng) ss = sq4(v[j], ss);
+  }
+  ss = block_sum(ss, red);
+  const float r = rsqrtf(ss / (float)h + eps);
+#pragma unroll
+  for (int j = 0; j < ROW_KEEP; ++j) {
+    const int g = threadIdx.x + j * B;
+    if (g < ng) {
+      const float4 gn = *reinterpret_cast<const float4*>(gain + 4 * g);
+      store_act4<MODE>(Xn, row + 4 * g, lo_off,
+                       make_float4(v[j].x * r * gn.x, v[j].y * r * gn.y, v[j].z * r * gn.z, v[j].w * r * gn.w));
+    }
+  }
+}
+static inline bool norm_rows_vec_ok(int h) { return h % 4 == 0 && h / 4 <= ROW_KEEP * 1024; }
+
+// scalar form for widths the vector form does not take
 template <int OUT_BF16>
 __global__ void __launch_bounds__(1024) rmsnorm_rows_kernel(const float* X, const float* gain, int h, float eps,
                                                           void* Xn, size_t lo_off) {
@@ -62,9 +151,22 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows_kernel(const float* X, cons
   }
 }
 
+template <int PARTS>
+static cudaError_t launch_norm_rows_vec(const LaunchCtx& c, const float* partials, int n_shards, int T, int h, float* X,
+                                        float* tap_last, const float* gain, float eps, void* Xn, int mode) {
+  const size_t lo = (size_t)T * h;
+#define TPI_NR(MODE, THREADS) \
+  launch_kernel(c, norm_rows_kernel<MODE, PARTS, THREADS>, dim3(T), dim3(THREADS), 0, partials, n_shards, T, h, X, tap_last, gain, eps, Xn, lo)
+  if (row_threads(h) == 256) return mode == 2 ? TPI_NR(2, 256) : mode == 1 ? TPI_NR(1, 256) : TPI_NR(0, 256);
+  return mode == 2 ? TPI_NR(2, 1024) : mode == 1 ? TPI_NR(1, 1024) : TPI_NR(0, 1024);
+#undef TPI_NR
+}
+
 cudaError_t launch_rmsnorm_rows(const LaunchCtx& c, const float* X, const float* gain, int T, int h,
                                 float eps, void* Xn, int out_bf16) {
   LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
+  if (norm_rows_vec_ok(h))
+    return launch_norm_rows_vec<0>(nc, nullptr, 0, T, h, const_cast<float*>(X), nullptr, gain, eps, Xn, out_bf16);
   const size_t lo = (size_t)T * h;
   if (out_bf16 == 2) return launch_kernel(nc, rmsnorm_rows_kernel<2>, dim3(T), dim3(h >= 4096 ? 1024 : 256), 0, X, gain, h, eps, Xn, lo);
   if (out_bf16) return launch_kernel(nc, rmsnorm_rows_kernel<1>, dim3(T), dim3(h >= 4096 ? 1024 : 256), 0, X, gain, h, eps, Xn, lo);
@@ -352,9 +454,58 @@ __global__ void reduce_residual_rows_kernel(const float* __restrict__ partials, 
 cudaError_t launch_reduce_residual_rows(const LaunchCtx& c, const float* partials, int n_shards, int T,
                                         int h, float* X, float* tap_last) {
   LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
+  if (norm_rows_vec_ok(h)) return launch_norm_rows_vec<1>(nc, partials, n_shards, T, h, X, tap_last, nullptr, 0.f, nullptr, 0);
   const size_t n = (size_t)T * h;
   return launch_kernel(nc, reduce_residual_rows_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0,
                        partials, n_shards, T, h, X, tap_last);
+}
+
+// The same followed by the next block's RMSNorm in one pass over the row (one CTA per position): the element to
+// thread mapping and the order of every sum are those of the two separate kernels, so the results are the same bits.
+template <int MODE>
+__global__ void __launch_bounds__(1024) reduce_residual_norm_rows_kernel(const float* __restrict__ partials, int n_shards,
+                                                                        int T, int h, float* X, float* tap_last,
+                                                                        const float* __restrict__ gain, float eps,
+                                                                        void* Xn, size_t lo_off) {
+  pdl_launch_dependents();
+  pdl_wait();  // inputs come from the previous kernel in the stream
+  __shared__ float red[32];
+  constexpr int KEEP = 8;
+  const size_t n = (size_t)T * h, row = (size_t)blockIdx.x * h;
+  float v[KEEP];
+  float ss = 0.f;
+  int j = 0;
+  for (int k = threadIdx.x; k < h; k += blockDim.x, ++j) {
+    const size_t i = row + k;
+    float s = partials[i];
+    for (int sh = 1; sh < n_shards; ++sh) s += partials[(size_t)sh * n + i];
+    s += X[i];
+    X[i] = s;
+    if (tap_last && blockIdx.x == T - 1) tap_last[k] = s;
+    if (j < KEEP) v[j] = s;
+    ss = fmaf(s, s, ss);
+  }
+  ss = block_sum(ss, red);
+  const float r = rsqrtf(ss / (float)h + eps);
+  j = 0;
+  for (int k = threadIdx.x; k < h; k += blockDim.x, ++j) {
+    const float x = j < KEEP ? v[j] : X[row + k];  // a thread re-reads only what it wrote itself
+    store_act<MODE>(Xn, row + k, lo_off, x * r * gain[k]);
+  }
+}
+
+cudaError_t launch_reduce_residual_norm_rows(const LaunchCtx& c, const float* partials, int n_shards, int T, int h,
+                                             float* X, float* tap_last, const float* gain, float eps, void* Xn,
+                                             int out_bf16) {
+  LaunchCtx nc = c;
+  if (norm_rows_vec_ok(h)) return launch_norm_rows_vec<1>(nc, partials, n_shards, T, h, X, tap_last, gain, eps, Xn, out_bf16);
+  const size_t lo = (size_t)T * h;
+  const dim3 block(h >= 4096 ? 1024 : 256);  // as launch_rmsnorm_rows: the same per-thread sums
+  if (out_bf16 == 2)
+    return launch_kernel(nc, reduce_residual_norm_rows_kernel<2>, dim3(T), block, 0, partials, n_shards, T, h, X, tap_last, gain, eps, Xn, lo);
+  if (out_bf16)
+    return launch_kernel(nc, reduce_residual_norm_rows_kernel<1>, dim3(T), block, 0, partials, n_shards, T, h, X, tap_last, gain, eps, Xn, lo);
+  return launch_kernel(nc, reduce_residual_norm_rows_kernel<0>, dim3(T), block, 0, partials, n_shards, T, h, X, tap_last, gain, eps, Xn, lo);
 }
 
 // ------------------------------------------------------------------ misc

@@ -119,6 +119,20 @@ extern "C" int tpi_op_gemm_bf16(const void* A, const void* A_lo, int lda, int a_
   return e == cudaErrorInvalidValue ? TPI_ERR_SHAPE : cu(e);
 }
 
+extern "C" int tpi_op_gemm_bf16_swiglu(const void* A, const void* A_lo, int lda, const void* Wgu, void* ACT, int split_out, int T,
+                                       int s, int K, int32_t* err_word, void* stream) {
+  if (!A || !Wgu || !ACT || !err_word || T < 1 || s < 1 || K < 1) return TPI_ERR_INVALID_ARG;
+  if (!gemm_tc_swiglu_supported(K, lda, s)) return TPI_ERR_SHAPE;
+  const cudaError_t e = launch_gemm_tc_swiglu(ctx(stream), A, A_lo, lda, Wgu, ACT, split_out ? 2 : 1, T, s, K, err_word);
+  return e == cudaErrorInvalidValue ? TPI_ERR_SHAPE : cu(e);
+}
+
+extern "C" int tpi_op_reduce_residual_norm_rows(const float* partials, int n_shards, int T, int h, float* X, const float* gain,
+                                                float rms_eps, float* Xn, void* stream) {
+  if (!partials || !X || !gain || !Xn || n_shards < 1 || T < 1 || h < 1) return TPI_ERR_INVALID_ARG;
+  return cu(launch_reduce_residual_norm_rows(ctx(stream), partials, n_shards, T, h, X, nullptr, gain, rms_eps, Xn, 0));
+}
+
 extern "C" int tpi_op_prefill_attention(int dtype, const float* Q, const void* kcache, const void* vcache, int T,
                                         int pos0, int a, int b, int d, int max_seq, float* O, void* stream) {
   if (bad_dtype(dtype) || !Q || !kcache || !vcache || !O || T < 1 || pos0 < 0) return TPI_ERR_INVALID_ARG;

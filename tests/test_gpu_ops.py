@@ -311,3 +311,60 @@ def test_gemm_tensor_core_bf16(T, Tn, K, n_out, nb, split):
     # products of bf16 pairs are exact in fp32; what is left is the tensor core's fp32 accumulation
     # over K / 16 (split: K / 8) partial sums, observed <= 1e-5
     assert rel_l2(got, want) < 2e-5
+
+
+@pytest.mark.parametrize("Tn,K,s", [(128, 4096, 11008), (70, 1024, 1360), (300, 512, 48)])
+@pytest.mark.parametrize("split_out", [False, True])
+def test_gemm_tensor_core_swiglu_epilogue(T, Tn, K, s, split_out):
+    """Eq. 2's gate/up projection for T positions with SwiGLU applied in the GEMM's epilogue (gate_j, up_j rows
+    interleaved): against the oracle's silu on the fp64 product of the same bf16 values."""
+    import paper_2410_00531_b200.ops as KK
+    rng = np.random.default_rng(Tn + K + s)
+    A32 = rng.standard_normal((Tn, K)).astype(np.float32)
+    A = S.f32_to_bf16_bits(A32).reshape(Tn, K)
+    Alo = S.f32_to_bf16_bits(A32 - S.bf16_bits_to_f32(A).reshape(A32.shape)).reshape(Tn, K)
+    W = S.f32_to_bf16_bits((rng.standard_normal((2 * s, K)) * 0.05).astype(np.float32)).reshape(2 * s, K)
+    ACT = T.full((2, Tn, s), -1, dtype=T.int16, device="cuda")       # hi plane, lo plane (bf16 bits)
+    err = T.zeros(1, dtype=T.int32, device="cuda")
+    KK.gemm_bf16_swiglu(dev(T, A).data_ptr(), K, dev(T, W).data_ptr(), ACT.data_ptr(), split_out, Tn, s, K,
+                        err.data_ptr(), A_lo=dev(T, Alo).data_ptr())
+    T.cuda.synchronize()
+    assert int(err[0]) == 0
+    y = (S.as_f64(A) + S.as_f64(Alo)) @ S.as_f64(W).T
+    want = O.silu(y[:, 0::2]) * y[:, 1::2]
+    planes = ACT.cpu().numpy().view(np.uint16)
+    hi = S.as_f64(planes[0])
+    if split_out:
+        got = hi + S.as_f64(planes[1])
+        assert rel_l2(got, want) < 2e-5                              # hi + lo keeps ~16 bits of the fp32 value
+    else:
+        assert (planes[1] == 0xFFFF).all()                           # the second plane is not touched
+        got = hi
+        assert rel_l2(got, want) < 3e-3                              # one bf16 rounding of each output
+    # element by element: the high plane is the fp32 result rounded to bf16 (half an ulp, 2^-9 relative), on top of
+    # the fp32 accumulation error of the two dot products, which scales with the size of y, not of the output
+    bound = np.abs(want) * 2.0 ** -8 + 2e-5 * np.abs(y).max() * (1 + np.abs(y[:, 1::2]))
+    assert (np.abs(hi - want) <= bound).all()
+
+
+@pytest.mark.parametrize("Tn,h,N", [(128, 4096, 4), (37, 8192, 8), (5, 256, 2), (200, 1000, 3)])
+def test_reduce_residual_norm_rows(T, Tn, h, N):
+    """Star sum in rank order + shortcut for T positions, then the next block's RMSNorm (Eq. 1-2 and the norm
+    of Step 3), against the oracle; the residual stream itself must equal the stand-alone sum kernel's bits."""
+    import paper_2410_00531_b200.ops as KK
+    rng = np.random.default_rng(Tn * h + N)
+    P = rng.standard_normal((N, Tn, h)).astype(np.float32)
+    X0 = rng.standard_normal((Tn, h)).astype(np.float32)
+    g = (1 + 0.1 * rng.standard_normal(h)).astype(np.float32)
+    eps = 1e-5
+    X = dev(T, X0.copy())
+    Xn = T.full((Tn, h), float("nan"), dtype=T.float32, device="cuda")
+    KK.reduce_residual_norm_rows(dev(T, P).data_ptr(), N, Tn, h, X.data_ptr(), dev(T, g).data_ptr(), eps, Xn.data_ptr())
+    T.cuda.synchronize()
+    want_x = P.astype(np.float64).sum(0) + X0
+    assert rel_l2(X.cpu().numpy(), want_x) < 1e-6
+    acc = P[0].copy()
+    for i in range(1, N):
+        acc = acc + P[i]                                             # fp32, rank order, shortcut last
+    assert np.array_equal(X.cpu().numpy(), acc + X0)
+    assert rel_l2(Xn.cpu().numpy(), O.rmsnorm(want_x, g.astype(np.float64), eps)) < 2e-6
