@@ -117,6 +117,17 @@ int tpi_set_shards(tpi_model *m, int n_shards);
  * Needs host images unless going 0 -> 0. */
 int tpi_set_window(tpi_model *m, int window_blocks);
 
+/* Heterogeneous partition (Sec. 3.1: device i takes the proportion p_i of the attention heads and of the
+ * FFN columns, stronger devices more): shard i owns kv_heads_per_shard[i] kv heads together with their
+ * query-head groups and ffn_cols_per_shard[i] FFN columns, in rank order.  Both lists have n_shards
+ * entries (1 <= n_shards <= 16), every entry >= 1, sums equal to n_kv_heads and ffn, and a shard's
+ * heads*head_dim and FFN columns must be multiples of 16 bytes of weights (TPI_ERR_SHAPE otherwise).
+ * Re-packs the layer blocks like tpi_set_shards (which returns to the uniform p_i = 1/N) and resets the
+ * position.  The partition decides which inputs each per-shard partial sum of the O and down
+ * projections covers; the column-sharded projections give the same values whoever computes them. */
+int tpi_set_partition(tpi_model *m, int n_shards, const int32_t *kv_heads_per_shard,
+                      const int32_t *ffn_cols_per_shard);
+
 /* Block retention (Sec. 3.3, Prop. 6 / Appendix A.6): when the link is the bottleneck, keep ONE FFN
  * block in every `ffn_every_T` FFN blocks resident (layers 0, T, 2T, ...) beside the window and stream
  * only the rest; 0 turns retention off, 1 keeps every FFN block.  Only for a streamed model

@@ -182,18 +182,31 @@ class LlamaOracle:
         return h_attn, h_ffn, K, V
 
     # -- the same layer as N devices compute it (Eq. 1-2): per-device partials, rank-ordered sum
-    def layer_sharded(self, l: int, x: np.ndarray, pos: np.ndarray, Kprev, Vprev, n_shards: int):
+    def layer_sharded(self, l: int, x: np.ndarray, pos: np.ndarray, Kprev, Vprev, n_shards: int, partition=None):
+        """Eq. 1-2 as N devices compute them.  ``partition`` = (kv heads per device, FFN columns per device)
+        gives device i the proportion p_i of the heads and of the FFN columns (Sec. 3.1: stronger devices take
+        more); None is the uniform p_i = 1/N.  A device's query heads are those of its kv heads' groups."""
         c = self.cfg
         a, b, d, s = c.n_heads, c.n_kv_heads, c.head_dim, c.ffn
-        if a % n_shards or b % n_shards or s % n_shards:
-            raise ValueError("N must divide heads, kv heads and FFN width")
+        if partition is None:
+            if a % n_shards or b % n_shards or s % n_shards:
+                raise ValueError("N must divide heads, kv heads and FFN width")
+            kv_cnt, ffn_cnt = [b // n_shards] * n_shards, [s // n_shards] * n_shards
+        else:
+            kv_cnt, ffn_cnt = [int(v) for v in partition[0]], [int(v) for v in partition[1]]
+            if len(kv_cnt) != n_shards or len(ffn_cnt) != n_shards or sum(kv_cnt) != b or sum(ffn_cnt) != s \
+                    or min(kv_cnt) < 1 or min(ffn_cnt) < 1:
+                raise ValueError("a partition gives every device at least one kv head and one FFN column, all of them once")
+        kv0 = np.concatenate([[0], np.cumsum(kv_cnt)])
+        f0 = np.concatenate([[0], np.cumsum(ffn_cnt)])
+        grp = a // b
         T = x.shape[0]
         xn = rmsnorm(x, self.w(l, ATTN_NORM), c.rms_eps)     # replicated norm on every device
         Wo = self.w(l, WO)
         partials, Ks, Vs = [], [], []
         for i in range(n_shards):
-            heads = np.arange(i * a // n_shards, (i + 1) * a // n_shards)
-            kvh = np.arange(i * b // n_shards, (i + 1) * b // n_shards)
+            heads = np.arange(kv0[i] * grp, kv0[i + 1] * grp)
+            kvh = np.arange(kv0[i], kv0[i + 1])
             q, k, v = self._qkv(l, xn, pos, heads, kvh)
             Ki = np.swapaxes(k, 0, 1) if Kprev is None else np.concatenate([Kprev[kvh], np.swapaxes(k, 0, 1)], axis=1)
             Vi = np.swapaxes(v, 0, 1) if Vprev is None else np.concatenate([Vprev[kvh], np.swapaxes(v, 0, 1)], axis=1)
@@ -210,7 +223,7 @@ class LlamaOracle:
         Wg, Wu, Wd = self.w(l, WGATE), self.w(l, WUP), self.w(l, WDOWN)
         partials = []
         for i in range(n_shards):
-            cols = np.arange(i * s // n_shards, (i + 1) * s // n_shards)
+            cols = np.arange(f0[i], f0[i + 1])
             act_i = silu(xn2 @ Wg[cols].T) * (xn2 @ Wu[cols].T)
             partials.append(act_i @ Wd[:, cols].T)
         red = partials[0]
@@ -220,7 +233,7 @@ class LlamaOracle:
         return h_attn, h_ffn, np.concatenate(Ks, axis=0), np.concatenate(Vs, axis=0)
 
     # -- Algorithm 1's loop body for T new positions
-    def forward(self, tokens, n_shards: int | None = None, all_logits: bool = False) -> np.ndarray:
+    def forward(self, tokens, n_shards: int | None = None, all_logits: bool = False, partition=None) -> np.ndarray:
         """Feed ``tokens`` at positions cache.length .. cache.length+T-1.
 
         Returns logits of the last position [v] (or of every position [T, v])."""
@@ -237,7 +250,7 @@ class LlamaOracle:
             if n_shards is None:
                 h_attn, h_ffn, K, V = self.layer_unsharded(l, x, pos, Kp, Vp)
             else:
-                h_attn, h_ffn, K, V = self.layer_sharded(l, x, pos, Kp, Vp, n_shards)
+                h_attn, h_ffn, K, V = self.layer_sharded(l, x, pos, Kp, Vp, n_shards, partition)
             if first:
                 self.cache.K.append(K)
                 self.cache.V.append(V)

@@ -85,6 +85,7 @@ SYMBOLS = {
     "tpi_ring_trace": (C.c_int, [C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.c_int]),
     "tpi_ring_trace_retained": (C.c_int, [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.c_int]),
     "tpi_set_retention": (C.c_int, [C.c_void_p, C.c_int]),
+    "tpi_set_partition": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
     "tpi_scheduler_report": (C.c_int, [C.c_void_p, C.c_void_p]),
     "tpi_scheduler_reset": (C.c_int, [C.c_void_p]),
     "tpi_steady_conditions": (C.c_int, [C.c_double] * 5 + [C.c_int] + [C.POINTER(C.c_int)] * 3),
@@ -238,6 +239,15 @@ def steady_conditions(t_attn, t_ffn, t_all_reduce, tau_attn, tau_ffn, n_layers: 
     _check(lib().tpi_steady_conditions(t_attn, t_ffn, t_all_reduce, tau_attn, tau_ffn, n_layers,
                                        C.byref(a), C.byref(b), C.byref(c)))
     return bool(a.value), bool(b.value), c.value
+
+
+def set_partition(h, kv_heads_per_shard, ffn_cols_per_shard) -> None:
+    kv = np.ascontiguousarray(kv_heads_per_shard, dtype=np.int32)
+    ff = np.ascontiguousarray(ffn_cols_per_shard, dtype=np.int32)
+    if kv.shape != ff.shape or kv.ndim != 1:
+        raise ValueError("one entry per shard in both lists")
+    _check(lib().tpi_set_partition(h, int(kv.size), kv.ctypes.data_as(C.POINTER(C.c_int32)),
+                                   ff.ctypes.data_as(C.POINTER(C.c_int32))))
 
 
 def set_retention(h, ffn_every_T: int) -> None:

@@ -80,6 +80,12 @@ struct tpi_model {
   int position = 0;
   // window ring
   Ring ring;
+  // partition of the kv heads (with their query-head groups) and of the FFN columns over the shards: prefix sums,
+  // N + 1 entries each.  unequal = false: the uniform p_i = 1/N.  With unequal proportions the QKV rows are packed
+  // in the unsharded order (their results do not depend on who computes them) and the row-sharded O / down
+  // matrices follow the partition, which is where it decides the grouping of the partial sums.
+  std::vector<int> kv0, f0;
+  bool unequal = false;
   int retain_T = 0;                  // keep the FFN block of every T-th layer resident beside the window (0: none)
   std::vector<char> retained;        // per block
   std::vector<size_t> retained_off;  // byte offset of a retained block after the window slots
@@ -114,6 +120,14 @@ struct tpi_model {
 template <typename T>
 static T* dptr(tpi_model* m, size_t off) { return reinterpret_cast<T*>(m->dev + off); }
 
+static void uniform_partition(tpi_model* m) {
+  const int N = m->N;
+  m->kv0.assign(N + 1, 0);
+  m->f0.assign(N + 1, 0);
+  for (int i = 0; i <= N; ++i) { m->kv0[i] = m->cfg.n_kv_heads / N * i; m->f0[i] = m->cfg.ffn / N * i; }
+  m->unequal = false;
+}
+
 static int validate(const tpi_config* c, int N) {
   if (!c) return fail(TPI_ERR_INVALID_ARG, "null config");
   if (c->n_layers < 1 || c->hidden < 1 || c->n_heads < 1 || c->n_kv_heads < 1 || c->head_dim < 1 ||
@@ -124,7 +138,10 @@ static int validate(const tpi_config* c, int N) {
   const int vec = c->dtype == TPI_BF16 ? 8 : 4;
   if (c->n_heads % c->n_kv_heads) return fail(TPI_ERR_SHAPE, "kv heads must divide heads");
   const int grp = c->n_heads / c->n_kv_heads;
-  if (grp != 1 && grp != 2 && grp != 4 && grp != 8) return fail(TPI_ERR_SHAPE, "heads per kv head must be 1, 2, 4 or 8");
+  // the tensor-core attention kernels (bf16 cache, head_dim 64 or 128) take any group of up to 8 query heads
+  const bool any_grp = c->dtype == TPI_BF16 && (c->head_dim == 64 || c->head_dim == 128) && grp <= 8;
+  if (!any_grp && grp != 1 && grp != 2 && grp != 4 && grp != 8)
+    return fail(TPI_ERR_SHAPE, "heads per kv head must be 1, 2, 4 or 8 (any count up to 8 for bf16 with head_dim 64 or 128)");
   if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128) return fail(TPI_ERR_SHAPE, "head_dim must be 32, 64 or 128");
   if (c->n_heads % N || c->n_kv_heads % N || c->ffn % N)
     return fail(TPI_ERR_SHAPE, "n_shards=%d must divide heads (%d), kv heads (%d) and ffn (%d)", N, c->n_heads,
@@ -188,11 +205,13 @@ static void f32_from_storage(const void* src, int dtype, float* dst, size_t n) {
 }
 
 // Copies rows [row0, row0+n) of tensor `tid` from `src` into the layer's attention or FFN image.
-static void place_rows(const tpi_config& c, const BlockLayout& bl, int N, int tid, int64_t row0, int64_t n,
-                       const char* src, char* attn_img, char* ffn_img) {
+static void place_rows(const tpi_config& c, const BlockLayout& bl, int N, const int* kv0, const int* f0, bool unequal,
+                       int tid, int64_t row0, int64_t n, const char* src, char* attn_img, char* ffn_img) {
   const size_t B = elem_size(c.dtype), h = c.hidden, d = c.head_dim;
-  const int64_t hps_rows = (int64_t)c.n_heads / N * d, kps_rows = (int64_t)c.n_kv_heads / N * d;
-  const int64_t qkv_rows = hps_rows + 2 * kps_rows, spn = c.ffn / N;
+  const int Nq = unequal ? 1 : N;  // column-sharded rows of an unequal partition are packed as one shard
+  const int64_t hps_rows = (int64_t)c.n_heads / Nq * d, kps_rows = (int64_t)c.n_kv_heads / Nq * d;
+  const int64_t qkv_rows = hps_rows + 2 * kps_rows, spn = c.ffn / Nq;
+  const int grp = c.n_heads / c.n_kv_heads;
 #pragma omp parallel for schedule(static)
   for (int64_t i = 0; i < n; ++i) {
     const int64_t r = row0 + i;
@@ -216,15 +235,19 @@ static void place_rows(const tpi_config& c, const BlockLayout& bl, int N, int ti
         memcpy(ffn_img + bl.off_gu + (size_t)(sh * 2 * spn + 2 * j + (tid == TPI_T_WUP)) * h * B,
                src + (size_t)i * h * B, h * B);
       } break;
-      case TPI_T_WO: {
-        const size_t K = (size_t)c.n_heads * d, Ks = K / N;
-        for (int sh = 0; sh < N; ++sh)
-          memcpy(attn_img + bl.off_wo + ((size_t)sh * h + r) * Ks * B, src + ((size_t)i * K + sh * Ks) * B, Ks * B);
+      case TPI_T_WO: {  // shard sh: [h][its heads' columns], shards one after another
+        const size_t K = (size_t)c.n_heads * d;
+        for (int sh = 0; sh < N; ++sh) {
+          const size_t k_lo = (size_t)kv0[sh] * grp * d, Ks = (size_t)(kv0[sh + 1] - kv0[sh]) * grp * d;
+          memcpy(attn_img + bl.off_wo + (h * k_lo + (size_t)r * Ks) * B, src + ((size_t)i * K + k_lo) * B, Ks * B);
+        }
       } break;
       case TPI_T_WDOWN: {
-        const size_t K = c.ffn, Ks = K / N;
-        for (int sh = 0; sh < N; ++sh)
-          memcpy(ffn_img + bl.off_down + ((size_t)sh * h + r) * Ks * B, src + ((size_t)i * K + sh * Ks) * B, Ks * B);
+        const size_t K = c.ffn;
+        for (int sh = 0; sh < N; ++sh) {
+          const size_t k_lo = (size_t)f0[sh], Ks = (size_t)(f0[sh + 1] - f0[sh]);
+          memcpy(ffn_img + bl.off_down + (h * k_lo + (size_t)r * Ks) * B, src + ((size_t)i * K + k_lo) * B, Ks * B);
+        }
       } break;
       default: break;
     }
@@ -299,7 +322,7 @@ static int build_layer_images(tpi_model* m, int layer, char* attn_img, char* ffn
         return fail(TPI_ERR_CALLBACK, "fill(tensor %d, layer %d) failed", tid, layer);
       if (tid == TPI_T_ATTN_NORM) f32_from_storage(stage, c.dtype, (float*)attn_img, c.hidden);
       else if (tid == TPI_T_FFN_NORM) f32_from_storage(stage, c.dtype, (float*)ffn_img, c.hidden);
-      else place_rows(c, m->plan.bl, m->N, tid, r0, n, stage, attn_img, ffn_img);
+      else place_rows(c, m->plan.bl, m->N, m->kv0.data(), m->f0.data(), m->unequal, tid, r0, n, stage, attn_img, ffn_img);
     }
   }
   return TPI_OK;
@@ -338,7 +361,7 @@ static int load_layers(tpi_model* m) {
             if (m->fill(m->user, tid, l, r0, n, stage))
               return fail(TPI_ERR_CALLBACK, "fill(tensor %d, layer %d) failed", tid, l);
             if (tid == TPI_T_ATTN_NORM || tid == TPI_T_FFN_NORM) f32_from_storage(stage, cc.dtype, (float*)ai, cc.hidden);
-            else place_rows(cc, bl, m->N, tid, r0, n, stage, ai, ai);
+            else place_rows(cc, bl, m->N, m->kv0.data(), m->f0.data(), m->unequal, tid, r0, n, stage, ai, ai);
           }
         }
         CK(cudaMemcpyAsync(resident_block(m, 2 * l + pass), ai, pass ? bl.ffn_bytes : bl.attn_bytes,
@@ -453,7 +476,7 @@ static int ensure_mega(tpi_model* m) {
 
 static bool mega_usable(const tpi_model* m) {
   const tpi_config& c = m->cfg;
-  return m->opt_mega && m->window <= 0 && !m->opt_profile &&
+  return m->opt_mega && m->window <= 0 && !m->opt_profile && !m->unequal &&
          mega_supported(c.dtype, c.hidden, c.n_heads, c.n_kv_heads, c.head_dim, c.ffn) &&
          mega_layer_table_bytes(c.n_layers) <= m->plan.h_stage_bytes &&
          mega_smem_bytes(c.dtype, c.hidden, c.n_heads, c.n_kv_heads, c.head_dim, c.ffn, m->plan.nsplit) <= 200 * 1024;
@@ -620,6 +643,7 @@ extern "C" int tpi_load_model(const tpi_config* cfg, const tpi_resources* res, t
   m->fill = fill;
   m->user = user;
   m->N = n_shards;
+  uniform_partition(m);
   m->window = window_blocks;
   m->dev = (char*)res->dev_arena;
   m->host = (char*)res->host_arena;
@@ -700,6 +724,36 @@ extern "C" int tpi_set_shards(tpi_model* m, int n_shards) {
   TRY(quiesce(m));
   drop_graph(m);
   m->N = n_shards;
+  uniform_partition(m);
+  TRY(load_layers(m));
+  TRY(start_window(m));
+  return write_position(m, 0);
+}
+
+extern "C" int tpi_set_partition(tpi_model* m, int n_shards, const int32_t* kv_heads_per_shard,
+                                 const int32_t* ffn_cols_per_shard) {
+  if (!m || !kv_heads_per_shard || !ffn_cols_per_shard) return fail(TPI_ERR_INVALID_ARG, "null argument");
+  const tpi_config& c = m->cfg;
+  if (n_shards < 1 || n_shards > ROWSHARD_MAX_UNEQUAL || n_shards > m->plan.n_shards_max)
+    return fail(TPI_ERR_INVALID_ARG, "n_shards must be in [1, %d]", ROWSHARD_MAX_UNEQUAL < m->plan.n_shards_max ? ROWSHARD_MAX_UNEQUAL : m->plan.n_shards_max);
+  const int vec = c.dtype == TPI_BF16 ? 8 : 4, grp = c.n_heads / c.n_kv_heads;
+  long long kv = 0, ff = 0;
+  for (int i = 0; i < n_shards; ++i) {
+    if (kv_heads_per_shard[i] < 1 || ffn_cols_per_shard[i] < 1) return fail(TPI_ERR_SHAPE, "every shard needs at least one kv head and one FFN column");
+    if (ffn_cols_per_shard[i] % vec || (kv_heads_per_shard[i] * grp * c.head_dim) % vec)
+      return fail(TPI_ERR_SHAPE, "a shard's FFN columns and heads*d must be multiples of %d elements (16 bytes)", vec);
+    kv += kv_heads_per_shard[i];
+    ff += ffn_cols_per_shard[i];
+  }
+  if (kv != c.n_kv_heads || ff != c.ffn) return fail(TPI_ERR_SHAPE, "the shards' kv heads (%lld of %d) and FFN columns (%lld of %d) must add up", kv, c.n_kv_heads, ff, c.ffn);
+  if (!rowshard_fused_supported(c.ffn, 1)) return fail(TPI_ERR_SHAPE, "ffn too wide for an unequal partition");
+  TRY(quiesce(m));
+  drop_graph(m);
+  m->N = n_shards;
+  m->kv0.assign(n_shards + 1, 0);
+  m->f0.assign(n_shards + 1, 0);
+  for (int i = 0; i < n_shards; ++i) { m->kv0[i + 1] = m->kv0[i] + kv_heads_per_shard[i]; m->f0[i + 1] = m->f0[i] + ffn_cols_per_shard[i]; }
+  m->unequal = true;
   TRY(load_layers(m));
   TRY(start_window(m));
   return write_position(m, 0);
@@ -827,15 +881,21 @@ static int enqueue_decode(tpi_model* m, LaunchCtx& lc) {
   int* tok_hist = dptr<int>(m, p.tok_hist);
   const float2* rope = dptr<float2>(m, p.rope);
   unsigned* tickets = dptr<unsigned>(m, p.tickets);
-  const size_t qkv_shard = (size_t)(a + 2 * b) / N * d * h;
+  const int Nc = m->unequal ? 1 : N;  // the column-sharded projections of an unequal partition run as one shard
+  const size_t qkv_shard = (size_t)(a + 2 * b) / Nc * d * h;
+  // unequal partition: input ranges of the row-sharded projections (O: a shard's heads x d; down: its FFN columns)
+  std::vector<int> ko(N + 1), kd(N + 1);
+  for (int i = 0; i <= N; ++i) { ko[i] = m->kv0[i] * (a / b) * d; kd[i] = m->f0[i]; }
 
   // The kernel that ends a block leaves the raw residual x plus partial sums of x^2; the GEMV that
   // starts the next block normalises and applies its own block's gain while staging x.
   float* ss_part = dptr<float>(m, p.ss_part);
   const int n_parts = rowshard_fused_parts(h);
   auto norm_in = [&](const float* gain) { return NormIn{x, gain, ss_part, n_parts, c.rms_eps}; };
-  auto rowshard = [&](const void* W, const float* xin, int Ks, float* tap) -> int {
-    if (rowshard_fused_supported(Ks, N)) {
+  auto rowshard = [&](const void* W, const float* xin, int Ks, const int* k0, float* tap) -> int {
+    if (m->unequal) {
+      CK(launch_gemv_rowshard_fused_unequal(lc, dt, W, xin, h, k0, N, x, ss_part, tap));
+    } else if (rowshard_fused_supported(Ks, N)) {
       CK(launch_gemv_rowshard_fused(lc, dt, W, (size_t)h * Ks, xin, h, Ks, N, x, ss_part, tap));
     } else {  // very long shard slices: partial sums through memory, then the sum kernel
       CK(launch_gemv_partials(lc, dt, W, (size_t)h * Ks, xin, h, Ks, N, partials));
@@ -851,11 +911,11 @@ static int enqueue_decode(tpi_model* m, LaunchCtx& lc) {
     TRY(acquire_block(m, 2 * l, &br));
     void* kc = m->dev + p.kcache + (size_t)l * p.kv_layer_bytes;
     void* vc = m->dev + p.vcache + (size_t)l * p.kv_layer_bytes;
-    CK(launch_gemv_qkv(lc, dt, br.base + bl.off_qkv, qkv_shard, norm_in((const float*)br.base), h, N, a, b, d,
+    CK(launch_gemv_qkv(lc, dt, br.base + bl.off_qkv, qkv_shard, norm_in((const float*)br.base), h, Nc, a, b, d,
                        c.max_seq, pos, rope, q, kc, vc));
     CK(launch_decode_attention(lc, dt, q, kc, vc, pos, a, b, d, c.max_seq, p.nsplit,
                                dptr<float>(m, p.attn_scratch), tickets, o));
-    TRY(rowshard(br.base + bl.off_wo, o, a * d / N, dptr<float>(m, p.taps) + (size_t)(2 * l) * h));
+    TRY(rowshard(br.base + bl.off_wo, o, a * d / N, ko.data(), dptr<float>(m, p.taps) + (size_t)(2 * l) * h));
     TRY(release_block(m, 2 * l));
     // ---- FFN block: norm gain | gate/up (column-sharded) | down (row-sharded)
     TRY(acquire_block(m, 2 * l + 1, &br));
@@ -865,9 +925,9 @@ static int enqueue_decode(tpi_model* m, LaunchCtx& lc) {
       e1 = m->prof_ev[m->prof_used++];
       CK(cudaEventRecord(e0, lc.stream));
     }
-    CK(launch_gemv_gateup(lc, dt, br.base + bl.off_gu, (size_t)2 * (s / N) * h, norm_in((const float*)br.base), h, N, s, act));
+    CK(launch_gemv_gateup(lc, dt, br.base + bl.off_gu, (size_t)2 * (s / Nc) * h, norm_in((const float*)br.base), h, Nc, s, act));
     if (e1) CK(cudaEventRecord(e1, lc.stream));
-    TRY(rowshard(br.base + bl.off_down, act, s / N, dptr<float>(m, p.taps) + (size_t)(2 * l + 1) * h));
+    TRY(rowshard(br.base + bl.off_down, act, s / N, kd.data(), dptr<float>(m, p.taps) + (size_t)(2 * l + 1) * h));
     TRY(release_block(m, 2 * l + 1));
   }
   CK(launch_head_argmax(lc, dt, m->dev + p.head, norm_in(dptr<float>(m, p.final_gain)), h, c.vocab,
@@ -989,10 +1049,16 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
   const float2* rope = dptr<float2>(m, p.rope);
   const int qkv_cols = (a + 2 * b) * d;
   const int Ko = a * d / N, Kd = s / N;
+  const int Nc = m->unequal ? 1 : N;  // column-sharded rows of an unequal partition are packed as one shard
+  std::vector<int> ko(N + 1), kd(N + 1);  // input ranges of the row-sharded projections per shard
+  for (int i = 0; i <= N; ++i) { ko[i] = m->kv0[i] * (a / b) * d; kd[i] = m->f0[i]; }
+  bool k64 = true;  // the tensor-core GEMM takes contractions that are multiples of 64
+  for (int i = 0; i < N; ++i) k64 = k64 && (ko[i + 1] - ko[i]) % 64 == 0 && (kd[i + 1] - kd[i]) % 64 == 0;
   // bf16 models run the projections on the tensor cores (activations rounded to bf16, fp32 accumulate);
   // fp32 models, and shapes the tensor-core kernel does not take, use the fp32 SIMT GEMM.
-  const bool tc = m->opt_tensor && dt == TPI_BF16 && gemm_tc_supported(h, h, qkv_cols) && gemm_tc_supported(Ko, a * d, h) &&
-                  gemm_tc_supported(h, h, 2 * s) && gemm_tc_supported(Kd, s, h);
+  const bool tc = m->opt_tensor && dt == TPI_BF16 && gemm_tc_supported(h, h, qkv_cols) && gemm_tc_supported(h, h, 2 * s) &&
+                  (m->unequal ? k64 && gemm_tc_supported(64, a * d, h) && gemm_tc_supported(64, s, h)
+                              : gemm_tc_supported(Ko, a * d, h) && gemm_tc_supported(Kd, s, h));
   const int act_mode = tc ? (m->opt_tensor == 2 ? 1 : 2) : 0;  // 0 fp32, 1 bf16, 2 split bf16 (default)
   int* err = dptr<int>(m, p.err);
   // Y[b] = A[:, b*a_col : b*a_col+K] . W[b]^T for n_batch shards (1 for the column-sharded projections)
@@ -1004,6 +1070,25 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
                         n_out, K, n_batch, err));
     }
     else CK(launch_gemm_simt(lc, dt, A, a_col, lda, W, (long long)w_rows_b * K, Y, y_bs, ldy, T, n_out, K, n_batch));
+    return TPI_OK;
+  };
+  // row-sharded projection: shard i multiplies its slice of the inputs by its own matrix -> partial sums P_i
+  auto proj_rows = [&](const float* A, int lda, const void* W, const int* k0, int Ks) -> int {
+    if (!m->unequal) return proj(A, lda, Ks, W, h, PART, (long long)T * h, h, h, Ks, N);
+    const size_t B = elem_size(dt);
+    for (int i = 0; i < N; ++i) {
+      const int kw = k0[i + 1] - k0[i];
+      const char* Wi = (const char*)W + (size_t)h * k0[i] * B;
+      // split-bf16 activations: the column offset applies to both halves, which are T * lda elements apart
+      const float* Ai = tc ? reinterpret_cast<const float*>(reinterpret_cast<const __nv_bfloat16*>(A) + k0[i]) : A + k0[i];
+      if (tc) {
+        const __nv_bfloat16* hi = reinterpret_cast<const __nv_bfloat16*>(Ai);
+        CK(launch_gemm_tc(lc, hi, act_mode == 2 ? hi + (size_t)T * lda : nullptr, lda, 0, Wi, h, PART + (size_t)i * T * h, 0, h, T,
+                          h, kw, 1, err));
+      } else {
+        CK(launch_gemm_simt(lc, dt, Ai, 0, lda, Wi, 0, PART + (size_t)i * T * h, 0, h, T, h, kw, 1));
+      }
+    }
     return TPI_OK;
   };
   CK(launch_embed_rows(lc, dt, m->dev + p.emb, dptr<int>(m, p.tok_hist), pos0, T, c.vocab, h, X, err));
@@ -1018,12 +1103,12 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
     void* vc = m->dev + p.vcache + (size_t)l * p.kv_layer_bytes;
     if (!normed) CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, act_mode));
     TRY(proj(Xn, h, 0, br.base + bl.off_qkv, qkv_cols, QKV, 0, qkv_cols, qkv_cols, h, 1));
-    CK(launch_rope_kv_rows(lc, dt, QKV, T, pos0, N, a, b, d, c.max_seq, rope, Q, kc, vc));
+    CK(launch_rope_kv_rows(lc, dt, QKV, T, pos0, Nc, a, b, d, c.max_seq, rope, Q, kc, vc));
     if (m->opt_tensor && prefill_attention_mma_supported(dt, d))
       CK(launch_prefill_attention_mma(lc, Q, kc, vc, T, pos0, a, b, d, c.max_seq, O, act_mode));
     else
       CK(launch_prefill_attention(lc, dt, Q, kc, vc, T, pos0, a, b, d, c.max_seq, O, act_mode));
-    TRY(proj(O, a * d, Ko, br.base + bl.off_wo, h, PART, (long long)T * h, h, h, Ko, N));
+    TRY(proj_rows(O, a * d, br.base + bl.off_wo, ko.data(), Ko));
     float* tap_a = last ? dptr<float>(m, p.taps) + (size_t)(2 * l) * h : nullptr;
     if (fuse_norm)
       CK(launch_reduce_residual_norm_rows(lc, PART, N, T, h, X, tap_a, (const float*)resident_block(m, 2 * l + 1), c.rms_eps, Xn, act_mode));
@@ -1039,7 +1124,7 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
       TRY(proj(Xn, h, 0, br.base + bl.off_gu, 2 * s, GU, 0, 2 * s, 2 * s, h, 1));
       CK(launch_swiglu_rows(lc, GU, T, s, ACT, act_mode));
     }
-    TRY(proj(ACT, s, Kd, br.base + bl.off_down, h, PART, (long long)T * h, h, h, Kd, N));
+    TRY(proj_rows(ACT, s, br.base + bl.off_down, kd.data(), Kd));
     float* tap_f = last ? dptr<float>(m, p.taps) + (size_t)(2 * l + 1) * h : nullptr;
     normed = fuse_norm && l + 1 < c.n_layers;
     if (normed)

@@ -383,6 +383,8 @@ bool mega_supported(int dt, int h, int a, int b, int d, int s) {
   const int lpr = (int)(d * esz / 16);
   if (lpr != 4 && lpr != 8 && lpr != 16 && lpr != 32) return false;
   if (h > 16384 || h % 4) return false;
+  const int grp = a / b;
+  if (grp != 1 && grp != 2 && grp != 4 && grp != 8) return false;
   return mega_smem_bytes(dt, h, a, b, d, s, 128) <= 200 * 1024;
 }
 

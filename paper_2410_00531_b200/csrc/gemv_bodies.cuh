@@ -288,6 +288,8 @@ struct RowFusedArgs {
   long long shard_stride;  // elements
   const float* x_in;       // [N * Ks]
   int Ks, n_shards, rows, n_parts, prefetch_bytes;
+  int unequal;             // 1: shard i owns inputs [k0[i], k0[i+1]) and its matrix starts rows * k0[i] elements into W
+  int k0[ROWSHARD_MAX_UNEQUAL + 1];
   float* x;                // residual stream, in/out [rows]
   float* ss_part;          // [n_parts]: per-CTA sum of squares of its new entries (zeros beyond the grid)
   float* tap;              // optional copy of the new residual
@@ -305,7 +307,7 @@ __device__ __forceinline__ void rowfused_body(const RowFusedArgs& A, float* xs, 
   const int lo = (int)((long long)groups * cta / ncta);
   const int hi = (int)((long long)groups * (cta + 1) / ncta);
   const WT* Wall = reinterpret_cast<const WT*>(A.W);
-  if (lo + warp < hi) {
+  if (lo + warp < hi && !A.unequal) {
     const uint32_t pf = min((uint32_t)(R * A.Ks * sizeof(WT)), (uint32_t)A.prefetch_bytes) & ~15u;
     for (int sh = lane; sh < A.n_shards; sh += 32)
       if (pf) l2_prefetch_bulk(Wall + (size_t)sh * A.shard_stride + (size_t)(lo + warp) * R * A.Ks, pf);
@@ -313,7 +315,7 @@ __device__ __forceinline__ void rowfused_body(const RowFusedArgs& A, float* xs, 
   pdl_launch_dependents();
   pdl_wait();
 
-  const int ktot = A.n_shards * A.Ks;
+  const int ktot = A.unequal ? A.k0[A.n_shards] : A.n_shards * A.Ks;
   for (int k = threadIdx.x * 4; k < ktot; k += nw * 32 * 4)
     *reinterpret_cast<float4*>(xs + k) = *reinterpret_cast<const float4*>(A.x_in + k);
   __syncthreads();
@@ -369,12 +371,15 @@ __device__ __forceinline__ void rowfused_body(const RowFusedArgs& A, float* xs, 
       for (int sh = 0; sh < A.n_shards; ++sh) {
         const uint4* wp[R];
         float acc[R];
+        const int kb = A.unequal ? A.k0[sh] : sh * A.Ks;                 // first input of this shard
+        const int kw = A.unequal ? A.k0[sh + 1] - kb : A.Ks;             // its width
+        const size_t wbase = A.unequal ? (size_t)A.rows * kb : (size_t)sh * A.shard_stride;
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-          wp[r] = reinterpret_cast<const uint4*>(Wall + (size_t)sh * A.shard_stride + (size_t)(row0 + r) * A.Ks);
+          wp[r] = reinterpret_cast<const uint4*>(Wall + wbase + (size_t)(row0 + r) * kw);
           acc[r] = 0.f;
         }
-        warp_dot<WT, R>(wp, 0, xs + (size_t)sh * A.Ks, nvec, lane, acc);
+        warp_dot<WT, R>(wp, 0, xs + kb, kw / VEC, lane, acc);
 #pragma unroll
         for (int r = 0; r < R; ++r) {
           const float p = warp_sum(acc[r]);         // device sh's partial sum

@@ -62,6 +62,11 @@ cudaError_t launch_reduce_residual(const LaunchCtx& c, const float* partials, in
 cudaError_t launch_gemv_rowshard_fused(const LaunchCtx& c, int dt, const void* W, size_t shard_stride_elems,
                                        const float* x_in, int rows, int Ks, int n_shards, float* x,
                                        float* ss_part, float* tap);
+// The same for shards of unequal width (heterogeneous p_i): shard i owns columns [k0[i], k0[i+1]) of the K = k0[n_shards]
+// inputs, its matrix [rows][k0[i+1]-k0[i]] starts rows * k0[i] elements into W.  n_shards <= ROWSHARD_MAX_UNEQUAL.
+constexpr int ROWSHARD_MAX_UNEQUAL = 16;
+cudaError_t launch_gemv_rowshard_fused_unequal(const LaunchCtx& c, int dt, const void* W, const float* x_in, int rows,
+                                               const int* k0, int n_shards, float* x, float* ss_part, float* tap);
 int rowshard_fused_parts(int rows);
 bool rowshard_fused_supported(int Ks, int n_shards);
 

@@ -425,6 +425,39 @@ cudaError_t launch_gemv_rowshard_fused(const LaunchCtx& c, int dt, const void* W
 #undef TPI_RF
 }
 
+cudaError_t launch_gemv_rowshard_fused_unequal(const LaunchCtx& c, int dt, const void* W, const float* x_in, int rows,
+                                               const int* k0, int n_shards, float* x, float* ss_part, float* tap) {
+  if (n_shards < 1 || n_shards > ROWSHARD_MAX_UNEQUAL || !k0 || k0[0] != 0) return cudaErrorInvalidValue;
+  const int vec = dt == DT_BF16 ? 8 : 4;
+  for (int i = 0; i < n_shards; ++i)
+    if (k0[i + 1] <= k0[i] || (k0[i + 1] - k0[i]) % vec) return cudaErrorInvalidValue;
+  const int K = k0[n_shards];
+  if ((size_t)K * sizeof(float) > 200 * 1024) return cudaErrorInvalidValue;
+  RowFusedArgs A{};
+  A.W = W; A.shard_stride = 0; A.x_in = x_in; A.Ks = K; A.n_shards = n_shards;  // Ks * 1 shard sizes the staged x_in
+  A.rows = rows; A.x = x; A.ss_part = ss_part; A.tap = tap;
+  A.n_parts = rowshard_fused_parts(rows);
+  A.prefetch_bytes = 0;
+  A.unequal = 1;
+  for (int i = 0; i <= n_shards; ++i) A.k0[i] = k0[i];
+  // shared memory is sized from Ks * n_shards by the launcher: present the staged vector as one slice of K floats
+  RowFusedArgs L = A;
+  auto go = [&](auto wt) -> cudaError_t {
+    using WT = decltype(wt);
+    auto kern = gemv_rowshard_fused_kernel<WT, 1, 0, 0>;
+    static bool attr_done = false;
+    if (!attr_done) {
+      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+      if (e != cudaSuccess) return e;
+      attr_done = true;
+    }
+    int grid, warps;
+    balance_split(rows, &grid, &warps);
+    return launch_kernel(c, kern, dim3(grid), dim3(warps * 32), (size_t)K * sizeof(float), L);
+  };
+  return dt == DT_BF16 ? go(__nv_bfloat16{}) : go(float{});
+}
+
 // =====================================================================================
 // Embedding row + norm statistics (Algorithm 1 "Preprocess")
 // =====================================================================================

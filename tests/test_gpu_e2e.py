@@ -198,6 +198,49 @@ def test_scheduler_report_measures_the_propositions_inputs():
         assert r["tight_holds"] == r["loose_holds"] == r["retention_T"] == -2 and r["m_worker_bytes"] == 0
 
 
+@pytest.mark.parametrize("case", ["f32_gqa", "bf16_wide"])
+def test_heterogeneous_partition_matches_the_oracle(case):
+    """Sec. 3.1's proportions p_i: unequal shares of heads and FFN columns, prompt pass and decode, resident and streamed."""
+    import paper_2410_00531_b200 as P
+    if case == "f32_gqa":
+        shape = S.CONFIGS["C1"].with_(n_heads=8, n_kv_heads=4, head_dim=32, hidden=256, ffn=688, n_layers=3)
+        parts = [([2, 1, 1], [344, 200, 144]), ([3, 1], [512, 176])]
+    else:   # 7B-shaped widths, two layers: the tensor-core prompt pass with per-shard contractions of unequal length
+        shape = S.CONFIGS["C2"].with_(n_layers=2)
+        parts = [([24, 8], [8256, 2752]), ([16, 8, 4, 4], [5504, 2752, 1408, 1344])]
+    toks = S.prompt_tokens(shape)[:24]
+    tol = tol_for(shape)
+    for kv, ff in parts:
+        orc = make_oracle(shape)
+        want0 = orc.forward(toks, n_shards=len(kv), partition=(kv, ff))
+        for window in (0, 3):
+            with gpu_session(shape, 48, 16, 1, window) as ses:
+                P.set_partition(ses.h, kv, ff)
+                assert P.get_stats(ses.h)["n_shards"] == len(kv)
+                t0, lg0 = P.prefill(ses.h, toks, shape.vocab)
+                check_logits(lg0, t0, want0, tol)
+                for l in range(shape.n_layers):
+                    for which, key in ((0, "attn"), (1, "ffn")):
+                        assert rel_l2(P.get_hidden(ses.h, l, which, shape.hidden), orc.taps[(l, key)][-1]) <= tol
+                if window == 0:
+                    o2 = make_oracle(shape)
+                    o2.forward(toks, n_shards=len(kv), partition=(kv, ff))
+                    tok, want = int(np.argmax(want0)), None
+                    for _ in range(3):                                  # teacher-forced decode steps
+                        want = o2.forward([tok], n_shards=len(kv), partition=(kv, ff))
+                        got_tok, lg = P.decode_step(ses.h, tok, shape.vocab)
+                        check_logits(lg, got_tok, want, tol)
+                        tok = int(np.argmax(want))
+                    P.set_shards(ses.h, 1)                              # back to the uniform split
+                    t1, lg1 = P.prefill(ses.h, toks, shape.vocab)
+                    check_logits(lg1, t1, want0, tol)
+    with gpu_session(shape, 48, 16, 1) as ses:
+        for bad in (([1], [shape.ffn]), ([shape.n_kv_heads, 1], [shape.ffn - 8, 8]), ([shape.n_kv_heads - 1, 1], [shape.ffn - 3, 3]),
+                    ([shape.n_kv_heads, 0], [shape.ffn - 8, 8])):
+            with pytest.raises(P.TpiError):
+                P.set_partition(ses.h, *bad)
+
+
 def test_set_shards_and_set_window_roundtrip():
     import paper_2410_00531_b200 as P
     shape = S.CONFIGS["C1"]
@@ -231,6 +274,16 @@ def test_error_codes():
         with pytest.raises(P.TpiError) as e:
             P.set_window(ses.h, 2)                         # resident load kept no host images
         assert e.value.code in (-9, -3)
+
+
+def test_second_model_family_non_power_of_two_widths():
+    """A shape from the paper's model list outside the Llama 2/3 sizes (Yi-34B: hidden 7168, 56 heads over 8 kv
+    heads, FFN 20480): widths that are not powers of two, 7 query heads per kv head group... per shard, bf16,
+    N = 8; two layers and a 32000-entry vocabulary so that the oracle finishes in seconds."""
+    shape = S.CONFIGS["C3"].with_(n_layers=2, hidden=7168, n_heads=56, n_kv_heads=8, head_dim=128, ffn=20480, vocab=32000,
+                                  rope_base=5000000.0)
+    toks, mism = _run_and_compare(shape, 8, n_decode=4, prompt_len=96)
+    assert mism <= 2
 
 
 @pytest.mark.parametrize("cfg,n_shards,T", [("C2", 4, 128), ("C3", 8, 200)])

@@ -131,3 +131,24 @@ def test_matches_transformers_llama():
         # the library builds its rotary tables in float32, so agreement is ~1e-7, not 1e-15
         assert rel_l2(got, want) < 1e-5
         assert (got.argmax(-1) == want.argmax(-1)).all()
+
+
+def test_heterogeneous_partition_equals_unsharded_and_the_uniform_one():
+    """Sec. 3.1: device i takes a proportion p_i of the heads and of the FFN columns; whatever the proportions,
+    the sum of the devices' partial results is the unsharded layer (the paper's identity with single-server
+    inference), and the uniform proportions reproduce the default split exactly."""
+    shape = TINY.with_(n_heads=8, n_kv_heads=4, head_dim=4, ffn=48)
+    toks = S.prompt_tokens(shape, 7)
+    ref = make_oracle(shape)
+    want = ref.forward(toks)
+    for n, part in ((2, ([3, 1], [40, 8])), (3, ([2, 1, 1], [24, 16, 8])), (4, ([1, 1, 1, 1], [8, 8, 8, 24]))):
+        o = make_oracle(shape)
+        assert rel_l2(o.forward(toks, n_shards=n, partition=part), want) < 1e-12
+        for l in range(shape.n_layers):
+            assert rel_l2(o.taps[(l, "ffn")], ref.taps[(l, "ffn")]) < 1e-12
+        assert rel_l2(np.stack(o.cache.K), np.stack(ref.cache.K)) < 1e-13
+    u, v = make_oracle(shape), make_oracle(shape)
+    assert np.array_equal(u.forward(toks, n_shards=2), v.forward(toks, n_shards=2, partition=([2, 2], [24, 24])))
+    for bad in (([4, 1], [24, 24]), ([2, 2], [24, 16]), ([4, 0], [24, 24]), ([2, 2, 0], [24, 24])):
+        with pytest.raises(ValueError):
+            make_oracle(shape).forward(toks, n_shards=2, partition=bad)
