@@ -47,6 +47,8 @@ __device__ __forceinline__ void store_out(void* base, size_t i, size_t lo_off, f
 }
 
 constexpr int QB = 64, KB = 64;
+// decode kernel: DW warps per CTA, each takes DKB-key tiles (shorter tiles, more warps: a shorter dependent MMA chain per warp)
+constexpr int DW = 8, DKB = 32;
 
 // byte offset of 16-byte chunk c of row r in a tile whose rows hold D bf16 (chunks XOR-swizzled in groups of 8)
 template <int D>
@@ -244,12 +246,13 @@ cudaError_t launch_t(const LaunchCtx& c, const float* Q, const void* kc, const v
 namespace {
 
 template <int D>
-__global__ void __launch_bounds__(128) decode_attn_mma_kernel(const float* __restrict__ q, const __nv_bfloat16* kc,
+__global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* __restrict__ q, const __nv_bfloat16* kc,
                                                               const __nv_bfloat16* vc, const int* pos, int grp,
                                                               int max_seq, int nsplit, float* scratch,
                                                               unsigned* tickets, float* o_out) {
+  constexpr int KB = DKB;  // this kernel's tile: DKB keys per warp
   constexpr int KS = D / 16, ND = D / 8, CPR = D / 8, TILE = KB * D * 2;
-  extern __shared__ __align__(128) uint8_t smem[];  // [4 warps][K tile | V tile], reused by the merge buffers
+  extern __shared__ __align__(128) uint8_t smem[];  // [DW warps][K tile | V tile], reused by the merge buffers
   __shared__ bool s_last;
   pdl_launch_dependents();
   pdl_wait();
@@ -265,6 +268,25 @@ __global__ void __launch_bounds__(128) decode_attn_mma_kernel(const float* __res
   const __nv_bfloat16* kg = kc + (size_t)kvh * max_seq * D;
   const __nv_bfloat16* vg = vc + (size_t)kvh * max_seq * D;
   const uint32_t my_k = (uint32_t)__cvta_generic_to_shared(smem) + warp * 2 * TILE, my_v = my_k + TILE;
+
+  // this warp's K/V tile of 64-byte-swizzled rows; the first one is requested before anything else is read
+  auto issue_tile = [&](int k0) {
+    for (int i = lane; i < KB * CPR; i += 32) {
+      const int r = i / CPR, c = i - r * CPR;
+      const uint32_t off = tile_off<D>(r, c);
+      if (k0 + r < s1) {
+        const size_t src = (size_t)(k0 + r) * D + c * 8;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(my_k + off), "l"(kg + src) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(my_v + off), "l"(vg + src) : "memory");
+      } else {
+        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(my_k + off), "r"(0u) : "memory");
+        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(my_v + off), "r"(0u) : "memory");
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  const int k_first = s0 + warp * KB;
+  if (k_first < s1) issue_tile(k_first);
 
   // Q fragments: row g = head g of the group (rows >= grp and rows 8..15 are zero)
   const float qscale = 1.4426950408889634f * rsqrtf((float)D);
@@ -286,21 +308,11 @@ __global__ void __launch_bounds__(128) decode_attn_mma_kernel(const float* __res
   for (int nd = 0; nd < ND; ++nd) { o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f; }
   float m_r = -INFINITY, l_r = 0.f;
 
-  for (int k0 = s0 + warp * KB; k0 < s1; k0 += 4 * KB) {  // this warp's tiles of the split
-    __syncwarp();
-    for (int i = lane; i < KB * CPR; i += 32) {
-      const int r = i / CPR, c = i - r * CPR;
-      const uint32_t off = tile_off<D>(r, c);
-      if (k0 + r < s1) {
-        const size_t src = (size_t)(k0 + r) * D + c * 8;
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(my_k + off), "l"(kg + src) : "memory");
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(my_v + off), "l"(vg + src) : "memory");
-      } else {
-        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(my_k + off), "r"(0u) : "memory");
-        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(my_v + off), "r"(0u) : "memory");
-      }
+  for (int k0 = k_first; k0 < s1; k0 += DW * KB) {  // this warp's tiles of the split
+    if (k0 != k_first) {
+      __syncwarp();
+      issue_tile(k0);
     }
-    asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncwarp();
     float s[KB / 8][4];
@@ -360,10 +372,10 @@ __global__ void __launch_bounds__(128) decode_attn_mma_kernel(const float* __res
 
   // ---- fold the 4 warps (fixed order).  Buffers alias the tiles, so everyone must be done reading them.
   __syncthreads();
-  float* w_m = reinterpret_cast<float*>(smem);  // [4][8]
-  float* w_l = w_m + 32;                        // [4][8]
-  float* w_o = w_l + 32;                        // [4][8][D]
-  float* mw = w_o + 4 * 8 * D;                  // [grp][nsplit] weights of the final merge
+  float* w_m = reinterpret_cast<float*>(smem);  // [DW][8]
+  float* w_l = w_m + DW * 8;                    // [DW][8]
+  float* w_o = w_l + DW * 8;                    // [DW][8][D]
+  float* mw = w_o + DW * 8 * D;                 // [grp][nsplit] weights of the final merge
   if (t == 0) { w_m[warp * 8 + g] = m_r; w_l[warp * 8 + g] = l_r; }
 #pragma unroll
   for (int nd = 0; nd < ND; ++nd) {
@@ -372,14 +384,14 @@ __global__ void __launch_bounds__(128) decode_attn_mma_kernel(const float* __res
   }
   __syncthreads();
   float* part = scratch + ((size_t)kvh * nsplit + split) * grp * (D + 2);
-  for (int e = threadIdx.x; e < grp * D; e += 128) {
+  for (int e = threadIdx.x; e < grp * D; e += DW * 32) {
     const int hh = e / D, dd = e - hh * D;
     float M = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < 4; ++w) M = fmaxf(M, w_m[w * 8 + hh]);
+    for (int w = 0; w < DW; ++w) M = fmaxf(M, w_m[w * 8 + hh]);
     float A = 0.f, L = 0.f;
 #pragma unroll
-    for (int w = 0; w < 4; ++w) {
+    for (int w = 0; w < DW; ++w) {
       const float sc = exp2f(w_m[w * 8 + hh] - M);  // a warp that saw no tile has m = -inf, weight 0
       A = fmaf(sc, w_o[(w * 8 + hh) * D + dd], A);
       L = fmaf(sc, w_l[w * 8 + hh], L);
@@ -402,7 +414,7 @@ __global__ void __launch_bounds__(128) decode_attn_mma_kernel(const float* __res
   if (!s_last) return;
   __threadfence();
   const float* pg = scratch + (size_t)kvh * nsplit * grp * (D + 2);
-  for (int hh = warp; hh < grp; hh += 4) {
+  for (int hh = warp; hh < grp; hh += DW) {
     float M = -INFINITY;
     for (int sI = lane; sI < nact; sI += 32) M = fmaxf(M, __ldcg(pg + (size_t)(sI * grp + hh) * (D + 2)));
 #pragma unroll
@@ -419,7 +431,7 @@ __global__ void __launch_bounds__(128) decode_attn_mma_kernel(const float* __res
     for (int sI = lane; sI < nact; sI += 32) mw[hh * nact + sI] *= inv;
   }
   __syncthreads();
-  for (int e = threadIdx.x; e < grp * D; e += 128) {
+  for (int e = threadIdx.x; e < grp * D; e += DW * 32) {
     const int hh = e / D, dd = e - hh * D;
     float A = 0.f;
 #pragma unroll 8
@@ -434,14 +446,14 @@ template <int D>
 cudaError_t launch_dec_t(const LaunchCtx& c, const float* q, const void* kc, const void* vc, const int* pos, int a,
                          int b, int max_seq, int nsplit, float* scratch, unsigned* tickets, float* o) {
   auto kern = decode_attn_mma_kernel<D>;
-  const size_t smem = (size_t)4 * 2 * KB * D * 2;  // >= merge buffers (64 + 32 D + grp * nsplit floats)
+  const size_t smem = (size_t)DW * 2 * DKB * D * 2;  // >= merge buffers (16 DW + 8 DW D + grp * nsplit floats)
   static bool attr_done = false;
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  return launch_kernel(c, kern, dim3(b, nsplit), dim3(128), smem, q, (const __nv_bfloat16*)kc,
+  return launch_kernel(c, kern, dim3(b, nsplit), dim3(DW * 32), smem, q, (const __nv_bfloat16*)kc,
                        (const __nv_bfloat16*)vc, pos, a / b, max_seq, nsplit, scratch, tickets, o);
 }
 
@@ -449,7 +461,7 @@ cudaError_t launch_dec_t(const LaunchCtx& c, const float* q, const void* kc, con
 
 bool decode_attention_mma_supported(int dt, int a, int b, int d, int nsplit) {
   const int grp = a / b;
-  return dt == DT_BF16 && (d == 128 || d == 64) && grp <= 8 && (size_t)(64 + 32 * d + grp * nsplit) * 4 <= (size_t)4 * 2 * KB * d * 2;
+  return dt == DT_BF16 && (d == 128 || d == 64) && grp <= 8 && (size_t)(16 * DW + 8 * DW * d + grp * nsplit) * 4 <= (size_t)DW * 2 * DKB * d * 2;
 }
 
 cudaError_t launch_decode_attention_mma(const LaunchCtx& c, const float* q, const void* kcache_layer,
