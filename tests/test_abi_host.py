@@ -149,6 +149,20 @@ def test_ring_with_block_retention_reproduces_the_oracle_timeline(w, T):
     assert np.allclose(stalls, want) and np.isclose(end, want_end)
 
 
+@pytest.mark.parametrize("w", [3, 5, 7])
+def test_ring_with_an_odd_window_follows_the_per_kind_places_of_prop5(w):
+    """Prop. 5 splits an odd window into floor(w/2) attention and ceil(w/2) FFN places; the ring deals its slots the
+    same way, so its stalls are those of the oracle's per-kind event model (retention off)."""
+    ta, tf, tr, la, lf = 11.0, 17.0, 2.0, 18.0, 30.0            # loads slower than compute: the window size matters
+    L, n_exec = 12, 70
+    ops = P.ring_trace(2 * L, w, n_exec)
+    stalls, end = replay(ops, (ta, tf), tr, (la, lf), 2 * L)
+    want, _, want_end = W.timeline_retained(ta, tf, tr, la, lf, n_exec, w, 0, L)
+    assert np.allclose(stalls, want) and np.isclose(end, want_end)
+    slots = {int(sl) for op, sl, _ in ops if op == 1}
+    assert len(slots) == w                                      # every place of the window gets used
+
+
 def test_ring_invariants():
     for w in (1, 2, 3, 5, 8):
         n_blocks = 8

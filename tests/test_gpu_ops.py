@@ -160,6 +160,8 @@ def test_qkv_rope_kv_append(T, cfg, n_shards, p):
     ("bf16", 8, 2, 128, 1, 3),           # the same on the tensor-core path
     ("bf16", 16, 2, 64, 700, 4),         # 8 heads per kv head, d = 64, three active splits
     ("bf16", 32, 8, 128, 257, 33),       # just past one split
+    ("bf16", 56, 8, 128, 300, 3),        # 7 query heads per kv head (Yi-34B shape)
+    ("bf16", 12, 4, 64, 95, 2),          # 3 per group, ragged 32-key tiles
     ("f32", 8, 4, 64, 33, 8),
 ])
 def test_decode_attention(T, dtype, a, b, d, n, nsplit):
