@@ -276,6 +276,47 @@ def test_error_codes():
         assert e.value.code in (-9, -3)
 
 
+def test_full_size_7b_shape_sampled_outputs_and_size_independent_properties():
+    """The benchmarked 7B-shaped workload at FULL depth in bench.py's launch configuration (graph + PDL).  The oracle
+    cannot run 32 layers in seconds, so (a) it computes what it can one by one: layer 0's two hidden states of the last
+    prompt position (a one-layer oracle sees the same embedding and layer-0 weights); (b) properties that hold at any
+    size: the result does not depend on the number of shards (the paper's identity with single-server inference, here
+    up to the fp32 order of the partial sums), a streamed model gives the resident model's bits, and one enqueue of
+    several tokens gives the per-token calls' tokens."""
+    import paper_2410_00531_b200 as P
+    shape = S.CONFIGS["C2"]
+    toks = S.prompt_tokens(shape)
+    T, n_dec = len(toks), 6
+    one = make_oracle(shape.with_(n_layers=1))
+    one.forward(toks)
+    res = {}
+    with gpu_session(shape, T + 2 * n_dec + 2, T, 4, 0, keep_host_images=True, other_windows=(4,)) as ses:
+        for key, n, w in (("n4", 4, 0), ("n1", 1, 0), ("n4w4", 4, 4)):
+            P.set_shards(ses.h, n)
+            P.set_window(ses.h, w)
+            P.set_option(ses.h, P.OPT_MEGA, 0)
+            t0, lg = P.prefill(ses.h, toks, shape.vocab)
+            h_attn, h_ffn = P.get_hidden(ses.h, 0, 0, shape.hidden), P.get_hidden(ses.h, 0, 1, shape.hidden)
+            assert rel_l2(h_attn, one.taps[(0, "attn")][-1]) <= 1e-2 and rel_l2(h_ffn, one.taps[(0, "ffn")][-1]) <= 1e-2
+            seq = P.decode_run(ses.h, t0, n_dec)                        # one enqueue (graph replay when resident)
+            P.set_position(ses.h, T)                                    # rewind: the same steps, one call each
+            step, tok = [], t0
+            for _ in range(n_dec):
+                tok, _ = P.decode_step(ses.h, tok, 0)
+                step.append(tok)
+            assert list(seq) == step
+            res[key] = (t0, lg, list(seq))
+    assert np.isfinite(res["n4"][1]).all()
+    assert res["n4w4"][0] == res["n4"][0] and np.array_equal(res["n4w4"][1], res["n4"][1]) and res["n4w4"][2] == res["n4"][2]
+    # Same bf16 weights and exact products; only the fp32 order of the partial sums differs.  Where that moves a key or
+    # value across a bf16 rounding boundary the cache entry changes by one bf16 ulp, and 32 layers carry it on:
+    # 1.7e-3 observed, inside the 1e-2 bar that bf16 weights are given.
+    assert rel_l2(res["n1"][1], res["n4"][1]) < 1e-2
+    g = np.sort(res["n4"][1])[::-1]
+    if g[0] - g[1] > 3e-2 * np.sqrt(np.mean(g * g)):
+        assert res["n1"][0] == res["n4"][0]
+
+
 def test_second_model_family_non_power_of_two_widths():
     """A shape from the paper's model list outside the Llama 2/3 sizes (Yi-34B: hidden 7168, 56 heads over 8 kv
     heads, FFN 20480): widths that are not powers of two, 7 query heads per kv head group... per shard, bf16,
