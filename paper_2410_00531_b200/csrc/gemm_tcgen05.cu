@@ -104,17 +104,6 @@ struct GemmTcArgs {
   int act_ld, act_split;
 };
 
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[32]) {  // columns [0, 16) of r
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
 constexpr int kBM = 128, kBK = 64;
 // tensor-memory columns are allocated in powers of two
 __host__ __device__ constexpr uint32_t tmem_cols(int bn) { return bn <= 32 ? 32u : bn <= 64 ? 64u : bn <= 128 ? 128u : 256u; }
@@ -135,6 +124,7 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES], acc_ready;
   __shared__ uint32_t tmem_base_s;
+  static_assert(BN % 32 == 0 && BN <= 256, "the epilogue reads 32 accumulator columns at a time");
   constexpr uint32_t TCOLS = tmem_cols(BN);
   constexpr uint32_t A_BYTES = kBM * kBK * 2, B_BYTES = BN * kBK * 2, STAGE_BYTES = (1 + SPLIT) * A_BYTES + B_BYTES;
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -208,13 +198,6 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         uint32_t r[32];
-        if (BN - c0 < 32) {  // a tile width that is an odd multiple of 16: the last 16 columns (plain output only)
-          tmem_ld16(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
-          if (row < a.T && !a.act)
-            for (int j = 0; j < 16; ++j)
-              if (n0 + c0 + j < a.n_out) yrow[c0 + j] = __uint_as_float(r[j]);
-          break;
-        }
         tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
         if (row < a.T && a.act) {
           __nv_bfloat16* arow = a.act + (size_t)row * a.act_ld + ((n0 + c0) >> 1);
