@@ -190,9 +190,14 @@ def run_gpu(args, shape):
     extra = 0
     if args.window > 0 and args.retain > 0:      # room for the kept FFN blocks beside the window (Prop. 6)
         extra = len(range(0, shape.n_layers, args.retain)) * P.block_bytes(cfg)[1]
+    elif args.window > 0 and args.retain == -1:  # as many as fit in what the GPU has free (leave 8 GiB of headroom)
+        import torch
+        free_b, _ = torch.cuda.mem_get_info(local)
+        base = P.query_arena(cfg, shape.n_shards, args.window, True)[0]
+        extra = max(0, min(shape.n_layers * P.block_bytes(cfg)[1], free_b - base - (8 << 30)))
     ses = P.Session(cfg, S.synth_fill(shape), shape.n_shards, args.window, device=local, extra_dev_bytes=extra)
     if extra:
-        P.set_retention(ses.h, args.retain)
+        P.set_retention(ses.h, args.retain)      # -1: the library picks the smallest T that fits the arena
     t_load = time.perf_counter() - t_load
     if args.window > 0:
         return run_streamed(args, shape, ses, t_load, local, rank)
@@ -365,7 +370,7 @@ def run_streamed(args, shape, ses, t_load, local, rank):
         "config": {"workload": workload_name(shape, args).replace("all weights resident", f"layer blocks streamed from pinned host memory, window {args.window} blocks"),
                    "l2": "inputs larger than L2 (every block is copied from host memory each token)",
                    "window_blocks": args.window, "window_device_bytes": st["window_peak_bytes"],
-                   "retain_ffn_every": args.retain, "retained_blocks": st["retained_blocks"],
+                   "retain_ffn_every": sched["retain_every_T"], "retained_blocks": st["retained_blocks"],
                    "retained_device_bytes": st["retained_bytes"],
                    "block_bytes": {"attention": attn_b, "ffn": ffn_b}, "load_s": round(t_load, 1)},
         "clocks": clocks,
@@ -392,7 +397,7 @@ def main():
     ap.add_argument("--workload", default="C2", choices=sorted(S.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--retain", type=int, default=0,
-                    help="with --window: keep one FFN block in every T resident beside the window (0 = none)")
+                    help="with --window: keep one FFN block in every T resident beside the window (0 = none, -1 = as many as fit)")
     ap.add_argument("--window", type=int, default=0,
                     help="stream the layer blocks through a window of this many blocks (0 = all resident)")
     ap.add_argument("--prompt", type=int, default=0, help="override the prompt length")

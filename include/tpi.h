@@ -130,7 +130,8 @@ int tpi_set_partition(tpi_model *m, int n_shards, const int32_t *kv_heads_per_sh
 
 /* Block retention (Sec. 3.3, Prop. 6 / Appendix A.6): when the link is the bottleneck, keep ONE FFN
  * block in every `ffn_every_T` FFN blocks resident (layers 0, T, 2T, ...) beside the window and stream
- * only the rest; 0 turns retention off, 1 keeps every FFN block.  Only for a streamed model
+ * only the rest; 0 turns retention off, 1 keeps every FFN block, -1 picks the smallest T whose kept
+ * blocks fit in the device arena beside the window (0 if none fits).  Only for a streamed model
  * (window >= 1).  The retained blocks live in the device arena after the window slots: the arena must
  * have room for them (TPI_ERR_NOMEM otherwise, and the previous setting stays in force).  Keeps the KV
  * cache and the position; results are bit-identical with and without retention.  tpi_set_window turns

@@ -779,8 +779,18 @@ extern "C" int tpi_set_window(tpi_model* m, int window_blocks) {
 }
 
 extern "C" int tpi_set_retention(tpi_model* m, int ffn_every_T) {
-  if (!m || ffn_every_T < 0) return fail(TPI_ERR_INVALID_ARG, "bad argument");
+  if (!m || ffn_every_T < -1) return fail(TPI_ERR_INVALID_ARG, "bad argument");
   if (m->window <= 0) return fail(TPI_ERR_STATE, "block retention applies to a streamed model (window >= 1)");
+  if (ffn_every_T == -1) {  // as many FFN blocks as the device arena has room for beside the window: the smallest T that fits
+    int nA, nF;
+    window_slots(m->window, &nA, &nF);
+    const size_t used = m->plan.blocks + (size_t)nA * m->plan.bl.attn_bytes + (size_t)nF * m->plan.bl.ffn_bytes;
+    const size_t spare = m->res.dev_bytes > used ? m->res.dev_bytes - used : 0;
+    const long long fit = (long long)(spare / m->plan.bl.ffn_bytes);
+    ffn_every_T = 0;
+    for (int T = 1; T <= m->cfg.n_layers && fit > 0; ++T)
+      if ((m->cfg.n_layers + T - 1) / T <= fit) { ffn_every_T = T; break; }
+  }
   TRY(quiesce(m));
   drop_graph(m);
   const int old = m->retain_T;

@@ -165,6 +165,12 @@ def test_block_retention_is_bit_identical_and_loads_less(window, T):
         assert a[0] == b[0] and a[3] == b[3] and (a[2] == b[2]).all()
         assert np.array_equal(a[1], b[1]) and np.array_equal(a[4], b[4])
     assert loads["retained"] < loads["streamed"]
+    # automatic period: the smallest T whose kept blocks fit the room that the arena has beside the window
+    for room, want_T in ((shape.n_layers, 1), (3, 2), (2, 3), (1, 6), (0, 0)):
+        with gpu_session(shape, 64, 16, 2, window, extra_dev_bytes=room * ffn_bytes + 64) as ses:
+            P.set_retention(ses.h, -1)
+            r = P.scheduler_report(ses.h)
+            assert r["retain_every_T"] == want_T and P.get_stats(ses.h)["retained_blocks"] == (len(range(0, 6, want_T)) if want_T else 0)
 
 
 def test_scheduler_report_measures_the_propositions_inputs():
