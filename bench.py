@@ -50,6 +50,32 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def tensor_peak():
+    """Measured dense bf16 throughput (TFLOP/s): (burst, sustained), kind."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["bf16_tflops"]), float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "measured"
+    return 1590.0, 1400.0, "fallback"
+
+
+def ttft_roofline(shape, T, ttft_ms, weight_bytes, hbm_gbs):
+    """The prompt pass against the slower of: every weight byte once over HBM, and its matrix products plus causal
+    attention on the tensor cores at the measured bf16 rate (one product per activation: the split-bf16 scheme's second
+    product is overhead).  The rate is the burst figure below ~10 ms of ideal time, the sustained one above."""
+    a, b, d, h, s_, L, v = shape.n_heads, shape.n_kv_heads, shape.head_dim, shape.hidden, shape.ffn, shape.n_layers, shape.vocab
+    per_layer = (a + 2 * b) * d * h + a * d * h + 3 * h * s_
+    flops = 2.0 * T * L * per_layer + 2.0 * v * h + 4.0 * (T * (T + 1) / 2) * a * d * L
+    burst, sustained, kind = tensor_peak()
+    t_hbm = weight_bytes / (hbm_gbs * 1e9) * 1e3
+    t_tc = flops / (burst * 1e12) * 1e3
+    if t_tc > 10.0:
+        t_tc = flops / (sustained * 1e12) * 1e3
+    ideal = max(t_hbm, t_tc)
+    return {"bound": "hbm" if t_hbm >= t_tc else "tensor", "ideal_ms": ideal, "hbm_ms": t_hbm, "tensor_ms": t_tc,
+            "flops": flops, "frac": ideal / ttft_ms, "peak_kind": kind}
+
+
 def traffic_from_profile(workload: str):
     """DRAM bytes per launch of the dominant kernel, from the committed ncu summary (or None)."""
     p = os.path.join(ROOT, "profiles", f"gemv_gateup_{workload.lower()}.md")
@@ -291,6 +317,7 @@ def run_gpu(args, shape):
         "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": 4, "d2h_bytes_per_step": 8},
         "gpu_launches": launches,
         "ttft_ms": ttft_ms, "ttft_prompt_tokens": T,
+        "ttft_roofline": ttft_roofline(shape, T, ttft_ms, st["weight_bytes_per_token"], peak),
         "token_roofline": {"bound": "hbm", "bytes_per_token": token_bytes, "achieved": token_gbs, "peak": peak,
                            "unit": "GB/s", "frac": token_gbs / peak, "peak_kind": peak_kind},
         "roofline": {"bound": "hbm", "kernel": "gemv_cols_kernel<bf16,EPI_SWIGLU> (gate/up + SwiGLU)",
