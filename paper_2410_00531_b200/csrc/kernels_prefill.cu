@@ -48,7 +48,7 @@ cudaError_t launch_embed_rows(const LaunchCtx& c, int dt, const void* emb, const
 // ------------------------------------------------------------------ RMSNorm rows
 // Row kernels below share one mapping so that their sums agree to the bit: thread tid owns the float4 groups
 // tid, tid + B, ... of the row (B threads), adds the squares of its elements in index order, then block_sum.
-constexpr int ROW_KEEP = 8;  // float4 groups a thread keeps in registers (rows up to 32 * B elements)
+constexpr int ROW_KEEP = 8;  // most float4 groups a thread keeps in registers (rows up to 32 * B elements)
 __device__ __forceinline__ float sq4(float4 v, float ss) {
   ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
   return ss;
@@ -75,7 +75,7 @@ __device__ __forceinline__ void store_act4(void* base, size_t i, size_t lo_off, 
 static inline int row_threads(int h) { return h / 4 <= 8 * 256 ? 256 : 1024; }
 
 // PARTS: 0 = plain RMSNorm of X; 1 = first X <- ((P_0 + P_1) + ...) + X (star sum in rank order + shortcut), then the norm.
-template <int MODE, int PARTS, int THREADS>
+template <int MODE, int PARTS, int THREADS, int KEEP>
 __global__ void __launch_bounds__(THREADS) norm_rows_kernel(const float* __restrict__ partials, int n_shards, int T, int h,
                                                         float* X, float* tap_last, const float* __restrict__ gain,
                                                         float eps, void* Xn, size_t lo_off) {
@@ -84,17 +84,17 @@ __global__ void __launch_bounds__(THREADS) norm_rows_kernel(const float* __restr
   __shared__ float red[32];
   const int B = blockDim.x, ng = h >> 2;
   const size_t n = (size_t)T * h, row = (size_t)blockIdx.x * h;
-  float4 v[ROW_KEEP];
+  float4 v[KEEP];
 #pragma unroll
-  for (int j = 0; j < ROW_KEEP; ++j) {
+  for (int j = 0; j < KEEP; ++j) {
     const int g = threadIdx.x + j * B;
     if (g < ng) v[j] = *reinterpret_cast<const float4*>(X + row + 4 * g);
   }
   if (PARTS) {
-    float4 acc[ROW_KEEP];
+    float4 acc[KEEP];
     for (int sh = 0; sh < n_shards; ++sh) {
 #pragma unroll
-      for (int j = 0; j < ROW_KEEP; ++j) {
+      for (int j = 0; j < KEEP; ++j) {
         const int g = threadIdx.x + j * B;
         if (g < ng) {
           const float4 p = *reinterpret_cast<const float4*>(partials + (size_t)sh * n + row + 4 * g);
@@ -104,7 +104,7 @@ __global__ void __launch_bounds__(THREADS) norm_rows_kernel(const float* __restr
       }
     }
 #pragma unroll
-    for (int j = 0; j < ROW_KEEP; ++j) {
+    for (int j = 0; j < KEEP; ++j) {
       const int g = threadIdx.x + j * B;
       if (g < ng) {
         v[j].x = acc[j].x + v[j].x; v[j].y = acc[j].y + v[j].y; v[j].z = acc[j].z + v[j].z; v[j].w = acc[j].w + v[j].w;
@@ -116,14 +116,14 @@ __global__ void __launch_bounds__(THREADS) norm_rows_kernel(const float* __restr
   if (!gain) return;  // sum and shortcut only
   float ss = 0.f;
 #pragma unroll
-  for (int j = 0; j < ROW_KEEP; ++j) {
+  for (int j = 0; j < KEEP; ++j) {
     const int g = threadIdx.x + j * B;
     if (g < ng) ss = sq4(v[j], ss);
   }
   ss = block_sum(ss, red);
   const float r = rsqrtf(ss / (float)h + eps);
 #pragma unroll
-  for (int j = 0; j < ROW_KEEP; ++j) {
+  for (int j = 0; j < KEEP; ++j) {
     const int g = threadIdx.x + j * B;
     if (g < ng) {
       const float4 gn = *reinterpret_cast<const float4*>(gain + 4 * g);
@@ -155,10 +155,14 @@ template <int PARTS>
 static cudaError_t launch_norm_rows_vec(const LaunchCtx& c, const float* partials, int n_shards, int T, int h, float* X,
                                         float* tap_last, const float* gain, float eps, void* Xn, int mode) {
   const size_t lo = (size_t)T * h;
-#define TPI_NR(MODE, THREADS) \
-  launch_kernel(c, norm_rows_kernel<MODE, PARTS, THREADS>, dim3(T), dim3(THREADS), 0, partials, n_shards, T, h, X, tap_last, gain, eps, Xn, lo)
-  if (row_threads(h) == 256) return mode == 2 ? TPI_NR(2, 256) : mode == 1 ? TPI_NR(1, 256) : TPI_NR(0, 256);
-  return mode == 2 ? TPI_NR(2, 1024) : mode == 1 ? TPI_NR(1, 1024) : TPI_NR(0, 1024);
+#define TPI_NR(MODE, THREADS, KEEP) \
+  launch_kernel(c, norm_rows_kernel<MODE, PARTS, THREADS, KEEP>, dim3(T), dim3(THREADS), 0, partials, n_shards, T, h, X, tap_last, gain, eps, Xn, lo)
+  if (row_threads(h) == 256) {
+    if (h / 4 <= 4 * 256)  // rows up to 4096: half the registers, more rows in flight per SM
+      return mode == 2 ? TPI_NR(2, 256, 4) : mode == 1 ? TPI_NR(1, 256, 4) : TPI_NR(0, 256, 4);
+    return mode == 2 ? TPI_NR(2, 256, 8) : mode == 1 ? TPI_NR(1, 256, 8) : TPI_NR(0, 256, 8);
+  }
+  return mode == 2 ? TPI_NR(2, 1024, 8) : mode == 1 ? TPI_NR(1, 1024, 8) : TPI_NR(0, 1024, 8);
 #undef TPI_NR
 }
 
