@@ -428,6 +428,7 @@ def main():
     ap.add_argument("--window", type=int, default=0,
                     help="stream the layer blocks through a window of this many blocks (0 = all resident)")
     ap.add_argument("--prompt", type=int, default=0, help="override the prompt length")
+    ap.add_argument("--shards", type=int, default=0, help="override the number of emulated shards N")
     ap.add_argument("--quick", action="store_true",
                     help="one prompt pass and the device-resident decode loop only (short runs under a profiler)")
     ap.add_argument("--layers", type=int, default=0, help="override the depth (small captures under a profiler)")
@@ -437,6 +438,8 @@ def main():
         shape = shape.with_(n_layers=args.layers)
     if args.prompt:
         shape = shape.with_(prompt_len=args.prompt)
+    if args.shards:
+        shape = shape.with_(n_shards=args.shards)
     if args.impl == "reference":
         run_reference(args, shape)
     else:
