@@ -255,10 +255,11 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
   extern __shared__ __align__(128) uint8_t smem[];  // [DW warps][K tile | V tile], reused by the merge buffers
   __shared__ bool s_last;
   pdl_launch_dependents();
-  pdl_wait();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int kvh = blockIdx.x, split = blockIdx.y;
+  // The position counter was advanced when the previous token ended, long before this launch; only the cache row of
+  // the newest position (and the queries) come from the kernel just before this one.
   const int n = *pos + 1;
   int chunk = (n + nsplit - 1) / nsplit;
   chunk = max(256, (chunk + 63) & ~63);
@@ -286,7 +287,10 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
   const int k_first = s0 + warp * KB;
-  if (k_first < s1) issue_tile(k_first);
+  const bool early = k_first + KB <= n - 1;  // a tile of older positions only: requested ahead of the dependency wait
+  if (k_first < s1 && early) issue_tile(k_first);
+  pdl_wait();
+  if (k_first < s1 && !early) issue_tile(k_first);
 
   // Q fragments: row g = head g of the group (rows >= grp and rows 8..15 are zero)
   const float qscale = 1.4426950408889634f * rsqrtf((float)D);
@@ -414,17 +418,30 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
   if (!s_last) return;
   __threadfence();
   const float* pg = scratch + (size_t)kvh * nsplit * grp * (D + 2);
+  // All partial results of this kv head come into shared memory in one batch of independent loads (one trip to L2
+  // instead of a dependent chain per pass) when they fit: nact * grp * (D + 2) floats next to the merge weights.
+  constexpr int SMEM_FLOATS = DW * 2 * DKB * D * 2 / 4;
+  const int tot = nact * grp * (D + 2);
+  const bool staged = tot + grp * nact <= SMEM_FLOATS;
+  float* sp = reinterpret_cast<float*>(smem);
+  if (staged) {
+    for (int i = threadIdx.x; i < tot / 2; i += DW * 32)
+      reinterpret_cast<float2*>(sp)[i] = __ldcg(reinterpret_cast<const float2*>(pg) + i);
+    mw = sp + tot;
+    __syncthreads();
+  }
+  auto part_at = [&](int idx) { return staged ? sp[idx] : __ldcg(pg + idx); };
   for (int hh = warp; hh < grp; hh += DW) {
     float M = -INFINITY;
-    for (int sI = lane; sI < nact; sI += 32) M = fmaxf(M, __ldcg(pg + (size_t)(sI * grp + hh) * (D + 2)));
+    for (int sI = lane; sI < nact; sI += 32) M = fmaxf(M, part_at((sI * grp + hh) * (D + 2)));
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, off));
     float L = 0.f;
     for (int sI = lane; sI < nact; sI += 32) {
-      const float* ps = pg + (size_t)(sI * grp + hh) * (D + 2);
-      const float w = exp2f(__ldcg(ps) - M);
+      const int ps = (sI * grp + hh) * (D + 2);
+      const float w = exp2f(part_at(ps) - M);
       mw[hh * nact + sI] = w;
-      L = fmaf(w, __ldcg(ps + 1), L);
+      L = fmaf(w, part_at(ps + 1), L);
     }
     L = warp_sum(L);
     const float inv = 1.f / L;
@@ -435,8 +452,7 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
     const int hh = e / D, dd = e - hh * D;
     float A = 0.f;
 #pragma unroll 8
-    for (int sI = 0; sI < nact; ++sI)
-      A = fmaf(mw[hh * nact + sI], __ldcg(pg + (size_t)(sI * grp + hh) * (D + 2) + 2 + dd), A);
+    for (int sI = 0; sI < nact; ++sI) A = fmaf(mw[hh * nact + sI], part_at((sI * grp + hh) * (D + 2) + 2 + dd), A);
     o_out[(size_t)(kvh * grp + hh) * D + dd] = A;
   }
   if (threadIdx.x == 0) tickets[kvh] = 0u;
