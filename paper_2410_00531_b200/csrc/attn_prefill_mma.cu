@@ -418,6 +418,45 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
   if (!s_last) return;
   __threadfence();
   const float* pg = scratch + (size_t)kvh * nsplit * grp * (D + 2);
+  constexpr int MAXN = 24, EPT = 2;  // register path: up to MAXN splits, up to EPT outputs per thread
+  if (nact <= MAXN && grp * D <= EPT * DW * 32) {
+    // Few splits: every thread requests the partial values of its own outputs straight away (independent loads, one
+    // trip to L2) while the first warps turn the splits' maxima and sums into merge weights; then the weighted sums.
+    float v[EPT][MAXN];
+#pragma unroll
+    for (int j = 0; j < EPT; ++j) {
+      const int e = threadIdx.x + j * DW * 32;
+      const int hh = e / D, dd = e - hh * D;
+#pragma unroll
+      for (int sI = 0; sI < MAXN; ++sI)
+        if (e < grp * D && sI < nact) v[j][sI] = __ldcg(pg + (size_t)(sI * grp + hh) * (D + 2) + 2 + dd);
+    }
+    for (int hh = warp; hh < grp; hh += DW) {
+      const float m_s = lane < nact ? __ldcg(pg + (size_t)(lane * grp + hh) * (D + 2)) : -INFINITY;  // nact <= 24 < 32 lanes
+      const float l_s = lane < nact ? __ldcg(pg + (size_t)(lane * grp + hh) * (D + 2) + 1) : 0.f;
+      float M = m_s;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, off));
+      const float w = lane < nact ? exp2f(m_s - M) : 0.f;
+      const float L = warp_sum(w * l_s);
+      if (lane < nact) mw[hh * nact + lane] = w / L;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < EPT; ++j) {
+      const int e = threadIdx.x + j * DW * 32;
+      if (e < grp * D) {
+        const int hh = e / D, dd = e - hh * D;
+        float A = 0.f;
+#pragma unroll
+        for (int sI = 0; sI < MAXN; ++sI)
+          if (sI < nact) A = fmaf(mw[hh * nact + sI], v[j][sI], A);
+        o_out[(size_t)(kvh * grp + hh) * D + dd] = A;
+      }
+    }
+    if (threadIdx.x == 0) tickets[kvh] = 0u;
+    return;
+  }
   // All partial results of this kv head come into shared memory in one batch of independent loads (one trip to L2
   // instead of a dependent chain per pass) when they fit: nact * grp * (D + 2) floats next to the merge weights.
   constexpr int SMEM_FLOATS = DW * 2 * DKB * D * 2 / 4;
