@@ -139,20 +139,24 @@ __device__ __forceinline__ void cols_body(const GemvArgs& A, float* xs, const in
       if (pf) l2_prefetch_bulk(wp[r], pf);
   }
   pdl_launch_dependents();
-  pdl_wait();  // x (and its norm statistics) come from the previous kernel
-
-  // ---- prologue: one round trip to L2 for the statistics, x and the gain together
-  float ss = 0.f;
-  if (A.ss_part)
-    for (int i = threadIdx.x; i < A.n_parts; i += nw * 32) ss += A.ss_part[i];
+  // the norm gain is a weight of this block: it is read ahead of the wait, so that afterwards every CTA asks L2 only
+  // for x and the statistics (the same few lines for all CTAs)
   float4 xr[XR], gr[XR];
 #pragma unroll
   for (int j = 0; j < XR; ++j) {
     const int k = (threadIdx.x + j * nw * 32) * 4;
-    if (k < A.K) {
-      xr[j] = *reinterpret_cast<const float4*>(A.x + k);
-      gr[j] = A.gain ? *reinterpret_cast<const float4*>(A.gain + k) : make_float4(1.f, 1.f, 1.f, 1.f);
-    }
+    if (k < A.K) gr[j] = A.gain ? *reinterpret_cast<const float4*>(A.gain + k) : make_float4(1.f, 1.f, 1.f, 1.f);
+  }
+  pdl_wait();  // x (and its norm statistics) come from the previous kernel
+
+  // ---- prologue: one round trip to L2 for the statistics and x
+  float ss = 0.f;
+  if (A.ss_part)
+    for (int i = threadIdx.x; i < A.n_parts; i += nw * 32) ss += A.ss_part[i];
+#pragma unroll
+  for (int j = 0; j < XR; ++j) {
+    const int k = (threadIdx.x + j * nw * 32) * 4;
+    if (k < A.K) xr[j] = *reinterpret_cast<const float4*>(A.x + k);
   }
   float rnorm = 1.f;
   if (A.ss_part) {
