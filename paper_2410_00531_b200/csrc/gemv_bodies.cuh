@@ -192,6 +192,14 @@ __device__ __forceinline__ void cols_body(const GemvArgs& A, float* xs, const in
     int shard, item;
     const uint4* wp[R];
     row_ptrs(it, shard, item, wp);
+    // QKV: the position and this pair's rotation are requested before the weight stream, not after it
+    int p_cur = 0;
+    float2 cs_cur = make_float2(1.f, 0.f);
+    if constexpr (EPI == EPI_QKV) {
+      const int half = A.d >> 1;
+      p_cur = *A.pos;
+      if (item < (A.hps + A.kps) * half) cs_cur = A.rope[(size_t)p_cur * half + (item % half)];
+    }
     float acc[R] = {0.f, 0.f};
     warp_dot<WT, R>(wp, 0, xs, nvec, lane, acc);
 #pragma unroll
@@ -200,12 +208,12 @@ __device__ __forceinline__ void cols_body(const GemvArgs& A, float* xs, const in
       if constexpr (EPI == EPI_QKV) {
         const int half = A.d >> 1;
         const int qp = A.hps * half, kp = A.kps * half;
-        const int p = *A.pos;
+        const int p = p_cur;
         if (item < qp + kp) {
           const bool is_q = item < qp;
           const int t = is_q ? item : item - qp;
           const int hl = t / half, ii = t - hl * half;
-          const float2 cs = A.rope[(size_t)p * half + ii];
+          const float2 cs = cs_cur;
           const float lo_v = acc[0] * cs.x - acc[1] * cs.y;
           const float hi_v = acc[1] * cs.x + acc[0] * cs.y;
           if (is_q) {
