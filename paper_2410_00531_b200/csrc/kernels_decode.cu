@@ -359,7 +359,13 @@ __global__ void __launch_bounds__(lb_threads(WARPS), lb_blocks(WARPS))
   rowfused_body<WT, R, NS, WARPS>(A, xs, blockIdx.x, gridDim.x);
 }
 
-int rowshard_fused_parts(int) { return sm_count() * 4; }
+// Entries of the per-CTA partial sums of squares that producers fill (zeros beyond their grid) and consumers add up:
+// one per SM with the balanced one-CTA-per-SM launch, four per SM when a fixed warp count is forced.  Never more than
+// the 1024 entries the arena plan reserves.
+int rowshard_fused_parts(int) {
+  const int n = g_tune.warps > 0 ? sm_count() * 4 : sm_count();
+  return n > 1024 ? 1024 : n;
+}
 bool rowshard_fused_supported(int Ks, int n_shards) { return (size_t)Ks * n_shards * sizeof(float) <= 200 * 1024; }
 
 template <typename WT, int R, int NS, int WARPS>

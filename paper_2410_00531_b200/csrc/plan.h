@@ -62,6 +62,9 @@ static inline int window_slots(int w, int* nA, int* nF) {
   return *nA + *nF;
 }
 
+// Upper bound of the entries the kernels use for the per-CTA partial sums of squares (4 per SM, up to 256 SMs).
+constexpr size_t kMaxNormParts = 1024;
+
 // Fills `p`; returns the bytes needed in each arena for the given residency mode.
 static inline void make_plan(const tpi_config& c, int n_shards_max, int window_blocks, int keep_host,
                              int head_blocks, Plan* p, size_t* dev_bytes, size_t* host_bytes) {
@@ -84,7 +87,7 @@ static inline void make_plan(const tpi_config& c, int n_shards_max, int window_b
   p->vcache = take(L * p->kv_layer_bytes);
   p->x = take(h * 4);
   p->xhat = take(h * 4);
-  p->ss_part = take(h * 4);
+  p->ss_part = take((h > kMaxNormParts ? h : kMaxNormParts) * 4);  // per-CTA partial sums of x^2: up to kMaxNormParts entries
   p->q = take(a * d * 4);
   p->o = take(a * d * 4);
   p->act = take(s * 4);
