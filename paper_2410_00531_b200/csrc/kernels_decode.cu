@@ -19,7 +19,7 @@ namespace tpi {
 struct Tuning {
   int cps_cols = 4;          // CTAs per SM, column-sharded GEMVs
   int cps_rows = 4;          // CTAs per SM, fused row-sharded GEMVs
-  int prefetch_bytes = 4096; // L2 prefetch per row issued before the dependency wait
+  int prefetch_bytes = 1024; // L2 prefetch per row issued before the dependency wait (more than ~2 KB measured slower)
   int warps = 0;             // 0: one CTA per SM with a balanced warp count; 8, 16, 32: that many warps, cps CTAs per SM
   int mega_prefetch = 2048;  // whole-token kernel: bytes per row requested from L2 ahead of a barrier
 };
