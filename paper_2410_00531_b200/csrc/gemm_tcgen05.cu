@@ -6,105 +6,17 @@
 // with tcgen05.ld and store fp32 rows.  Every wait on an mbarrier is bounded: when a limit runs
 // out the kernel writes DEVERR_WAIT_TIMEOUT to the error word, skips its remaining work, frees its
 // tensor memory and returns.
-#include <cuda.h>
-#include <cuda_bf16.h>
-#include <cuda_runtime.h>
-#include <stdint.h>
+#include <stdlib.h>
 
-#include "kernels.h"
+#include "gemm_tc_common.cuh"
 
 namespace tpi {
 
 namespace {
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+using namespace tc;
 
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: about a quarter of a second at most, then the error word is set.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* err) {
-  for (int i = 0; i < (1 << 21); ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (i > 128) __nanosleep(100);
-  }
-  atomicCAS(err, DEVERR_NONE, DEVERR_WAIT_TIMEOUT);
-  return false;
-}
-
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int x, int y) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y)
-      : "memory");
-}
-
-// K-major operand tile written by TMA with the 128-byte swizzle: rows of 64 bf16 (128 B), groups of
-// 8 rows 1024 B apart.  Descriptor: start address >> 4, leading offset (unused for this layout) 1,
-// stride offset 1024 >> 4, version 1 (sm_100), layout type 2 = 128-byte swizzle.
-__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
-  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
-         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-struct GemmTcArgs {
-  float* Y;
-  long long y_bs;   // floats between batches of Y
-  int ldy, T, n_out, K;
-  int a_col_batch;  // A's column offset per batch (elements)
-  int w_row_batch;  // W's row offset per batch
-  int* err;
-  // SwiGLU epilogue (gate/up projection whose output columns are interleaved gate_j, up_j): when act != nullptr
-  // nothing is written to Y; act[t][c / 2] = silu(y[t][c]) * y[t][c + 1] goes out as bf16 (hi, and in split mode
-  // lo = bf16(v - hi) act_lo_off elements further), row stride act_ld.
-  __nv_bfloat16* act;
-  long long act_lo_off;
-  int act_ld, act_split;
-};
-
-constexpr int kBM = 128, kBK = 64;
+constexpr int kBM = 128;
 // tensor-memory columns are allocated in powers of two
 __host__ __device__ constexpr uint32_t tmem_cols(int bn) { return bn <= 32 ? 32u : bn <= 64 ? 64u : bn <= 128 ? 128u : 256u; }
 // pipeline depth that fits one SM's shared memory
@@ -252,35 +164,6 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)p;
-  }
-  return fn;
-}
-
-// 2-D bf16 tensor [rows][cols] with row stride ld elements; box = 64 columns x box_rows rows, 128B swizzle.
-bool make_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uint64_t ld, uint32_t box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[2] = {cols, rows};
-  const cuuint64_t strides[1] = {ld * 2};
-  const cuuint32_t box[2] = {kBK, box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 bool gemm_tc_supported(int K, int a_cols_total, int ldy) {
@@ -314,6 +197,16 @@ static cudaError_t launch_tc_t(const LaunchCtx& c, const CUtensorMap& tmA, const
   return cudaLaunchKernelEx(&cfg, kern, tmA, tmAlo, tmW, a);
 }
 
+// TPI_GEMM_PAIR=0 in the environment keeps every projection on single-CTA tiles (for comparisons)
+static bool gemm_pair_enabled() {
+  static int on = -1;
+  if (on < 0) {
+    const char* e = getenv("TPI_GEMM_PAIR");
+    on = !(e && e[0] == '0');
+  }
+  return on != 0;
+}
+
 static cudaError_t launch_gemm_tc_any(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
                                       const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T,
                                       int n_out, int K, int n_batch, int* err, void* act, int act_ld, long long act_lo_off,
@@ -325,17 +218,27 @@ static cudaError_t launch_gemm_tc_any(const LaunchCtx& c, const void* A_bf16, co
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&nsm, cudaDevAttrMultiProcessorCount, dev);
   static const int cand[4] = {256, 160, 128, 96};  // 112 (148 CTAs for a 4096-wide output x 4 shards) measured slower than 128
+  static const double tile_us[4] = {0.97, 0.66, 0.55, 0.47};  // measured per tile and k-block at more than 128 positions
   const long long mt = (T + kBM - 1) / kBM;
   int BN = 128;
-  double best = 1e30;
+  double best = 1e30, best_us = 1e30;
   for (int i = 0; i < 4; ++i) {
     const int bn = cand[i];
     if (act && bn % 32) continue;                 // the SwiGLU epilogue works on 32-column groups
     if (bn > 128 && n_out < bn) continue;
     const long long tiles = (long long)((n_out + bn - 1) / bn) * mt * n_batch;
     const long long waves = (tiles + nsm - 1) / nsm;
-    const double cost = (double)waves * ((A_lo_bf16 ? 2 : 1) * kBM * kBK * 2 + bn * kBK * 2);
-    if (cost < best - 1e-9) { best = cost; BN = bn; }
+    // up to 128 positions a CTA's ingest bounds it: bytes per k-block; beyond, the measured tile times
+    const double cost = T <= kBM ? (double)waves * ((A_lo_bf16 ? 2 : 1) * kBM * kBK * 2 + bn * kBK * 2)
+                                 : (double)waves * ((K / kBK) * tile_us[i] + 4.0 + bn / 64.0);
+    if (cost < best - 1e-9) { best = cost; BN = bn; best_us = cost; }
+  }
+  if (A_lo_bf16 && T > kBM && gemm_pair_enabled()) {  // a CTA pair (M = 256) pulls half the weight bytes per MMA
+    double pair_us = 0;
+    const int shape = gemm_tc_pair_choose(T, n_out, K, n_batch, nsm, &pair_us);
+    if (shape >= 0 && pair_us < best_us)
+      return launch_gemm_tc_pair(c, shape, A_bf16, A_lo_bf16, lda, a_col_batch, W_bf16, w_row_batch, Y, y_batch_stride, ldy, T,
+                                 n_out, K, n_batch, err, act, act_ld, act_lo_off, act_split);
   }
   CUtensorMap tmA, tmAlo, tmW;
   // A: [T][lda] (each batch reads K columns starting at batch * a_col_batch); W: [n_batch * w_row_batch][K]

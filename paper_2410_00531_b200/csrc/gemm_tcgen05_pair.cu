@@ -1,0 +1,306 @@
+// Prompt-pass projections on CTA pairs (tcgen05.mma.cta_group::2), for the same contract as gemm_tcgen05.cu:
+//   Y[b][t][o] = sum_k (A_hi + A_lo)[t][b*Ka + k] * W[b*rows_b + o][k]     (bf16 x bf16 -> fp32)
+// The two CTAs of a cluster sit on the two SMs of one TPC and compute ONE tile of 256 positions x BNT outputs:
+// each CTA stages its own 128 positions of the activations and only its own BNT/2 weight rows, and the pair's
+// MMA (M = 256) reads both halves: per MMA every SM pulls half the weight bytes of a single-CTA tile of the same
+// width.  Used for prompts of more than 128 positions, where it measured 5-20 % faster on the wide projections;
+// a pair with M = 128 (64 positions per CTA, half the activation bytes per SM) was also built and measured
+// slower at 128 positions than single-CTA tiles, since 64 rows per SM run the tensor pipe at half rate.
+//
+// Roles per CTA: warp 0 lane 0 issues the TMA loads of its halves (completion bytes are counted on the LEADER's
+// barrier, the CTA with cluster rank 0); warp 1 lane 0 of the leader issues every MMA and releases a stage in both
+// CTAs with tcgen05.commit; warps 2-5 of each CTA read their own accumulator rows back (a CTA's tensor memory
+// holds its 128 positions x N columns).
+// Every mbarrier wait is bounded; nothing here uses multicast.
+#include <stdlib.h>
+
+#include "gemm_tc_common.cuh"
+
+namespace tpi {
+
+namespace {
+
+using namespace tc;
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address of the same shared-memory object in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA tile load into this CTA's shared memory whose completion bytes go to a barrier of either CTA of the pair
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void umma2_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// arrive on a barrier (shared::cluster address, either CTA) once the pair's MMAs issued so far have completed
+__device__ __forceinline__ void umma2_commit(uint32_t bar_cluster_addr) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+__host__ __device__ constexpr uint32_t pow2_cols(int c) { return c <= 32 ? 32u : c <= 64 ? 64u : c <= 128 ? 128u : c <= 256 ? 256u : 512u; }
+constexpr int kMH = 128;  // positions per CTA; the pair's MMA has M = 256
+__host__ __device__ constexpr int pair_stage_bytes(int BNT) { return 2 * kMH * kBK * 2 + (BNT / 2) * kBK * 2; }
+constexpr int pair_stages(int BNT) {
+  const int n = (226 * 1024 - 1024) / pair_stage_bytes(BNT);
+  return n > 8 ? 8 : n;
+}
+
+// 32 accumulator values of one position, output columns col .. col + 31 (col a multiple of 32): plain fp32 stores,
+// or SwiGLU on the (gate, up) pairs -> 16 activations as bf16 hi (+ lo)
+__device__ __forceinline__ void store32(const GemmTcArgs& a, int batch, int row, int col, const uint32_t (&r)[32]) {
+  if (row >= a.T || col >= a.n_out) return;
+  if (a.act) {
+    __nv_bfloat16* arow = a.act + (size_t)row * a.act_ld + (col >> 1);
+    uint32_t hi[8], lo[8];
+#pragma unroll
+    for (int j = 0; j < 32; j += 4) {  // two (gate, up) pairs -> two activations packed in one word
+      float v[2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const float g = __uint_as_float(r[j + 2 * e]), u = __uint_as_float(r[j + 2 * e + 1]);
+        v[e] = g / (1.f + expf(-g)) * u;
+      }
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(v[0]), h1 = __float2bfloat16_rn(v[1]);
+      hi[j >> 2] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+      const __nv_bfloat16 l0 = __float2bfloat16_rn(v[0] - __bfloat162float(h0)), l1 = __float2bfloat16_rn(v[1] - __bfloat162float(h1));
+      lo[j >> 2] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+    }
+    if (col + 32 <= a.n_out) {
+      *reinterpret_cast<uint4*>(arow) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      *reinterpret_cast<uint4*>(arow + 8) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+      if (a.act_split) {
+        *reinterpret_cast<uint4*>(arow + a.act_lo_off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        *reinterpret_cast<uint4*>(arow + a.act_lo_off + 8) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+      }
+    } else {
+      for (int j = 0; j < 16; ++j)
+        if (col + 2 * j + 1 < a.n_out) {
+          arow[j] = __ushort_as_bfloat16((unsigned short)(hi[j >> 1] >> ((j & 1) * 16)));
+          if (a.act_split) arow[a.act_lo_off + j] = __ushort_as_bfloat16((unsigned short)(lo[j >> 1] >> ((j & 1) * 16)));
+        }
+    }
+    return;
+  }
+  float* y = a.Y + (size_t)batch * a.y_bs + (size_t)row * a.ldy + col;
+  if (col + 32 <= a.n_out) {
+#pragma unroll
+    for (int j = 0; j < 32; j += 4)
+      *reinterpret_cast<float4*>(y + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+  } else {
+    for (int j = 0; j < 32; ++j)
+      if (col + j < a.n_out) y[j] = __uint_as_float(r[j]);
+  }
+}
+
+// BNA = N of one MMA of the pair (multiple of 64); NACC accumulators share one activation tile; the pair's tile is
+// 256 positions x BNT = NACC*BNA outputs.  CTA r of the pair loads weight rows n0 + r*BNT/2 + [0, BNT/2);
+// accumulator j multiplies rows [j*BNA/2, (j+1)*BNA/2) of both CTAs' slices, so its output column n is weight row
+// n0 + j*BNA/2 + n of the leader's slice for n < BNA/2 and row n0 + BNT/2 + j*BNA/2 + (n - BNA/2) otherwise.
+template <int BNA, int NACC, int STAGES>
+__global__ void __launch_bounds__(192) gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                           const __grid_constant__ CUtensorMap tmAlo,
+                                                           const __grid_constant__ CUtensorMap tmW, const GemmTcArgs a) {
+  static_assert(BNA % 64 == 0 && BNA <= 256, "each CTA's half of an MMA's width is read back 32 columns at a time");
+  constexpr int BNT = NACC * BNA, HALF = BNA / 2;  // HALF: this CTA's weight rows per accumulator
+  constexpr uint32_t A_BYTES = kMH * kBK * 2, B_BYTES = (BNT / 2) * kBK * 2, STAGE_BYTES = 2 * A_BYTES + B_BYTES;
+  constexpr uint32_t TCOLS = pow2_cols(BNT);
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES], acc_ready;
+  __shared__ uint32_t tmem_base_s;
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();  // 0 = leader
+  const int pair = blockIdx.x >> 1;
+  const int n0 = pair * BNT, m0 = blockIdx.y * 2 * kMH + (int)rank * kMH, batch = blockIdx.z;
+  const int kblocks = a.K / kBK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(&acc_ready, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {  // the same warp of both CTAs allocates the pair's tensor memory
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(TCOLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // both CTAs' barriers exist before either signals the other's
+  tc_fence_after();
+  const uint32_t tmem_acc = tmem_base_s;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  if (warp == 0) {
+    if (lane == 0) {  // ---- TMA producer of this CTA's halves
+      const uint32_t bar0 = map_to_cta(smem_u32(&full[0]), 0);
+      for (int kb = 0; kb < kblocks; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        if (!mbar_wait(&empty[s], ph ^ 1, a.err)) break;
+        uint8_t* sa = smem + (size_t)s * STAGE_BYTES;
+        if (rank == 0) mbar_expect_tx(&full[s], 2 * STAGE_BYTES);  // both CTAs' bytes land on the leader's barrier
+        const uint32_t bar = bar0 + (uint32_t)s * 8;
+        const int kx = batch * a.a_col_batch + kb * kBK;
+        tma_load_2d_pair(sa, &tmA, bar, kx, m0);
+        tma_load_2d_pair(sa + A_BYTES, &tmAlo, bar, kx, m0);
+        tma_load_2d_pair(sa + 2 * A_BYTES, &tmW, bar, kb * kBK, batch * a.w_row_batch + n0 + (int)rank * (BNT / 2));
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {  // ---- the leader issues the pair's MMAs
+      // instruction descriptor: D fp32, A and B bf16, both K-major, N = BNA, M = 256
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BNA >> 3) << 17) | ((uint32_t)((2 * kMH) >> 4) << 24);
+      const uint32_t empty0_peer = map_to_cta(smem_u32(&empty[0]), 1);
+      bool ok = true;
+      for (int kb = 0; kb < kblocks && ok; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        ok = mbar_wait(&full[s], ph, a.err);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
+        const uint64_t dh = umma_desc_sw128(sa), dl = umma_desc_sw128(sa + A_BYTES);
+#pragma unroll
+        for (int j = 0; j < NACC; ++j) {
+          const uint64_t db = umma_desc_sw128(sa + 2 * A_BYTES + (uint32_t)j * HALF * kBK * 2);
+          const uint32_t d = tmem_acc + (uint32_t)(j * BNA);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) umma2_bf16(d, dh + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) umma2_bf16(d, dl + 2 * k, db + 2 * k, idesc, 1u);
+        }
+        umma2_commit(smem_u32(&empty[s]));           // the stage is free in this CTA ...
+        umma2_commit(empty0_peer + (uint32_t)s * 8);  // ... and in the other one
+      }
+      umma2_commit(smem_u32(&acc_ready));
+      umma2_commit(map_to_cta(smem_u32(&acc_ready), 1));
+    }
+  } else {  // ---- epilogue: warps 2..5 cover the four 32-lane quarters of this CTA's tensor memory
+    const int q = warp & 3;
+    const bool ok = mbar_wait(&acc_ready, 0, a.err);
+    tc_fence_after();
+    if (ok && kblocks > 0) {
+      const int row = m0 + q * 32 + lane;
+#pragma unroll 1
+      for (int j = 0; j < NACC; ++j)
+#pragma unroll 1
+        for (int hh = 0; hh < 2; ++hh)
+#pragma unroll 1
+          for (int c = 0; c < HALF; c += 32) {
+            uint32_t r[32];
+            tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(j * BNA + hh * HALF + c), r);
+            store32(a, batch, row, n0 + hh * (BNT / 2) + j * HALF + c, r);
+          }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // neither CTA frees tensor memory or leaves while the other may still use the pair's state
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(TCOLS) : "memory");
+  }
+}
+
+template <int BNA, int NACC>
+cudaError_t launch_pair_t(const LaunchCtx& c, const void* A, const void* Alo, int lda, const void* W, uint64_t w_rows,
+                          const GemmTcArgs& a, int n_batch) {
+  constexpr int BNT = NACC * BNA, STAGES = pair_stages(BNT);
+  CUtensorMap tmA, tmAlo, tmW;
+  if (!make_map(&tmA, A, (uint64_t)lda, (uint64_t)a.T, (uint64_t)lda, kMH)) return cudaErrorInvalidValue;
+  if (!make_map(&tmAlo, Alo, (uint64_t)lda, (uint64_t)a.T, (uint64_t)lda, kMH)) return cudaErrorInvalidValue;
+  if (!make_map(&tmW, W, (uint64_t)a.K, w_rows, (uint64_t)a.K, BNT / 2)) return cudaErrorInvalidValue;
+  auto kern = gemm_tc_pair_kernel<BNA, NACC, STAGES>;
+  const size_t smem = (size_t)STAGES * pair_stage_bytes(BNT) + 1024;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  if (c.launches) ++*c.launches;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(2 * ((a.n_out + BNT - 1) / BNT), (a.T + 2 * kMH - 1) / (2 * kMH), n_batch);
+  cfg.blockDim = dim3(192);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = c.stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.numAttrs = 1;
+  if (c.pdl) {
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 2;
+  }
+  cfg.attrs = attr;
+  return cudaLaunchKernelEx(&cfg, kern, tmA, tmAlo, tmW, a);
+}
+
+struct PairShape { int bna, nacc; };
+constexpr PairShape kShapes[] = {{128, 1}, {192, 1}, {256, 1}, {256, 2}};
+constexpr int kNumShapes = (int)(sizeof(kShapes) / sizeof(kShapes[0]));
+
+}  // namespace
+
+// Predicted time of the best pair shape for this problem, from the measured time one tile takes per 64-wide k-block
+// (0.53 / 0.66 / 0.82 / 1.57 us for the four shapes) plus a fixed cost per tile, times the waves of pairs over the
+// TPCs.  Returns the index into kShapes, or -1 when no pair shape applies (T <= 128).
+int gemm_tc_pair_choose(int T, int n_out, int K, int n_batch, int nsm, double* us_out) {
+  if (T <= kMH) return -1;
+  static const double tile_us[kNumShapes] = {0.53, 0.66, 0.82, 1.57};
+  int best_i = -1;
+  double best = 1e30;
+  const char* force = getenv("TPI_GEMM_PAIR_SHAPE");  // development aid: pin one shape
+  for (int i = 0; i < kNumShapes; ++i) {
+    const int bnt = kShapes[i].bna * kShapes[i].nacc;
+    if (force && atoi(force) != i) continue;
+    if (bnt > 128 && n_out < bnt) continue;
+    const long long pairs = (long long)((n_out + bnt - 1) / bnt) * ((T + 2 * kMH - 1) / (2 * kMH)) * n_batch;
+    const long long waves = (pairs + nsm / 2 - 1) / (nsm / 2);
+    const double us = (double)waves * ((K / kBK) * tile_us[i] + 6.0 + bnt / 64.0);
+    if (us < best - 1e-9) { best = us; best_i = i; }
+  }
+  if (us_out) *us_out = force && best_i >= 0 ? 0 : best;
+  return best_i;
+}
+
+cudaError_t launch_gemm_tc_pair(const LaunchCtx& c, int shape, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
+                                const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T, int n_out,
+                                int K, int n_batch, int* err, void* act, int act_ld, long long act_lo_off, int act_split) {
+  if (shape < 0 || shape >= kNumShapes || !A_lo_bf16) return cudaErrorInvalidValue;
+  const uint64_t w_rows = (uint64_t)(n_batch - 1) * w_row_batch + n_out;
+  GemmTcArgs a{Y, y_batch_stride, ldy, T, n_out, K, a_col_batch, w_row_batch, err, (__nv_bfloat16*)act, act_lo_off, act_ld, act_split};
+  switch (shape) {
+    case 0: return launch_pair_t<128, 1>(c, A_bf16, A_lo_bf16, lda, W_bf16, w_rows, a, n_batch);
+    case 1: return launch_pair_t<192, 1>(c, A_bf16, A_lo_bf16, lda, W_bf16, w_rows, a, n_batch);
+    case 2: return launch_pair_t<256, 1>(c, A_bf16, A_lo_bf16, lda, W_bf16, w_rows, a, n_batch);
+    case 3: return launch_pair_t<256, 2>(c, A_bf16, A_lo_bf16, lda, W_bf16, w_rows, a, n_batch);
+  }
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace tpi

@@ -116,6 +116,13 @@ cudaError_t launch_gemm_tc(const LaunchCtx& c, const void* A_bf16, const void* A
                            int n_out, int K, int n_batch, int* err);
 // Gate/up projection with the SwiGLU of launch_swiglu_rows applied in the epilogue (same arithmetic, same bits):
 // Wgu rows interleaved gate_j, up_j; ACT [T][s] bf16 (out_mode 1) or split bf16 (2: lo at + T*s elements).
+// CTA-pair tiles (tcgen05.mma.cta_group::2) for the same contract, split activations only.  gemm_tc_pair_choose returns
+// the tile shape with the lowest predicted time (us_out), or -1 when none applies (T <= 128); launch_gemm_tc_pair
+// runs that shape (act != nullptr: SwiGLU epilogue as above).
+int gemm_tc_pair_choose(int T, int n_out, int K, int n_batch, int nsm, double* us_out);
+cudaError_t launch_gemm_tc_pair(const LaunchCtx& c, int shape, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
+                                const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T, int n_out,
+                                int K, int n_batch, int* err, void* act, int act_ld, long long act_lo_off, int act_split);
 bool gemm_tc_swiglu_supported(int K, int lda, int s);
 cudaError_t launch_gemm_tc_swiglu(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, const void* Wgu_bf16,
                                   void* ACT, int out_mode, int T, int s, int K, int* err);

@@ -315,6 +315,32 @@ def test_gemm_tensor_core_bf16(T, Tn, K, n_out, nb, split):
     assert rel_l2(got, want) < 2e-5
 
 
+@pytest.mark.parametrize("shape", [0, 1, 2, 3])
+@pytest.mark.parametrize("Tn,K,n_out,nb", [(300, 1024, 1000, 2), (513, 192, 2048, 1)])
+def test_gemm_tensor_core_pair_shapes(T, monkeypatch, shape, Tn, K, n_out, nb):
+    """Every CTA-pair tile shape (M = 256, one or two accumulators) on ragged position and column counts, pinned
+    through the environment, against fp64 on the same bf16 values; tiles past the edge must not write."""
+    import paper_2410_00531_b200.ops as KK
+    monkeypatch.setenv("TPI_GEMM_PAIR_SHAPE", str(shape))
+    rng = np.random.default_rng(Tn + K + shape)
+    A32 = rng.standard_normal((Tn, nb * K)).astype(np.float32)
+    A = S.f32_to_bf16_bits(A32).reshape(Tn, nb * K)
+    Alo = S.f32_to_bf16_bits(A32 - S.bf16_bits_to_f32(A).reshape(A32.shape)).reshape(Tn, nb * K)
+    W = S.f32_to_bf16_bits((rng.standard_normal((nb, n_out, K)) * 0.02).astype(np.float32)).reshape(nb, n_out, K)
+    Y = T.full((nb * Tn * n_out + 4096,), 7.0, dtype=T.float32, device="cuda")
+    err = T.zeros(1, dtype=T.int32, device="cuda")
+    KK.gemm_bf16(dev(T, A).data_ptr(), nb * K, K, dev(T, W).data_ptr(), n_out, Y.data_ptr(), Tn * n_out, n_out,
+                 Tn, n_out, K, nb, err.data_ptr(), A_lo=dev(T, Alo).data_ptr())
+    T.cuda.synchronize()
+    assert int(err[0]) == 0
+    A64 = S.as_f64(A) + S.as_f64(Alo)
+    W64 = S.as_f64(W)
+    want = np.stack([A64[:, b * K:(b + 1) * K] @ W64[b].T for b in range(nb)])
+    got = Y.cpu().numpy()
+    assert (got[nb * Tn * n_out:] == 7.0).all()
+    assert rel_l2(got[:nb * Tn * n_out].reshape(nb, Tn, n_out), want) < 2e-5
+
+
 @pytest.mark.parametrize("Tn,K,s", [(128, 4096, 11008), (70, 1024, 1360), (300, 512, 48)])
 @pytest.mark.parametrize("split_out", [False, True])
 def test_gemm_tensor_core_swiglu_epilogue(T, Tn, K, s, split_out):
