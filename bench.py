@@ -211,7 +211,7 @@ def run_gpu(args, shape):
     torch.cuda.set_device(local)
     K, W, T = args.steps, args.warmup, shape.prompt_len
     max_seq = T + W + K + 8 + (K + 8 if args.window > 0 else 0)   # the streamed leg also decodes its e2e and diagnostic tokens
-    cfg = tpi_config(shape, max_seq, min(T, 512))
+    cfg = tpi_config(shape, max_seq, min(T, args.prefill_chunk))
     t_load = time.perf_counter()
     extra = 0
     if args.window > 0 and args.retain > 0:      # room for the kept FFN blocks beside the window (Prop. 6)
@@ -429,6 +429,7 @@ def main():
                     help="stream the layer blocks through a window of this many blocks (0 = all resident)")
     ap.add_argument("--prompt", type=int, default=0, help="override the prompt length")
     ap.add_argument("--shards", type=int, default=0, help="override the number of emulated shards N")
+    ap.add_argument("--prefill-chunk", type=int, default=4096, help="prompt positions processed per pass over the weights")
     ap.add_argument("--quick", action="store_true",
                     help="one prompt pass and the device-resident decode loop only (short runs under a profiler)")
     ap.add_argument("--layers", type=int, default=0, help="override the depth (small captures under a profiler)")
