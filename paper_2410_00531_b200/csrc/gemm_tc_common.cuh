@@ -37,7 +37,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* e
     if (mbar_try_wait(bar, parity)) return true;
     if (i > 128) __nanosleep(100);
   }
-  atomicCAS(err, DEVERR_NONE, DEVERR_WAIT_TIMEOUT);
+  if (err) atomicCAS(err, DEVERR_NONE, DEVERR_WAIT_TIMEOUT);
   return false;
 }
 

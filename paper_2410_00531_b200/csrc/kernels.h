@@ -139,6 +139,11 @@ bool prefill_attention_mma_supported(int dt, int d);
 cudaError_t launch_prefill_attention_mma(const LaunchCtx& c, const float* Q, const void* kcache_layer,
                                          const void* vcache_layer, int T, int pos0, int a, int b, int d, int max_seq,
                                          void* O, int out_mode);
+// The same on tcgen05 (head dimension 128, bf16 cache, at least 256 positions): 128 queries x 128 keys per step, S and
+// O in tensor memory.  err: device error word for the bounded waits (may be null).
+bool prefill_attention_tc_supported(int dt, int d, int T);
+cudaError_t launch_prefill_attention_tc(const LaunchCtx& c, const float* Q, const void* kcache_layer, const void* vcache_layer,
+                                        int T, int pos0, int a, int b, int max_seq, void* O, int out_mode, int* err);
 // act[t][j] = silu(GU[t][2j]) * GU[t][2j+1] per shard-major interleaved rows
 cudaError_t launch_swiglu_rows(const LaunchCtx& c, const float* GU, int T, int s, void* ACT, int out_bf16);
 // X[t] <- sum_i P_i[t] + X[t]; optional tap of the last row

@@ -137,7 +137,9 @@ extern "C" int tpi_op_prefill_attention(int dtype, const float* Q, const void* k
                                         int pos0, int a, int b, int d, int max_seq, float* O, void* stream) {
   if (bad_dtype(dtype) || !Q || !kcache || !vcache || !O || T < 1 || pos0 < 0) return TPI_ERR_INVALID_ARG;
   if (a % b) return TPI_ERR_SHAPE;
-  const cudaError_t e = prefill_attention_mma_supported(dtype, d)
+  const cudaError_t e = prefill_attention_tc_supported(dtype, d, T)
+                            ? launch_prefill_attention_tc(ctx(stream), Q, kcache, vcache, T, pos0, a, b, max_seq, O, 0, nullptr)
+                        : prefill_attention_mma_supported(dtype, d)
                             ? launch_prefill_attention_mma(ctx(stream), Q, kcache, vcache, T, pos0, a, b, d, max_seq, O, 0)
                             : launch_prefill_attention(ctx(stream), dtype, Q, kcache, vcache, T, pos0, a, b, d, max_seq, O, 0);
   return e == cudaErrorInvalidValue ? TPI_ERR_SHAPE : cu(e);

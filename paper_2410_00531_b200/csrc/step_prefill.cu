@@ -73,7 +73,9 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
     if (!normed) CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, act_mode));
     TRY(proj(Xn, h, 0, br.base + bl.off_qkv, qkv_cols, QKV, 0, qkv_cols, qkv_cols, h, 1));
     CK(launch_rope_kv_rows(lc, dt, QKV, T, pos0, Nc, a, b, d, c.max_seq, rope, Q, kc, vc));
-    if (m->opt_tensor && prefill_attention_mma_supported(dt, d))
+    if (m->opt_tensor && prefill_attention_tc_supported(dt, d, T))
+      CK(launch_prefill_attention_tc(lc, Q, kc, vc, T, pos0, a, b, c.max_seq, O, act_mode, err));
+    else if (m->opt_tensor && prefill_attention_mma_supported(dt, d))
       CK(launch_prefill_attention_mma(lc, Q, kc, vc, T, pos0, a, b, d, c.max_seq, O, act_mode));
     else
       CK(launch_prefill_attention(lc, dt, Q, kc, vc, T, pos0, a, b, d, c.max_seq, O, act_mode));

@@ -239,7 +239,8 @@ def test_gemm_batched_ragged(T, dtype):
 
 @pytest.mark.parametrize("dtype,a,b,d,Tq,pos0", [("f32", 4, 4, 64, 16, 0), ("bf16", 8, 2, 128, 37, 20), ("bf16", 8, 1, 32, 5, 0),
                                                     ("bf16", 4, 4, 128, 200, 0), ("bf16", 8, 2, 64, 130, 77), ("bf16", 2, 1, 128, 64, 64),
-                                                    ("bf16", 4, 2, 128, 1, 300)])
+                                                    ("bf16", 4, 2, 128, 1, 300), ("bf16", 8, 2, 128, 300, 77),
+                                                    ("bf16", 2, 1, 128, 513, 0), ("bf16", 2, 2, 128, 257, 1000)])
 def test_prefill_attention(T, dtype, a, b, d, Tq, pos0):
     import paper_2410_00531_b200.ops as K
     n = pos0 + Tq
@@ -250,6 +251,7 @@ def test_prefill_attention(T, dtype, a, b, d, Tq, pos0):
     q = S.kv_contents(33, (Tq, a, d))
     tt = T.bfloat16 if dtype == "bf16" else T.float32
     kc, vc = T.from_numpy(k).cuda().to(tt), T.from_numpy(v).cuda().to(tt)
+    kc[:, n:], vc[:, n:] = float("nan"), float("nan")                # nothing past the newest position may be read
     o = T.empty((Tq, a, d), dtype=T.float32, device="cuda")
     K.prefill_attention(1 if dtype == "bf16" else 0, dev(T, q).data_ptr(), kc.data_ptr(), vc.data_ptr(), Tq, pos0, a, b, d,
                         max_seq, o.data_ptr())
