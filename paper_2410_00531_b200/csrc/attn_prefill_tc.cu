@@ -1,15 +1,17 @@
 // Causal attention of the prompt pass on the 5th-generation tensor cores (bf16 KV cache, head dimension 128):
 // Eq. 1's softmax(QK^T/sqrt d)V for T query positions at once.  One CTA = 128 queries of one head; keys are walked
 // in tiles of 128.  Per tile: S = Q K^T (tcgen05.mma, fp32 in tensor memory), an online softmax by 4 warps in
-// which every thread owns one query row (no shuffles), the weights P written to shared memory as an MMA operand,
-// and O += P V (tcgen05.mma, V read in place as an MN-major operand) accumulated in tensor memory.
+// which every thread owns one query row (no shuffles), the weights P written back over S in tensor memory as packed
+// bf16 (the MMA's A operand is read from there), and O += P V (tcgen05.mma, V read in place as an MN-major operand)
+// accumulated in tensor memory.
 //   * K and V tiles come straight from the cache by TMA (128B swizzle; rows past the last valid position are
 //     zero-filled by the tensor map's bounds, so nothing beyond position pos0 + T - 1 is read).
 //   * The fp32 queries and the softmax weights are split into bf16 hi + lo and multiplied twice (K and V are exact
 //     bf16, the cache's storage type), as in the mma.sync kernel this replaces for long prompts.
-//   * S is double-buffered in tensor memory, so S of tile k+1 is computed while the softmax of tile k runs; O is
-//     rescaled only when a row's maximum has grown by more than 2^8 since the reference in use (the final 1/l
-//     normalisation makes a stale reference exact).
+//   * S / P is double-buffered in tensor memory: S of tile k+1 is computed and O += P V of tile k-1 runs while the
+//     softmax of tile k works.  O is rescaled only when a row's maximum has grown by more than 2^8 since the
+//     reference in use (the final 1/l normalisation makes a stale reference exact), and only then does the softmax
+//     wait for the previous tile's P V.
 // Roles: warp 0 lane 0 TMA producer, warp 1 lane 0 MMA issuer, warps 2-5 softmax and epilogue.  Every mbarrier
 // wait is bounded; a role that gives up leaves its loop, the others follow at their next wait, and the error word
 // is set.
@@ -26,8 +28,7 @@ using namespace tc;
 constexpr int AD = 128;          // head dimension
 constexpr int AQ = 128, AK = 128;  // queries per CTA, keys per tile
 constexpr uint32_t BLK = AQ * 64 * 2;    // one [128 rows][64 elements] bf16 block, 128B-swizzled: 16 KB
-constexpr uint32_t OFF_QH = 0, OFF_QL = 2 * BLK, OFF_K0 = 4 * BLK, OFF_K1 = 6 * BLK, OFF_V = 8 * BLK, OFF_PH = 10 * BLK,
-                   OFF_PL = 12 * BLK, ATT_SMEM = 14 * BLK;  // 224 KB
+constexpr uint32_t OFF_QH = 0, OFF_QL = 2 * BLK, OFF_K = 4 * BLK, OFF_V = 8 * BLK, ATT_SMEM = 12 * BLK;  // 192 KB: Q, 2 x K, 2 x V
 constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_O = 256, TM_COLS = 512;
 
 __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, uint64_t* bar, int x, int y, int z) {
@@ -38,6 +39,14 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(  // A operand from tensor memory (row = lane, two bf16 per column), B from shared memory
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(
@@ -108,7 +117,7 @@ __global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_const
                                                               const float* __restrict__ Q, int T, int pos0, int a, int b,
                                                               void* O, size_t lo_off, int* err) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t k_full[2], k_empty[2], v_full, v_empty, s_ready[2], s_free[2], p_ready, pv_done;
+  __shared__ __align__(8) uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2], s_ready[2], p_ready, pv_done;
   __shared__ uint32_t tmem_base_s;
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -119,8 +128,10 @@ __global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_const
   const int n_tiles = (n_keys + AK - 1) / AK;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 2; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); mbar_init(&s_ready[i], 1); mbar_init(&s_free[i], 4); }
-    mbar_init(&v_full, 1); mbar_init(&v_empty, 1); mbar_init(&p_ready, 4); mbar_init(&pv_done, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1); mbar_init(&s_ready[i], 1);
+    }
+    mbar_init(&p_ready, 4); mbar_init(&pv_done, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -158,18 +169,20 @@ __global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_const
   const bool live = err == nullptr || *reinterpret_cast<volatile int*>(err) == DEVERR_NONE;  // an earlier CTA gave up: skip
 
   if (warp == 0) {
-    if (lane == 0 && live) {  // ---- TMA producer: K tile kt into buffer kt & 1, V tile kt into the single V buffer
+    if (lane == 0 && live) {  // ---- TMA producer: K and V tiles kt into their buffers kt & 1
       for (int kt = 0; kt < n_tiles; ++kt) {
         const int bi = kt & 1;
-        if (!mbar_wait(&k_empty[bi], ((kt >> 1) & 1) ^ 1, err)) break;
-        uint8_t* kd = smem + (bi ? OFF_K1 : OFF_K0);
+        const uint32_t ph = (kt >> 1) & 1;
+        if (!mbar_wait(&k_empty[bi], ph ^ 1, err)) break;
+        uint8_t* kd = smem + OFF_K + bi * 2 * BLK;
         mbar_expect_tx(&k_full[bi], 2 * BLK);
         tma_load_3d(kd, &tmK, &k_full[bi], 0, kt * AK, kvh);
         tma_load_3d(kd + BLK, &tmK, &k_full[bi], 64, kt * AK, kvh);
-        if (!mbar_wait(&v_empty, (kt & 1) ^ 1, err)) break;
-        mbar_expect_tx(&v_full, 2 * BLK);
-        tma_load_3d(smem + OFF_V, &tmV, &v_full, 0, kt * AK, kvh);
-        tma_load_3d(smem + OFF_V + BLK, &tmV, &v_full, 64, kt * AK, kvh);
+        if (!mbar_wait(&v_empty[bi], ph ^ 1, err)) break;
+        uint8_t* vd = smem + OFF_V + bi * 2 * BLK;
+        mbar_expect_tx(&v_full[bi], 2 * BLK);
+        tma_load_3d(vd, &tmV, &v_full[bi], 0, kt * AK, kvh);
+        tma_load_3d(vd + BLK, &tmV, &v_full[bi], 64, kt * AK, kvh);
       }
     }
   } else if (warp == 1) {
@@ -178,12 +191,11 @@ __global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_const
       constexpr uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(AK >> 3) << 17) | ((uint32_t)(AQ >> 4) << 24);
       constexpr uint32_t idesc_o = idesc_s | (1u << 16);
       const uint32_t sb = smem_u32(smem);
-      auto issue_s = [&](int kt) -> bool {  // S(kt) = Q K(kt)^T into S buffer kt & 1
+      auto issue_s = [&](int kt) -> bool {  // S(kt) = Q K(kt)^T into S buffer kt & 1 (free: P V of tile kt - 2 is complete)
         const int bi = kt & 1;
         if (!mbar_wait(&k_full[bi], (kt >> 1) & 1, err)) return false;
-        if (!mbar_wait(&s_free[bi], ((kt >> 1) & 1) ^ 1, err)) return false;
         tc_fence_after();
-        const uint32_t kb = sb + (bi ? OFF_K1 : OFF_K0), d = tmem + (bi ? TM_S1 : TM_S0);
+        const uint32_t kb = sb + OFF_K + (uint32_t)bi * 2 * BLK, d = tmem + (bi ? TM_S1 : TM_S0);
 #pragma unroll
         for (int ks = 0; ks < AD / 16; ++ks) {
           const uint32_t o = (uint32_t)(ks >> 2) * BLK;
@@ -196,21 +208,25 @@ __global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_const
         return true;
       };
       bool ok = n_tiles > 0 && issue_s(0);
+      if (ok && n_tiles > 1) ok = issue_s(1);
       for (int kt = 0; kt < n_tiles && ok; ++kt) {
-        if (kt + 1 < n_tiles) ok = issue_s(kt + 1);
-        if (!ok) break;
-        ok = mbar_wait(&p_ready, kt & 1, err) && mbar_wait(&v_full, kt & 1, err);
+        const int bi = kt & 1;
+        ok = mbar_wait(&p_ready, kt & 1, err) && mbar_wait(&v_full[bi], (kt >> 1) & 1, err);
         if (!ok) break;
         tc_fence_after();
+        const uint32_t pa = tmem + (bi ? TM_S1 : TM_S0), vb = sb + OFF_V + (uint32_t)bi * 2 * BLK;
 #pragma unroll
-        for (int ks = 0; ks < AK / 16; ++ks) {  // 16 keys per step: two 8-key groups of the V tile
-          const uint32_t o = (uint32_t)(ks >> 2) * BLK;
-          const uint64_t dv = umma_desc_sw128_mn(sb + OFF_V + (uint32_t)ks * 2048);
-          umma_bf16(tmem + TM_O, umma_desc_sw128(sb + OFF_PH + o) + 2 * (ks & 3), dv, idesc_o, (kt | ks) ? 1u : 0u);
-          umma_bf16(tmem + TM_O, umma_desc_sw128(sb + OFF_PL + o) + 2 * (ks & 3), dv, idesc_o, 1u);
+        for (int ks = 0; ks < AK / 16; ++ks) {  // 16 keys per step: 8 columns of P (hi, then lo 16 columns on), two 8-key groups of V
+          const uint64_t dv = umma_desc_sw128_mn(vb + (uint32_t)ks * 2048);
+          const uint32_t pc = pa + (uint32_t)((ks >> 1) * 32 + (ks & 1) * 8);
+          umma_bf16_ta(tmem + TM_O, pc, dv, idesc_o, (kt | ks) ? 1u : 0u);
+          umma_bf16_ta(tmem + TM_O, pc + 16, dv, idesc_o, 1u);
         }
         umma_commit(&pv_done);
-        umma_commit(&v_empty);
+        umma_commit(&v_empty[bi]);
+        if (kt + 2 < n_tiles) {  // the S / P buffer of tile kt is rewritten only after its P V has completed
+          ok = mbar_wait(&pv_done, kt & 1, err) && issue_s(kt + 2);
+        }
       }
     }
   } else if (live) {  // ---- softmax and epilogue: thread = query row, warp q covers tensor-memory lanes 32q..32q+31
@@ -218,7 +234,6 @@ __global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_const
     const uint32_t lane_sel = (uint32_t)(q * 32) << 16;
     const int qpos = pos0 + q0 + r;
     float m_ref = -INFINITY, l = 0.f;
-    const uint32_t prow = (uint32_t)r * 128;  // this row's 128 bytes inside a 64-key block of P
     bool ok = true;
     for (int kt = 0; kt < n_tiles && ok; ++kt) {
       const int bi = kt & 1, k0 = kt * AK;
@@ -249,49 +264,41 @@ __global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_const
       }
       // the reference moves only when the row's maximum outgrew it by more than 2^8 (always on the first tile)
       const bool need = mx > m_ref + 8.f;
-      const bool any = __any_sync(0xFFFFFFFFu, need);
-      if (kt > 0) {
-        ok = mbar_wait(&pv_done, (kt - 1) & 1, err);  // O holds tiles 0..kt-1 and the P buffer is free again
+      if (kt > 0 && __any_sync(0xFFFFFFFFu, need)) {
+        ok = mbar_wait(&pv_done, (kt - 1) & 1, err);  // O holds tiles 0..kt-1 and nothing is adding to it
         if (!ok) break;
         tc_fence_after();
-        if (any) {
-          const float alpha = need ? ex2(m_ref - mx) : 1.f;
+        const float alpha = need ? ex2(m_ref - mx) : 1.f;
 #pragma unroll 1
-          for (int c = 0; c < AD; c += 32) {
-            uint32_t o[32];
-            tmem_ld32(tmem + lane_sel + TM_O + (uint32_t)c, o);
+        for (int c = 0; c < AD; c += 32) {
+          uint32_t o[32];
+          tmem_ld32(tmem + lane_sel + TM_O + (uint32_t)c, o);
 #pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st32(tmem + lane_sel + TM_O + (uint32_t)c, o);
-          }
-          l *= alpha;
+          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+          tmem_st32(tmem + lane_sel + TM_O + (uint32_t)c, o);
         }
+        l *= alpha;
       }
       if (need) m_ref = mx;
 #pragma unroll 1
-      for (int c = 0; c < AK; c += 32) {
-        uint32_t s[32];
+      for (int c = 0; c < AK; c += 32) {  // 32 scores -> 16 columns of packed P_hi and 16 of P_lo, in place
+        uint32_t s[32], pk[32];
         tmem_ld32(ts + (uint32_t)c, s);
 #pragma unroll
-        for (int g8 = 0; g8 < 4; ++g8) {
-          float p[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            p[e] = ex2(__uint_as_float(s[g8 * 8 + e]) - m_ref);
-            if (!full && k0 + c + g8 * 8 + e > qpos) p[e] = 0.f;
+        for (int e = 0; e < 32; e += 2) {
+          float p0 = ex2(__uint_as_float(s[e]) - m_ref), p1 = ex2(__uint_as_float(s[e + 1]) - m_ref);
+          if (!full) {
+            if (k0 + c + e > qpos) p0 = 0.f;
+            if (k0 + c + e + 1 > qpos) p1 = 0.f;
           }
-          l += ((p[0] + p[1]) + (p[2] + p[3])) + ((p[4] + p[5]) + (p[6] + p[7]));
-          uint4 hi, lo;
-          split8(p, hi, lo);
-          const uint32_t off = prow + (uint32_t)(c >> 6) * BLK + (uint32_t)(((((c >> 3) + g8) & 7) ^ (r & 7)) << 4);
-          *reinterpret_cast<uint4*>(smem + OFF_PH + off) = hi;
-          *reinterpret_cast<uint4*>(smem + OFF_PL + off) = lo;
+          l += p0 + p1;
+          split2(p0, p1, pk[e >> 1], pk[16 + (e >> 1)]);
         }
+        tmem_st32(ts + (uint32_t)c, pk);
       }
-      tc_fence_before();                                           // this thread's reads of S and writes of O are done
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // P becomes visible to the tensor core
+      tc_fence_before();  // this thread's reads of S and writes of P and O are done
       __syncwarp();
-      if (lane == 0) { mbar_arrive(&s_free[bi]); mbar_arrive(&p_ready); }
+      if (lane == 0) mbar_arrive(&p_ready);
     }
     if (ok && n_tiles > 0) ok = mbar_wait(&pv_done, (n_tiles - 1) & 1, err);
     if (ok && n_tiles > 0) {
