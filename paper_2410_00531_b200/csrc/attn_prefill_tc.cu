@@ -8,11 +8,13 @@
 //     zero-filled by the tensor map's bounds, so nothing beyond position pos0 + T - 1 is read).
 //   * The fp32 queries and the softmax weights are split into bf16 hi + lo and multiplied twice (K and V are exact
 //     bf16, the cache's storage type), as in the mma.sync kernel this replaces for long prompts.
-//   * S / P is double-buffered in tensor memory: S of tile k+1 is computed and O += P V of tile k-1 runs while the
-//     softmax of tile k works.  O is rescaled only when a row's maximum has grown by more than 2^8 since the
-//     reference in use (the final 1/l normalisation makes a stale reference exact), and only then does the softmax
-//     wait for the previous tile's P V.
-// Roles: warp 0 lane 0 TMA producer, warp 1 lane 0 MMA issuer, warps 2-5 softmax and epilogue.  Every mbarrier
+//   * Two softmax streams: warps 2-5 take the even key tiles (S / P buffer 0, accumulator O_0), warps 6-9 the odd
+//     ones (buffer 1, O_1), each with its own running reference and sum; one warp per SM sub-partition cannot issue
+//     the softmax of a tile as fast as the tensor core multiplies it, two can.  The epilogue merges the two
+//     streams (weights 2^(m - M)), so tensor memory holds S_0, S_1, O_0, O_1 = 512 columns.
+//   * O is rescaled only when a row's maximum has grown by more than 2^8 since the reference in use (the final
+//     1/l normalisation makes a stale reference exact), and only then does a stream wait for its previous P V.
+// Roles: warp 0 lane 0 TMA producer, warp 1 lane 0 MMA issuer, warps 2-9 softmax and epilogue.  Every mbarrier
 // wait is bounded; a role that gives up leaves its loop, the others follow at their next wait, and the error word
 // is set.
 #include <stdlib.h>
@@ -29,7 +31,8 @@ constexpr int AD = 128;          // head dimension
 constexpr int AQ = 128, AK = 128;  // queries per CTA, keys per tile
 constexpr uint32_t BLK = AQ * 64 * 2;    // one [128 rows][64 elements] bf16 block, 128B-swizzled: 16 KB
 constexpr uint32_t OFF_QH = 0, OFF_QL = 2 * BLK, OFF_K = 4 * BLK, OFF_V = 8 * BLK, ATT_SMEM = 12 * BLK;  // 192 KB: Q, 2 x K, 2 x V
-constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_O = 256, TM_COLS = 512;
+constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_O = 256, TM_COLS = 512;  // O_0 at TM_O, O_1 at TM_O + 128
+constexpr int ATT_THREADS = 320;
 
 __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, uint64_t* bar, int x, int y, int z) {
   asm volatile(
@@ -112,12 +115,13 @@ __device__ __forceinline__ void store_row32(void* base, size_t i, size_t lo_off,
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK,
+__global__ void __launch_bounds__(ATT_THREADS) prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                               const __grid_constant__ CUtensorMap tmV,
                                                               const float* __restrict__ Q, int T, int pos0, int a, int b,
                                                               void* O, size_t lo_off, int* err) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2], s_ready[2], p_ready, pv_done;
+  __shared__ __align__(8) uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2], s_ready[2], p_ready[2], pv_done[2];
+  __shared__ float st_m[2][AQ], st_l[2][AQ];  // the two streams' final reference and sum per row
   __shared__ uint32_t tmem_base_s;
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -130,8 +134,8 @@ __global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_const
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1); mbar_init(&s_ready[i], 1);
+      mbar_init(&p_ready[i], 4); mbar_init(&pv_done[i], 1);
     }
-    mbar_init(&p_ready, 4); mbar_init(&pv_done, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -143,7 +147,7 @@ __global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_const
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (warp >= 2) {  // stage the CTA's queries: scaled into the log2 domain, split hi / lo, in MMA operand layout
     const float qscale = 1.4426950408889634f * rsqrtf((float)AD);
-    for (int i = threadIdx.x - 64; i < AQ * 16; i += 128) {
+    for (int i = threadIdx.x - 64; i < AQ * 16; i += ATT_THREADS - 64) {
       const int r = i >> 4, c8 = i & 15;
       float v[8];
       if (q0 + r < T) {
@@ -211,7 +215,7 @@ __global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_const
       if (ok && n_tiles > 1) ok = issue_s(1);
       for (int kt = 0; kt < n_tiles && ok; ++kt) {
         const int bi = kt & 1;
-        ok = mbar_wait(&p_ready, kt & 1, err) && mbar_wait(&v_full[bi], (kt >> 1) & 1, err);
+        ok = mbar_wait(&p_ready[bi], (kt >> 1) & 1, err) && mbar_wait(&v_full[bi], (kt >> 1) & 1, err);
         if (!ok) break;
         tc_fence_after();
         const uint32_t pa = tmem + (bi ? TM_S1 : TM_S0), vb = sb + OFF_V + (uint32_t)bi * 2 * BLK;
@@ -219,26 +223,28 @@ __global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_const
         for (int ks = 0; ks < AK / 16; ++ks) {  // 16 keys per step: 8 columns of P (hi, then lo 16 columns on), two 8-key groups of V
           const uint64_t dv = umma_desc_sw128_mn(vb + (uint32_t)ks * 2048);
           const uint32_t pc = pa + (uint32_t)((ks >> 1) * 32 + (ks & 1) * 8);
-          umma_bf16_ta(tmem + TM_O, pc, dv, idesc_o, (kt | ks) ? 1u : 0u);
-          umma_bf16_ta(tmem + TM_O, pc + 16, dv, idesc_o, 1u);
+          umma_bf16_ta(tmem + TM_O + (uint32_t)bi * 128, pc, dv, idesc_o, ((kt >> 1) | ks) ? 1u : 0u);
+          umma_bf16_ta(tmem + TM_O + (uint32_t)bi * 128, pc + 16, dv, idesc_o, 1u);
         }
-        umma_commit(&pv_done);
+        umma_commit(&pv_done[bi]);
         umma_commit(&v_empty[bi]);
         if (kt + 2 < n_tiles) {  // the S / P buffer of tile kt is rewritten only after its P V has completed
-          ok = mbar_wait(&pv_done, kt & 1, err) && issue_s(kt + 2);
+          ok = mbar_wait(&pv_done[bi], (kt >> 1) & 1, err) && issue_s(kt + 2);
         }
       }
     }
-  } else if (live) {  // ---- softmax and epilogue: thread = query row, warp q covers tensor-memory lanes 32q..32q+31
+  } else {  // ---- softmax and epilogue: thread = query row, warp q covers tensor-memory lanes 32q..32q+31
+    const int strm = warp >= 6 ? 1 : 0;  // stream 0: even key tiles, stream 1: odd key tiles
     const int q = warp & 3, r = q * 32 + lane;
     const uint32_t lane_sel = (uint32_t)(q * 32) << 16;
     const int qpos = pos0 + q0 + r;
+    const uint32_t ts = tmem + lane_sel + (strm ? TM_S1 : TM_S0), to = tmem + lane_sel + TM_O + (uint32_t)strm * 128;
     float m_ref = -INFINITY, l = 0.f;
-    bool ok = true;
-    for (int kt = 0; kt < n_tiles && ok; ++kt) {
-      const int bi = kt & 1, k0 = kt * AK;
-      const uint32_t ts = tmem + lane_sel + (bi ? TM_S1 : TM_S0);
-      ok = mbar_wait(&s_ready[bi], (kt >> 1) & 1, err);
+    bool ok = live;
+    for (int kt = strm; kt < n_tiles && ok; kt += 2) {
+      const int k0 = kt * AK;
+      const uint32_t ph = (kt >> 1) & 1;
+      ok = mbar_wait(&s_ready[strm], ph, err);
       if (!ok) break;
       tc_fence_after();
       // tiles left of the diagonal are visible to every row of the warp: no masking there
@@ -262,20 +268,21 @@ __global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_const
             if (k0 + c + e <= qpos) mx = fmaxf(mx, __uint_as_float(s[e]));
         }
       }
-      // the reference moves only when the row's maximum outgrew it by more than 2^8 (always on the first tile)
+      // the reference moves only when the row's maximum outgrew it by more than 2^8 (always on a stream's first tile
+      // that shows the row a key; a row that sees none keeps -inf and weights 0)
       const bool need = mx > m_ref + 8.f;
-      if (kt > 0 && __any_sync(0xFFFFFFFFu, need)) {
-        ok = mbar_wait(&pv_done, (kt - 1) & 1, err);  // O holds tiles 0..kt-1 and nothing is adding to it
+      if (kt >= 2 && __any_sync(0xFFFFFFFFu, need)) {
+        ok = mbar_wait(&pv_done[strm], ph ^ 1, err);  // O holds the stream's earlier tiles and nothing is adding to it
         if (!ok) break;
         tc_fence_after();
-        const float alpha = need ? ex2(m_ref - mx) : 1.f;
+        const float alpha = need ? ex2(m_ref - mx) : 1.f;  // m_ref = -inf: the row has added nothing yet, alpha = 0
 #pragma unroll 1
         for (int c = 0; c < AD; c += 32) {
           uint32_t o[32];
-          tmem_ld32(tmem + lane_sel + TM_O + (uint32_t)c, o);
+          tmem_ld32(to + (uint32_t)c, o);
 #pragma unroll
           for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-          tmem_st32(tmem + lane_sel + TM_O + (uint32_t)c, o);
+          tmem_st32(to + (uint32_t)c, o);
         }
         l *= alpha;
       }
@@ -298,20 +305,37 @@ __global__ void __launch_bounds__(192) prefill_attn_tc_kernel(const __grid_const
       }
       tc_fence_before();  // this thread's reads of S and writes of P and O are done
       __syncwarp();
-      if (lane == 0) mbar_arrive(&p_ready);
+      if (lane == 0) mbar_arrive(&p_ready[strm]);
     }
-    if (ok && n_tiles > 0) ok = mbar_wait(&pv_done, (n_tiles - 1) & 1, err);
-    if (ok && n_tiles > 0) {
-      tc_fence_after();
-      const float inv = 1.f / l;
+    // ---- merge the two streams and store: each stream's warp takes half of the output columns of its rows
+    const int my_tiles = (n_tiles - strm + 1) / 2;  // key tiles this stream has seen
+    if (ok && my_tiles > 0) ok = mbar_wait(&pv_done[strm], (my_tiles - 1) & 1, err);
+    st_m[strm][r] = m_ref;
+    st_l[strm][r] = l;
+    tc_fence_before();
+    asm volatile("bar.sync 1, 256;" ::: "memory");  // the 8 softmax warps (every one of them reaches this point)
+    tc_fence_after();
+    if (ok && n_tiles > 0 && (err == nullptr || *reinterpret_cast<volatile int*>(err) == DEVERR_NONE)) {
+      const bool two = n_tiles > 1;
+      const float m0 = st_m[0][r], m1 = two ? st_m[1][r] : -INFINITY;
+      const float M = fmaxf(m0, m1);
+      const float w0 = ex2(m0 - M), w1 = two ? ex2(m1 - M) : 0.f;  // a stream whose rows saw no key has m = -inf, weight 0
+      const float inv = 1.f / (st_l[0][r] * w0 + (two ? st_l[1][r] * w1 : 0.f));
+      const float f0 = w0 * inv, f1 = w1 * inv;
       const int row = q0 + r;
 #pragma unroll 1
-      for (int c = 0; c < AD; c += 32) {
-        uint32_t o[32];
-        tmem_ld32(tmem + lane_sel + TM_O + (uint32_t)c, o);
+      for (int c = strm * 64; c < strm * 64 + 64; c += 32) {
+        uint32_t o0[32];
         float v[32];
+        tmem_ld32(tmem + lane_sel + TM_O + (uint32_t)c, o0);
 #pragma unroll
-        for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(o[e]) * inv;
+        for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(o0[e]) * f0;
+        if (two) {
+          uint32_t o1[32];
+          tmem_ld32(tmem + lane_sel + TM_O + 128 + (uint32_t)c, o1);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = fmaf(__uint_as_float(o1[e]), f1, v[e]);
+        }
         if (row < T) store_row32<MODE>(O, ((size_t)row * a + j) * AD + c, lo_off, v);
       }
     }
@@ -351,7 +375,7 @@ cudaError_t launch_att_t(const LaunchCtx& c, const CUtensorMap& tmK, const CUten
   if (c.launches) ++*c.launches;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((T + AQ - 1) / AQ, a);
-  cfg.blockDim = dim3(192);
+  cfg.blockDim = dim3(ATT_THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = c.stream;
   cudaLaunchAttribute attr[1];
