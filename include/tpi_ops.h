@@ -122,6 +122,15 @@ int tpi_op_gemm_bf16(const void *A, const void *A_lo, int lda, int a_col_batch, 
 int tpi_op_gemm_bf16_swiglu(const void *A, const void *A_lo, int lda, const void *Wgu, void *ACT, int split_out, int T,
                             int s, int K, int32_t *err_word, void *stream);
 
+/* A row-sharded projection of Eq. 1-2 for T > 128 positions with the star sum and the shortcut in the GEMM's epilogue:
+ * X[t][o] <- ((P_0[t][o] + P_1[t][o]) + ...) + X[t][o],  P_i = A[:, i*a_col_batch : i*a_col_batch + K] . W_i^T,
+ * W_i = rows [i * w_row_batch, i * w_row_batch + n_out) of W (bf16, [.][K]); the partial sums P_i are formed in tensor
+ * memory one shard after the other and added in rank order in fp32, the shortcut last; they never reach memory.
+ * A, A_lo (required), err_word as tpi_op_gemm_bf16; X float [T][ldx] in/out (ldx, n_out multiples of 4).
+ * TPI_ERR_SHAPE when T <= 128 or a size rule fails. */
+int tpi_op_gemm_bf16_rowsum(const void *A, const void *A_lo, int lda, int a_col_batch, const void *W, int w_row_batch,
+                            float *X, int ldx, int T, int n_out, int K, int n_shards, int32_t *err_word, void *stream);
+
 /* Eq. 1-2's star sum and shortcut for T positions followed by the next block's RMSNorm:
  * X[t] <- ((P_0[t] + P_1[t]) + ...) + X[t];  Xn[t] = X[t] * rsqrt(mean(X[t]^2) + rms_eps) * gain.
  * partials: float[n_shards][T][h]; X in/out float[T][h]; gain float[h]; Xn float[T][h]. */

@@ -223,6 +223,167 @@ __global__ void __launch_bounds__(192) gemm_tc_pair_kernel(const __grid_constant
   }
 }
 
+// Row-sharded projection with the star sum in the epilogue (Eq. 1-2 for T positions): for each of n_shards shards
+// in rank order the pair's MMA forms the shard's partial sum P_i of a 256-position x 256-column tile in tensor
+// memory (two accumulator buffers, so shard i+1 multiplies while shard i is read back); 8 epilogue warps per CTA
+// keep the running sum ((P_0 + P_1) + ...) in registers (one row and 128 columns per thread), add the shortcut X
+// last and write the new residual stream over X.  The partial sums never reach memory.
+constexpr int RS_BN = 256, RS_THREADS = 320;
+constexpr uint32_t RS_A_BYTES = kMH * kBK * 2, RS_B_BYTES = (RS_BN / 2) * kBK * 2, RS_STAGE = 2 * RS_A_BYTES + RS_B_BYTES;
+constexpr int RS_STAGES = (226 * 1024 - 1024) / RS_STAGE;
+
+struct RowSumArgs {
+  float* X;  // [T][ldx] fp32, residual in, new residual out
+  int ldx, T, n_out, K, n_shards;
+  int a_col_batch;  // A's column offset per shard (elements)
+  int w_row_batch;  // W's row offset per shard
+  int* err;
+};
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+
+__global__ void __launch_bounds__(RS_THREADS) gemm_tc_pair_rowsum_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                                         const __grid_constant__ CUtensorMap tmAlo,
+                                                                         const __grid_constant__ CUtensorMap tmW,
+                                                                         const RowSumArgs a) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full[RS_STAGES], empty[RS_STAGES], acc_ready[2], acc_free[2];
+  __shared__ uint32_t tmem_base_s;
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();  // 0 = leader
+  const int pair = blockIdx.x >> 1;
+  const int n0 = pair * RS_BN, m0 = blockIdx.y * 2 * kMH + (int)rank * kMH;
+  const int kblocks = a.K / kBK;  // per shard
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < RS_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_ready[i], 1); mbar_init(&acc_free[i], 16); }  // 8 warps of each CTA
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_acc = tmem_base_s;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  if (warp == 0) {
+    if (lane == 0) {  // ---- TMA producer: shard after shard, the stage ring runs on across shards
+      const uint32_t bar0 = map_to_cta(smem_u32(&full[0]), 0);
+      int it = 0;
+      bool ok = true;
+      for (int sh = 0; sh < a.n_shards && ok; ++sh)
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % RS_STAGES;
+          const uint32_t ph = (it / RS_STAGES) & 1;
+          if (!mbar_wait(&empty[s], ph ^ 1, a.err)) { ok = false; break; }
+          uint8_t* sa = smem + (size_t)s * RS_STAGE;
+          if (rank == 0) mbar_expect_tx(&full[s], 2 * RS_STAGE);
+          const uint32_t bar = bar0 + (uint32_t)s * 8;
+          const int kx = sh * a.a_col_batch + kb * kBK;
+          tma_load_2d_pair(sa, &tmA, bar, kx, m0);
+          tma_load_2d_pair(sa + RS_A_BYTES, &tmAlo, bar, kx, m0);
+          tma_load_2d_pair(sa + 2 * RS_A_BYTES, &tmW, bar, kb * kBK, sh * a.w_row_batch + n0 + (int)rank * (RS_BN / 2));
+        }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {  // ---- the leader issues the pair's MMAs; shard sh accumulates in buffer sh & 1
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(RS_BN >> 3) << 17) | ((uint32_t)((2 * kMH) >> 4) << 24);
+      const uint32_t empty0_peer = map_to_cta(smem_u32(&empty[0]), 1);
+      int it = 0;
+      bool ok = true;
+      for (int sh = 0; sh < a.n_shards && ok; ++sh) {
+        const int bi = sh & 1;
+        ok = mbar_wait(&acc_free[bi], ((sh >> 1) & 1) ^ 1, a.err);  // both CTAs have read this buffer's previous shard back
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d = tmem_acc + (uint32_t)bi * RS_BN;
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % RS_STAGES;
+          const uint32_t ph = (it / RS_STAGES) & 1;
+          ok = mbar_wait(&full[s], ph, a.err);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + (size_t)s * RS_STAGE);
+          const uint64_t dh = umma_desc_sw128(sa), dl = umma_desc_sw128(sa + RS_A_BYTES), db = umma_desc_sw128(sa + 2 * RS_A_BYTES);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) umma2_bf16(d, dh + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) umma2_bf16(d, dl + 2 * k, db + 2 * k, idesc, 1u);
+          umma2_commit(smem_u32(&empty[s]));
+          umma2_commit(empty0_peer + (uint32_t)s * 8);
+        }
+        umma2_commit(smem_u32(&acc_ready[bi]));
+        umma2_commit(map_to_cta(smem_u32(&acc_ready[bi]), 1));
+      }
+    }
+  } else {  // ---- epilogue: warps 2..9; warp (q, hs) owns rows 32q.. and columns 128 hs .. 128 hs + 127 of the CTA's tile
+    const int q = warp & 3, hs = (warp - 2) >> 2;
+    const uint32_t tbase = tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)hs * 128;
+    const uint32_t free0 = map_to_cta(smem_u32(&acc_free[0]), 0);
+    float sum[128];
+    bool ok = true;
+    for (int sh = 0; sh < a.n_shards && ok; ++sh) {
+      const int bi = sh & 1;
+      ok = mbar_wait(&acc_ready[bi], (sh >> 1) & 1, a.err);
+      if (!ok) break;
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < 128; c += 16) {  // 16 columns at a time: the running sum takes 128 of the thread's registers
+        uint32_t r[16];
+        tmem_ld16(tbase + (uint32_t)bi * RS_BN + (uint32_t)c, r);
+#pragma unroll
+        for (int e = 0; e < 16; ++e) sum[c + e] = sh ? sum[c + e] + __uint_as_float(r[e]) : __uint_as_float(r[e]);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(free0 + (uint32_t)bi * 8);  // on the leader's barrier: its MMA thread reuses the buffer
+    }
+    const int row = m0 + q * 32 + lane;
+    if (ok && row < a.T && a.n_shards > 0 && kblocks > 0) {
+      // column hs*128 + c of the CTA's tile is weight row n0 + hs * 128 + c (the leader's half first)
+      float* x = a.X + (size_t)row * a.ldx + n0 + hs * 128;
+#pragma unroll
+      for (int c = 0; c < 128; c += 4) {
+        const int col = n0 + hs * 128 + c;
+        if (col + 4 <= a.n_out) {
+          const float4 v = *reinterpret_cast<const float4*>(x + c);
+          *reinterpret_cast<float4*>(x + c) = make_float4(sum[c] + v.x, sum[c + 1] + v.y, sum[c + 2] + v.z, sum[c + 3] + v.w);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            if (col + e < a.n_out) x[c + e] = sum[c + e] + x[c + e];
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(512u) : "memory");
+  }
+}
+
 template <int BNA, int NACC>
 cudaError_t launch_pair_t(const LaunchCtx& c, const void* A, const void* Alo, int lda, const void* W, uint64_t w_rows,
                           const GemmTcArgs& a, int n_batch) {
@@ -301,6 +462,50 @@ cudaError_t launch_gemm_tc_pair(const LaunchCtx& c, int shape, const void* A_bf1
     case 3: return launch_pair_t<256, 2>(c, A_bf16, A_lo_bf16, lda, W_bf16, w_rows, a, n_batch);
   }
   return cudaErrorInvalidValue;
+}
+
+bool gemm_tc_rowsum_supported(int T, int K, int a_cols_total, int n_out, int ldx) {
+  const char* e = getenv("TPI_GEMM_ROWSUM");  // TPI_GEMM_ROWSUM=0 keeps the partial sums in memory (for comparisons)
+  return !(e && e[0] == '0') && T > kMH && K > 0 && K % kBK == 0 && a_cols_total % 8 == 0 && ldx % 4 == 0 && n_out % 4 == 0;
+}
+
+cudaError_t launch_gemm_tc_rowsum(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
+                                  const void* W_bf16, int w_row_batch, float* X, int ldx, int T, int n_out, int K, int n_shards,
+                                  int* err) {
+  if (!A_lo_bf16 || n_shards < 1) return cudaErrorInvalidValue;
+  CUtensorMap tmA, tmAlo, tmW;
+  const uint64_t w_rows = (uint64_t)(n_shards - 1) * w_row_batch + n_out;
+  if (!make_map(&tmA, A_bf16, (uint64_t)lda, (uint64_t)T, (uint64_t)lda, kMH)) return cudaErrorInvalidValue;
+  if (!make_map(&tmAlo, A_lo_bf16, (uint64_t)lda, (uint64_t)T, (uint64_t)lda, kMH)) return cudaErrorInvalidValue;
+  if (!make_map(&tmW, W_bf16, (uint64_t)K, w_rows, (uint64_t)K, RS_BN / 2)) return cudaErrorInvalidValue;
+  auto kern = gemm_tc_pair_rowsum_kernel;
+  const size_t smem = (size_t)RS_STAGES * RS_STAGE + 1024;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  if (c.launches) ++*c.launches;
+  RowSumArgs a{X, ldx, T, n_out, K, n_shards, a_col_batch, w_row_batch, err};
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(2 * ((n_out + RS_BN - 1) / RS_BN), (T + 2 * kMH - 1) / (2 * kMH), 1);
+  cfg.blockDim = dim3(RS_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = c.stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.numAttrs = 1;
+  if (c.pdl) {
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 2;
+  }
+  cfg.attrs = attr;
+  return cudaLaunchKernelEx(&cfg, kern, tmA, tmAlo, tmW, a);
 }
 
 }  // namespace tpi

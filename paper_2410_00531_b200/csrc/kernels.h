@@ -123,6 +123,12 @@ int gemm_tc_pair_choose(int T, int n_out, int K, int n_batch, int nsm, double* u
 cudaError_t launch_gemm_tc_pair(const LaunchCtx& c, int shape, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
                                 const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T, int n_out,
                                 int K, int n_batch, int* err, void* act, int act_ld, long long act_lo_off, int act_split);
+// Row-sharded projection of T > 128 positions with the star sum in its epilogue: X[t][o] = ((P_0 + P_1) + ... ) + X[t][o],
+// P_i[t][o] = sum_k (A_hi + A_lo)[t][i*a_col_batch + k] * W[i*w_row_batch + o][k]; the partial sums stay on chip.
+bool gemm_tc_rowsum_supported(int T, int K, int a_cols_total, int n_out, int ldx);
+cudaError_t launch_gemm_tc_rowsum(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
+                                  const void* W_bf16, int w_row_batch, float* X, int ldx, int T, int n_out, int K, int n_shards,
+                                  int* err);
 bool gemm_tc_swiglu_supported(int K, int lda, int s);
 cudaError_t launch_gemm_tc_swiglu(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, const void* Wgu_bf16,
                                   void* ACT, int out_mode, int T, int s, int K, int* err);

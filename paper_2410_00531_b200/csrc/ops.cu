@@ -127,6 +127,15 @@ extern "C" int tpi_op_gemm_bf16_swiglu(const void* A, const void* A_lo, int lda,
   return e == cudaErrorInvalidValue ? TPI_ERR_SHAPE : cu(e);
 }
 
+extern "C" int tpi_op_gemm_bf16_rowsum(const void* A, const void* A_lo, int lda, int a_col_batch, const void* W, int w_row_batch,
+                                       float* X, int ldx, int T, int n_out, int K, int n_shards, int32_t* err_word, void* stream) {
+  if (!A || !A_lo || !W || !X || !err_word || T < 1 || n_out < 1 || K < 1 || n_shards < 1) return TPI_ERR_INVALID_ARG;
+  if (!gemm_tc_rowsum_supported(T, K, lda, n_out, ldx)) return TPI_ERR_SHAPE;
+  const cudaError_t e = launch_gemm_tc_rowsum(ctx(stream), A, A_lo, lda, a_col_batch, W, w_row_batch, X, ldx, T, n_out, K, n_shards,
+                                              err_word);
+  return e == cudaErrorInvalidValue ? TPI_ERR_SHAPE : cu(e);
+}
+
 extern "C" int tpi_op_reduce_residual_norm_rows(const float* partials, int n_shards, int T, int h, float* X, const float* gain,
                                                 float rms_eps, float* Xn, void* stream) {
   if (!partials || !X || !gain || !Xn || n_shards < 1 || T < 1 || h < 1) return TPI_ERR_INVALID_ARG;

@@ -60,6 +60,23 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
     }
     return TPI_OK;
   };
+  // What ends a block: the row-sharded projection -> per-shard partial sums, their star sum in rank order + the shortcut
+  // (Eq. 1-2), the hidden-state tap of the last position, and (next_gain != nullptr) the next block's RMSNorm.  More
+  // than 128 positions of an equal partition: the partial sums are formed and summed inside the GEMM (tensor memory
+  // and registers); otherwise they go through PART.
+  auto block_end = [&](const float* A, int lda, const void* W, const int* k0, int Ks, float* tap, const float* next_gain) -> int {
+    if (tc && act_mode == 2 && !m->unequal && gemm_tc_rowsum_supported(T, Ks, lda, h, h)) {
+      const __nv_bfloat16* hi = reinterpret_cast<const __nv_bfloat16*>(A);
+      CK(launch_gemm_tc_rowsum(lc, hi, hi + (size_t)T * lda, lda, Ks, W, h, X, h, T, h, Ks, N, err));
+      if (tap) CK(cudaMemcpyAsync(tap, X + (size_t)(T - 1) * h, (size_t)h * 4, cudaMemcpyDeviceToDevice, lc.stream));
+      if (next_gain) CK(launch_rmsnorm_rows(lc, X, next_gain, T, h, c.rms_eps, Xn, act_mode));
+      return TPI_OK;
+    }
+    TRY(proj_rows(A, lda, W, k0, Ks));
+    if (next_gain) CK(launch_reduce_residual_norm_rows(lc, PART, N, T, h, X, tap, next_gain, c.rms_eps, Xn, act_mode));
+    else CK(launch_reduce_residual_rows(lc, PART, N, T, h, X, tap));
+    return TPI_OK;
+  };
   CK(launch_embed_rows(lc, dt, m->dev + p.emb, dptr<int>(m, p.tok_hist), pos0, T, c.vocab, h, X, err));
   // With every block resident, the kernel that ends a block (star sum + shortcut) also applies the next block's
   // RMSNorm, whose gain lives in that next block's image; a streamed model may not hold the next block yet.
@@ -79,12 +96,8 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
       CK(launch_prefill_attention_mma(lc, Q, kc, vc, T, pos0, a, b, d, c.max_seq, O, act_mode));
     else
       CK(launch_prefill_attention(lc, dt, Q, kc, vc, T, pos0, a, b, d, c.max_seq, O, act_mode));
-    TRY(proj_rows(O, a * d, br.base + bl.off_wo, ko.data(), Ko));
     float* tap_a = last ? dptr<float>(m, p.taps) + (size_t)(2 * l) * h : nullptr;
-    if (fuse_norm)
-      CK(launch_reduce_residual_norm_rows(lc, PART, N, T, h, X, tap_a, (const float*)resident_block(m, 2 * l + 1), c.rms_eps, Xn, act_mode));
-    else
-      CK(launch_reduce_residual_rows(lc, PART, N, T, h, X, tap_a));
+    TRY(block_end(O, a * d, br.base + bl.off_wo, ko.data(), Ko, tap_a, fuse_norm ? (const float*)resident_block(m, 2 * l + 1) : nullptr));
     TRY(release_block(m, 2 * l));
     TRY(acquire_block(m, 2 * l + 1, &br));
     if (!fuse_norm) CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, act_mode));
@@ -95,13 +108,9 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
       TRY(proj(Xn, h, 0, br.base + bl.off_gu, 2 * s, GU, 0, 2 * s, 2 * s, h, 1));
       CK(launch_swiglu_rows(lc, GU, T, s, ACT, act_mode));
     }
-    TRY(proj_rows(ACT, s, br.base + bl.off_down, kd.data(), Kd));
     float* tap_f = last ? dptr<float>(m, p.taps) + (size_t)(2 * l + 1) * h : nullptr;
     normed = fuse_norm && l + 1 < c.n_layers;
-    if (normed)
-      CK(launch_reduce_residual_norm_rows(lc, PART, N, T, h, X, tap_f, (const float*)resident_block(m, 2 * l + 2), c.rms_eps, Xn, act_mode));
-    else
-      CK(launch_reduce_residual_rows(lc, PART, N, T, h, X, tap_f));
+    TRY(block_end(ACT, s, br.base + bl.off_down, kd.data(), Kd, tap_f, normed ? (const float*)resident_block(m, 2 * l + 2) : nullptr));
     TRY(release_block(m, 2 * l + 1));
   }
   if (last) {

@@ -29,6 +29,7 @@ OPS_SYMBOLS = {
     "tpi_op_gemm_bf16": (_I, [_P, _P, _I, _I, _P, _I, _P, _LL, _I, _I, _I, _I, _I, _P, _P]),
     "tpi_op_prefill_attention": (_I, [_I, _P, _P, _P, _I, _I, _I, _I, _I, _I, _P, _P]),
     "tpi_op_gemm_bf16_swiglu": (_I, [_P, _P, _I, _P, _P, _I, _I, _I, _I, _P, _P]),
+    "tpi_op_gemm_bf16_rowsum": (_I, [_P, _P, _I, _I, _P, _I, _P, _I, _I, _I, _I, _I, _P, _P]),
     "tpi_op_reduce_residual_norm_rows": (_I, [_P, _I, _I, _I, _P, _P, _F, _P, _P]),
 }
 _BOUND = False
@@ -116,6 +117,10 @@ def gemm_bf16(A, lda, a_col_batch, W, w_row_batch, Y, y_bs, ldy, T, n_out, K, n_
 
 def gemm_bf16_swiglu(A, lda, Wgu, ACT, split_out, T, s, K, err_word, stream=None, A_lo=None):
     _check(_ops().tpi_op_gemm_bf16_swiglu(A, A_lo, lda, Wgu, ACT, int(split_out), T, s, K, err_word, stream))
+
+
+def gemm_bf16_rowsum(A, A_lo, lda, a_col_batch, W, w_row_batch, X, ldx, T, n_out, K, n_shards, err_word, stream=None):
+    _check(_ops().tpi_op_gemm_bf16_rowsum(A, A_lo, lda, a_col_batch, W, w_row_batch, X, ldx, T, n_out, K, n_shards, err_word, stream))
 
 
 def reduce_residual_norm_rows(partials, n_shards, T, h, X, gain, rms_eps, Xn, stream=None):

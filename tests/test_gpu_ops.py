@@ -343,6 +343,43 @@ def test_gemm_tensor_core_pair_shapes(T, monkeypatch, shape, Tn, K, n_out, nb):
     assert rel_l2(got[:nb * Tn * n_out].reshape(nb, Tn, n_out), want) < 2e-5
 
 
+@pytest.mark.parametrize("Tn,K,n_out,nb", [(300, 512, 1000, 4), (513, 192, 4096, 8), (129, 64, 260, 1), (1024, 1792, 512, 3)])
+def test_gemm_rowsum_star_sum_in_epilogue(T, Tn, K, n_out, nb):
+    """Row-sharded projection with the star sum and shortcut in the GEMM's epilogue (Eq. 1-2 for T positions): against
+    fp64, and bit for bit against the two-kernel path (partial sums in memory, then the rank-ordered sum)."""
+    import paper_2410_00531_b200.ops as KK
+    rng = np.random.default_rng(Tn + K + nb)
+    A32 = rng.standard_normal((Tn, nb * K)).astype(np.float32)
+    A = S.f32_to_bf16_bits(A32).reshape(Tn, nb * K)
+    Alo = S.f32_to_bf16_bits(A32 - S.bf16_bits_to_f32(A).reshape(A32.shape)).reshape(Tn, nb * K)
+    W = S.f32_to_bf16_bits((rng.standard_normal((nb, n_out, K)) * 0.02).astype(np.float32)).reshape(nb, n_out, K)
+    X0 = rng.standard_normal((Tn, n_out)).astype(np.float32)
+    Ad, Ald, Wd = dev(T, A), dev(T, Alo), dev(T, W)
+    err = T.zeros(1, dtype=T.int32, device="cuda")
+    Xa = T.cat([dev(T, X0.copy()).flatten(), T.full((1024,), 7.0, dtype=T.float32, device="cuda")])
+    KK.gemm_bf16_rowsum(Ad.data_ptr(), Ald.data_ptr(), nb * K, K, Wd.data_ptr(), n_out, Xa.data_ptr(), n_out, Tn, n_out, K, nb,
+                        err.data_ptr())
+    T.cuda.synchronize()
+    assert int(err[0]) == 0
+    got = Xa.cpu().numpy()
+    assert (got[Tn * n_out:] == 7.0).all()
+    got = got[:Tn * n_out].reshape(Tn, n_out)
+    A64, W64 = S.as_f64(A) + S.as_f64(Alo), S.as_f64(W)
+    want = sum(A64[:, b * K:(b + 1) * K] @ W64[b].T for b in range(nb)) + X0
+    assert rel_l2(got, want) < 2e-5
+    # the same partial sums through memory, summed by the row kernel in rank order
+    P = T.empty((nb, Tn, n_out), dtype=T.float32, device="cuda")
+    KK.gemm_bf16(Ad.data_ptr(), nb * K, K, Wd.data_ptr(), n_out, P.data_ptr(), Tn * n_out, n_out, Tn, n_out, K, nb,
+                 err.data_ptr(), A_lo=Ald.data_ptr())
+    Xb = dev(T, X0.copy())
+    g = T.ones(n_out, dtype=T.float32, device="cuda")
+    Xn = T.empty((Tn, n_out), dtype=T.float32, device="cuda")
+    KK.reduce_residual_norm_rows(P.data_ptr(), nb, Tn, n_out, Xb.data_ptr(), g.data_ptr(), 1e-5, Xn.data_ptr())
+    T.cuda.synchronize()
+    assert int(err[0]) == 0
+    assert np.array_equal(Xb.cpu().numpy(), got)
+
+
 @pytest.mark.parametrize("Tn,K,s", [(128, 4096, 11008), (70, 1024, 1360), (300, 512, 48)])
 @pytest.mark.parametrize("split_out", [False, True])
 def test_gemm_tensor_core_swiglu_epilogue(T, Tn, K, s, split_out):
