@@ -369,11 +369,30 @@ def test_second_model_family_non_power_of_two_widths():
     assert mism <= 2
 
 
-@pytest.mark.parametrize("cfg,n_shards,T", [("C2", 4, 128), ("C3", 8, 200)])
-def test_full_width_reduced_depth(cfg, n_shards, T):
+@pytest.mark.parametrize("cfg,n_shards,T,chunk", [("C2", 4, 128, None), ("C3", 8, 200, None), ("C3", 8, 300, None),
+                                                   ("C3", 8, 300, 256)])
+def test_full_width_reduced_depth(cfg, n_shards, T, chunk):
     """The benchmarked shapes end to end at full width (bf16, launch configuration of bench.py:
     graph + PDL), depth reduced to 2 layers and the vocabulary to 32000 so that the fp64 oracle
-    finishes in seconds; teacher-forced, token rule applied at every step."""
+    finishes in seconds; teacher-forced, token rule applied at every step.  300 positions take the
+    long-prompt kernels (CTA-pair projections, star sum in the GEMM epilogue, tcgen05 attention); in chunks
+    of 256 + 44 the second chunk takes the short-prompt kernels on top of the first chunk's cache."""
     shape = S.CONFIGS[cfg].with_(n_layers=2, vocab=32000)
-    toks, mism = _run_and_compare(shape, n_shards, n_decode=6, prompt_len=T)
+    toks, mism = _run_and_compare(shape, n_shards, n_decode=6, prompt_len=T, max_prefill=chunk)
     assert mism <= 3
+
+
+def test_long_prompt_streamed_is_bit_identical_to_resident():
+    """A 300-token prompt of the 8B shape (2 layers) through the long-prompt kernels: the window-streamed model must
+    produce the resident model's bits (first token, its logits, and the tokens after it)."""
+    import paper_2410_00531_b200 as P
+    shape = S.CONFIGS["C3"].with_(n_layers=2, vocab=32000)
+    toks = S.prompt_tokens(shape, 300)
+    res = {}
+    for w in (0, 2):
+        with gpu_session(shape, 320, 300, 8, w) as ses:
+            t0, lg0 = P.prefill(ses.h, toks, shape.vocab)
+            seq = P.decode_run(ses.h, t0, 4)
+            res[w] = (t0, lg0, seq)
+    assert res[0][0] == res[2][0] and (res[0][2] == res[2][2]).all()
+    assert np.array_equal(res[0][1], res[2][1])
