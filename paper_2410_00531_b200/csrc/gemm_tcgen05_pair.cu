@@ -129,8 +129,9 @@ __global__ void __launch_bounds__(192) gemm_tc_pair_kernel(const __grid_constant
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();  // 0 = leader
-  const int pair = blockIdx.x >> 1;
-  const int n0 = pair * BNT, m0 = blockIdx.y * 2 * kMH + (int)rank * kMH, batch = blockIdx.z;
+  // position tiles run fastest over the grid: the pairs in flight share a few weight tiles (read from DRAM once) and
+  // sweep the activations, which fit in L2
+  const int n0 = blockIdx.y * BNT, m0 = (blockIdx.x >> 1) * 2 * kMH + (int)rank * kMH, batch = blockIdx.z;
   const int kblocks = a.K / kBK;
 
   if (threadIdx.x == 0) {
@@ -263,8 +264,7 @@ __global__ void __launch_bounds__(RS_THREADS) gemm_tc_pair_rowsum_kernel(const _
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();  // 0 = leader
-  const int pair = blockIdx.x >> 1;
-  const int n0 = pair * RS_BN, m0 = blockIdx.y * 2 * kMH + (int)rank * kMH;
+  const int n0 = blockIdx.y * RS_BN, m0 = (blockIdx.x >> 1) * 2 * kMH + (int)rank * kMH;  // position tiles run fastest
   const int kblocks = a.K / kBK;  // per shard
 
   if (threadIdx.x == 0) {
@@ -402,7 +402,7 @@ cudaError_t launch_pair_t(const LaunchCtx& c, const void* A, const void* Alo, in
   }
   if (c.launches) ++*c.launches;
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(2 * ((a.n_out + BNT - 1) / BNT), (a.T + 2 * kMH - 1) / (2 * kMH), n_batch);
+  cfg.gridDim = dim3(2 * ((a.T + 2 * kMH - 1) / (2 * kMH)), (a.n_out + BNT - 1) / BNT, n_batch);
   cfg.blockDim = dim3(192);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = c.stream;
@@ -489,7 +489,7 @@ cudaError_t launch_gemm_tc_rowsum(const LaunchCtx& c, const void* A_bf16, const 
   if (c.launches) ++*c.launches;
   RowSumArgs a{X, ldx, T, n_out, K, n_shards, a_col_batch, w_row_batch, err};
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(2 * ((n_out + RS_BN - 1) / RS_BN), (T + 2 * kMH - 1) / (2 * kMH), 1);
+  cfg.gridDim = dim3(2 * ((T + 2 * kMH - 1) / (2 * kMH)), (n_out + RS_BN - 1) / RS_BN, 1);
   cfg.blockDim = dim3(RS_THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = c.stream;
