@@ -1,7 +1,7 @@
 // Prompt-pass projections on the 5th-generation tensor cores (sm_100a):
 //   Y[b][t][o] = sum_k A[t][b*Ka + k] * W[b*rows_b + o][k]     (bf16 x bf16 -> fp32)
 // One CTA computes a 128 x BN tile.  Warp 0 streams 128B-swizzled K-major tiles of A and W into a
-// shared-memory ring with TMA (cp.async.bulk.tensor, no multicast), one thread of warp 1 issues
+// shared-memory ring with TMA (cp.async.bulk.tensor, every CTA loading its own tiles), one thread of warp 1 issues
 // tcgen05.mma (kind::f16, fp32 accumulator in tensor memory), warps 2-5 read the accumulator back
 // with tcgen05.ld and store fp32 rows.  Every wait on an mbarrier is bounded: when a limit runs
 // out the kernel writes DEVERR_WAIT_TIMEOUT to the error word, skips its remaining work, frees its

@@ -11,7 +11,7 @@
 // barrier, the CTA with cluster rank 0); warp 1 lane 0 of the leader issues every MMA and releases a stage in both
 // CTAs with tcgen05.commit; warps 2-5 of each CTA read their own accumulator rows back (a CTA's tensor memory
 // holds its 128 positions x N columns).
-// Every mbarrier wait is bounded; nothing here uses multicast.
+// Every mbarrier wait is bounded; every CTA loads its own tiles.
 #include <stdlib.h>
 
 #include "gemm_tc_common.cuh"
