@@ -137,8 +137,11 @@ int tpi_op_gemm_bf16_rowsum(const void *A, const void *A_lo, int lda, int a_col_
 int tpi_op_reduce_residual_norm_rows(const float *partials, int n_shards, int T, int h, float *X, const float *gain,
                                      float rms_eps, float *Xn, void *stream);
 
-/* Causal attention of T query positions [pos0, pos0+T) over cache positions [0, pos0+T).
- * Q, O: float[T][a][d]. */
+/* Causal attention (Eq. 1) of T query positions [pos0, pos0+T) over cache positions [0, pos0+T); position pos0+t sees
+ * cache rows 0 .. pos0+t.  Q, O: float[T][a][d] (Q after the rotation); kcache, vcache: one layer's cache,
+ * [b][max_seq][d] in dtype, of which nothing past row pos0+T-1 is read.  bf16 caches run on tensor cores with the
+ * queries and the softmax weights split into bf16 hi + lo (d = 128 and T >= 256: tcgen05 with S, P and O in tensor
+ * memory; d = 64 / 128 otherwise: mma.sync); fp32 caches and other d on the fp32 SIMT kernel.  a % b == 0. */
 int tpi_op_prefill_attention(int dtype, const float *Q, const void *kcache, const void *vcache, int T, int pos0,
                              int a, int b, int d, int max_seq, float *O, void *stream);
 
