@@ -247,6 +247,25 @@ def test_heterogeneous_partition_matches_the_oracle(case):
                 P.set_partition(ses.h, *bad)
 
 
+def test_heterogeneous_partition_long_prompt():
+    """Unequal shares with more than 128 prompt positions: one CTA-pair GEMM per shard with contractions of unequal
+    length (the star sum then runs as its own kernel), 7B-shaped widths, two layers, against the oracle."""
+    import paper_2410_00531_b200 as P
+    shape = S.CONFIGS["C2"].with_(n_layers=2, vocab=32000)
+    kv, ff = [16, 8, 4, 4], [5504, 2752, 1408, 1344]
+    toks = S.prompt_tokens(shape, 160)
+    tol = tol_for(shape)
+    orc = make_oracle(shape)
+    want = orc.forward(toks, n_shards=len(kv), partition=(kv, ff))
+    with gpu_session(shape, 176, 160, 1, 0) as ses:
+        P.set_partition(ses.h, kv, ff)
+        t0, lg0 = P.prefill(ses.h, toks, shape.vocab)
+        check_logits(lg0, t0, want, tol)
+        for l in range(shape.n_layers):
+            for which, key in ((0, "attn"), (1, "ffn")):
+                assert rel_l2(P.get_hidden(ses.h, l, which, shape.hidden), orc.taps[(l, key)][-1]) <= tol
+
+
 def test_set_shards_and_set_window_roundtrip():
     import paper_2410_00531_b200 as P
     shape = S.CONFIGS["C1"]

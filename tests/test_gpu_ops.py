@@ -240,7 +240,8 @@ def test_gemm_batched_ragged(T, dtype):
 @pytest.mark.parametrize("dtype,a,b,d,Tq,pos0", [("f32", 4, 4, 64, 16, 0), ("bf16", 8, 2, 128, 37, 20), ("bf16", 8, 1, 32, 5, 0),
                                                     ("bf16", 4, 4, 128, 200, 0), ("bf16", 8, 2, 64, 130, 77), ("bf16", 2, 1, 128, 64, 64),
                                                     ("bf16", 4, 2, 128, 1, 300), ("bf16", 8, 2, 128, 300, 77),
-                                                    ("bf16", 2, 1, 128, 513, 0), ("bf16", 2, 2, 128, 257, 1000)])
+                                                    ("bf16", 2, 1, 128, 513, 0), ("bf16", 2, 2, 128, 257, 1000),
+                                                    ("bf16", 16, 2, 128, 300, 5)])
 def test_prefill_attention(T, dtype, a, b, d, Tq, pos0):
     import paper_2410_00531_b200.ops as K
     n = pos0 + Tq
