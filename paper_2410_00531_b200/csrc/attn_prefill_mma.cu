@@ -6,6 +6,8 @@
 // split into bf16 hi + lo and multiplied twice, so the result keeps fp32-level accuracy.
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "kernels.h"
 #include "launch.cuh"
@@ -239,19 +241,23 @@ cudaError_t launch_t(const LaunchCtx& c, const float* Q, const void* kc, const v
 
 // =====================================================================================================
 // Decode attention on tensor cores: one query position, the GRP query heads of a kv head are the rows
-// (padded to 16) of the same m16n8k16 tiles.  Grid (kv head, split); the 4 warps of a CTA take 64-key
-// tiles of the split in turn (each stages its own K/V tile in shared memory), then the CTA folds the
-// warps' partial results, and the last split of a kv head to finish merges the splits in split order.
+// (padded to 16) of the same m16n8k16 tiles.  Grid (kv head, split); the 8 warps of a CTA take 32 keys each per
+// round of the split, staged in shared memory as two 16-key half tiles with a buffer each.  A split of one round
+// (256 positions) requests both halves up front and multiplies them in one step; longer splits (chosen so that the
+// grid stays within one wave of CTAs: at most SMs / kv heads splits per head) pipeline the halves, the one after
+// next loading while one is multiplied.  Then the CTA folds the warps' partial results, and the last split of a kv
+// head to finish merges the splits in split order.
 // =====================================================================================================
 namespace {
 
 template <int D>
 __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* __restrict__ q, const __nv_bfloat16* kc,
                                                               const __nv_bfloat16* vc, const int* pos, int grp,
-                                                              int max_seq, int nsplit, float* scratch,
+                                                              int max_seq, int nsplit, int max_sph, float* scratch,
                                                               unsigned* tickets, float* o_out) {
-  constexpr int KB = DKB;  // this kernel's tile: DKB keys per warp
-  constexpr int KS = D / 16, ND = D / 8, CPR = D / 8, TILE = KB * D * 2;
+  constexpr int KB = DKB;  // keys per warp and round: two halves of HK keys, each in its own buffer
+  constexpr int HK = KB / 2;
+  constexpr int KS = D / 16, ND = D / 8, CPR = D / 8, TILE = KB * D * 2, HALF = HK * D * 2;
   extern __shared__ __align__(128) uint8_t smem[];  // [DW warps][K tile | V tile], reused by the merge buffers
   __shared__ bool s_last;
   pdl_launch_dependents();
@@ -261,36 +267,46 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
   // The position counter was advanced when the previous token ended, long before this launch; only the cache row of
   // the newest position (and the queries) come from the kernel just before this one.
   const int n = *pos + 1;
-  int chunk = (n + nsplit - 1) / nsplit;
+  // splits of at least 256 positions, and no more of them per kv head than keeps the grid within one wave of CTAs
+  // (max_sph): a warp then walks several rounds of its split, the next half tile loading while one is multiplied
+  const int lim = max(1, min(nsplit, max_sph));
+  int chunk = (n + lim - 1) / lim;
   chunk = max(256, (chunk + 63) & ~63);
   const int nact = (n + chunk - 1) / chunk;
   if (split >= nact) return;  // this split sees no position (its ticket is not counted)
   const int s0 = split * chunk, s1 = min(n, s0 + chunk);
   const __nv_bfloat16* kg = kc + (size_t)kvh * max_seq * D;
   const __nv_bfloat16* vg = vc + (size_t)kvh * max_seq * D;
-  const uint32_t my_k = (uint32_t)__cvta_generic_to_shared(smem) + warp * 2 * TILE, my_v = my_k + TILE;
-
-  // this warp's K/V tile of 64-byte-swizzled rows; the first one is requested before anything else is read
-  auto issue_tile = [&](int k0) {
-    for (int i = lane; i < KB * CPR; i += 32) {
-      const int r = i / CPR, c = i - r * CPR;
-      const uint32_t off = tile_off<D>(r, c);
-      if (k0 + r < s1) {
-        const size_t src = (size_t)(k0 + r) * D + c * 8;
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(my_k + off), "l"(kg + src) : "memory");
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(my_v + off), "l"(vg + src) : "memory");
-      } else {
-        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(my_k + off), "r"(0u) : "memory");
-        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(my_v + off), "r"(0u) : "memory");
+  // per warp: two buffers, each a K half tile and a V half tile of HK rows (64-byte-swizzled 16-byte chunks)
+  const uint32_t my_base = (uint32_t)__cvta_generic_to_shared(smem) + warp * 2 * TILE;
+  // half h of this warp: round h / 2 of the split (DW * KB keys per round), first or second HK keys of the warp's KB
+  auto half_k0 = [&](int hI) { return s0 + (hI >> 1) * (DW * KB) + warp * KB + (hI & 1) * HK; };
+  auto issue_half = [&](int hI) {  // always commits a group, so that "all but the newest group" means "half h landed"
+    const int k0 = half_k0(hI);
+    const uint32_t bk = my_base + (uint32_t)(hI & 1) * 2 * HALF, bv = bk + HALF;
+    if (k0 < s1 || hI < 2) {  // the first two halves are always defined (zeros past the split's end)
+      for (int i = lane; i < HK * CPR; i += 32) {
+        const int r = i / CPR, c = i - r * CPR;
+        const uint32_t off = tile_off<D>(r, c);
+        if (k0 + r < s1) {
+          const size_t src = (size_t)(k0 + r) * D + c * 8;
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(bk + off), "l"(kg + src) : "memory");
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(bv + off), "l"(vg + src) : "memory");
+        } else {
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(bk + off), "r"(0u) : "memory");
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(bv + off), "r"(0u) : "memory");
+        }
       }
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
-  const int k_first = s0 + warp * KB;
-  const bool early = k_first + KB <= n - 1;  // a tile of older positions only: requested ahead of the dependency wait
-  if (k_first < s1 && early) issue_tile(k_first);
+  // halves of older positions only are requested ahead of the dependency wait (the newest row comes from the kernel before)
+  const bool early0 = half_k0(0) + HK <= n - 1, early1 = half_k0(1) + HK <= n - 1;
+  if (early0) issue_half(0);
+  if (early0 && early1) issue_half(1);
   pdl_wait();
-  if (k_first < s1 && !early) issue_tile(k_first);
+  if (!early0) issue_half(0);
+  if (!(early0 && early1)) issue_half(1);
 
   // Q fragments: row g = head g of the group (rows >= grp and rows 8..15 are zero)
   const float qscale = 1.4426950408889634f * rsqrtf((float)D);
@@ -312,21 +328,19 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
   for (int nd = 0; nd < ND; ++nd) { o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f; }
   float m_r = -INFINITY, l_r = 0.f;
 
-  for (int k0 = k_first; k0 < s1; k0 += DW * KB) {  // this warp's tiles of the split
-    if (k0 != k_first) {
-      __syncwarp();
-      issue_tile(k0);
-    }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    __syncwarp();
-    float s[KB / 8][4];
+  // NH half tiles (buffers hI & 1, (hI + 1) & 1) as one step of the online softmax: scores, weights, O += P V
+  auto step = [&](auto nh_c, int hI) {
+    constexpr int NH = decltype(nh_c)::value, NK = NH * HK;
+    const int k0 = half_k0(hI);
+    float s[NK / 8][4];
 #pragma unroll
-    for (int nb = 0; nb < KB / 8; ++nb) {
+    for (int nb = 0; nb < NK / 8; ++nb) {
+      const uint32_t my_k = my_base + (uint32_t)((hI + nb / (HK / 8)) & 1) * 2 * HALF;
       s[nb][0] = s[nb][1] = s[nb][2] = s[nb][3] = 0.f;
 #pragma unroll
       for (int ks = 0; ks < KS; ks += 2) {
         uint32_t kb[4];
-        ldsm_x4(kb, my_k + tile_off<D>(nb * 8 + (lane & 7), ks * 2 + (lane >> 3)));
+        ldsm_x4(kb, my_k + tile_off<D>((nb % (HK / 8)) * 8 + (lane & 7), ks * 2 + (lane >> 3)));
         mma_bf16(s[nb], qh[ks], kb[0], kb[1]);
         mma_bf16(s[nb], ql[ks], kb[0], kb[1]);
         mma_bf16(s[nb], qh[ks + 1], kb[2], kb[3]);
@@ -335,23 +349,23 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
     }
     float mx = -INFINITY;
 #pragma unroll
-    for (int nb = 0; nb < KB / 8; ++nb) {
-      const int key = k0 + nb * 8 + 2 * t;
+    for (int nb = 0; nb < NK / 8; ++nb) {
+      const int key = k0 + nb * 8 + 2 * t;  // the NH halves cover NK consecutive keys
       if (key >= s1) s[nb][0] = -INFINITY;
       if (key + 1 >= s1) s[nb][1] = -INFINITY;
       mx = fmaxf(mx, fmaxf(s[nb][0], s[nb][1]));
     }
     mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
     mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
-    const float mn = fmaxf(m_r, mx);  // finite: the tile's first key is valid
+    const float mn = fmaxf(m_r, mx);  // finite: the step's first key is valid
     const float sc = exp2f(m_r - mn);
     m_r = mn;
     l_r *= sc;
 #pragma unroll
     for (int nd = 0; nd < ND; ++nd) { o[nd][0] *= sc; o[nd][1] *= sc; }
-    uint32_t ph[KB / 16][4], pl[KB / 16][4];
+    uint32_t ph[NK / 16][4], pl[NK / 16][4];
 #pragma unroll
-    for (int nb = 0; nb < KB / 8; ++nb) {
+    for (int nb = 0; nb < NK / 8; ++nb) {
       const float p0 = exp2f(s[nb][0] - mn), p1 = exp2f(s[nb][1] - mn);
       l_r += p0 + p1;
       const int kk = nb >> 1, half = nb & 1;
@@ -359,18 +373,33 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
       ph[kk][half * 2 + 1] = pl[kk][half * 2 + 1] = 0u;
     }
 #pragma unroll
-    for (int kk = 0; kk < KB / 16; ++kk) {
+    for (int kk = 0; kk < NK / 16; ++kk) {
+      const uint32_t my_v = my_base + (uint32_t)((hI + kk / (HK / 16)) & 1) * 2 * HALF + HALF;
 #pragma unroll
       for (int nd = 0; nd < ND; nd += 2) {
         uint32_t vb[4];
-        ldsm_x4_trans(vb, my_v + tile_off<D>(kk * 16 + ((lane >> 3) & 1) * 8 + (lane & 7), nd + (lane >> 4)));
+        ldsm_x4_trans(vb, my_v + tile_off<D>((kk % (HK / 16)) * 16 + ((lane >> 3) & 1) * 8 + (lane & 7), nd + (lane >> 4)));
         mma_bf16(o[nd], ph[kk], vb[0], vb[1]);
         mma_bf16(o[nd], pl[kk], vb[0], vb[1]);
         mma_bf16(o[nd + 1], ph[kk], vb[2], vb[3]);
         mma_bf16(o[nd + 1], pl[kk], vb[2], vb[3]);
       }
     }
+  };
+  if (chunk <= DW * KB) {  // one round per warp: both halves were requested up front and make one step
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncwarp();
+    if (half_k0(0) < s1) step(std::integral_constant<int, 2>{}, 0);
+  } else {
+    for (int hI = 0; half_k0(hI) < s1; ++hI) {  // several rounds: halves hI and hI + 1 are in flight
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+      __syncwarp();
+      step(std::integral_constant<int, 1>{}, hI);
+      __syncwarp();        // every lane is done reading this buffer
+      issue_half(hI + 2);  // the half after next goes into it
+    }
   }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
   l_r += __shfl_xor_sync(0xFFFFFFFFu, l_r, 1);
   l_r += __shfl_xor_sync(0xFFFFFFFFu, l_r, 2);
 
@@ -508,8 +537,11 @@ cudaError_t launch_dec_t(const LaunchCtx& c, const float* q, const void* kc, con
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
+  int sms = 148, dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   return launch_kernel(c, kern, dim3(b, nsplit), dim3(DW * 32), smem, q, (const __nv_bfloat16*)kc,
-                       (const __nv_bfloat16*)vc, pos, a / b, max_seq, nsplit, scratch, tickets, o);
+                       (const __nv_bfloat16*)vc, pos, a / b, max_seq, nsplit, sms / b, scratch, tickets, o);
 }
 
 }  // namespace
