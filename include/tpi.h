@@ -228,11 +228,8 @@ int tpi_steady_conditions(double t_attn, double t_ffn, double t_all_reduce, doub
  * fp32 activation split into two bf16 values, hi + lo, so ~16 mantissa bits
  * survive; 2 = a single bf16 per activation: twice the tensor throughput, but
  * the rounding alone costs ~1e-2 relative error on the logits after two
- * layers of the synthetic workloads; 0 = fp32 SIMT GEMM everywhere; default 1),
- * TPI_OPT_MEGA (1 = with all blocks resident, run a decode step as ONE cooperative
- * kernel with grid barriers between its phases instead of five kernels per layer;
- * default 0: measured slower than the graph of per-phase kernels on B200). */
-enum { TPI_OPT_GRAPH = 0, TPI_OPT_PDL = 1, TPI_OPT_PROFILE = 2, TPI_OPT_TENSOR = 3, TPI_OPT_MEGA = 4 };
+ * layers of the synthetic workloads; 0 = fp32 SIMT GEMM everywhere; default 1). */
+enum { TPI_OPT_GRAPH = 0, TPI_OPT_PDL = 1, TPI_OPT_PROFILE = 2, TPI_OPT_TENSOR = 3 };
 int tpi_set_option(tpi_model *m, int option, int value);
 
 /* Host-only test hook (needs no GPU): drives the window scheduler's ordering

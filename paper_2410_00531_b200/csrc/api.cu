@@ -527,7 +527,6 @@ extern "C" int tpi_set_option(tpi_model* m, int option, int value) {
   switch (option) {
     case TPI_OPT_GRAPH: m->opt_graph = value != 0; break;
     case TPI_OPT_PDL: m->opt_pdl = value != 0; break;
-    case TPI_OPT_MEGA: m->opt_mega = value != 0; break;
     case TPI_OPT_TENSOR: m->opt_tensor = value < 0 ? 0 : (value > 2 ? 2 : value); break;
     case TPI_OPT_PROFILE:
       m->opt_profile = value != 0;

@@ -227,11 +227,11 @@ cudaError_t launch_t(const LaunchCtx& c, const float* Q, const void* kc, const v
                      int max_seq, void* O) {
   auto kern = prefill_attn_mma_kernel<D, MODE>;
   const size_t smem = (size_t)2 * 2 * KB * D * 2;
-  static bool attr_done = false;
-  if (!attr_done && smem > 48 * 1024) {
+  static PerDeviceOnce attr_done;
+  if (!attr_done.get() && smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   return launch_kernel(c, kern, dim3((T + QB - 1) / QB, a), dim3(128), smem, Q, (const __nv_bfloat16*)kc,
                        (const __nv_bfloat16*)vc, T, pos0, a, b, max_seq, O, (size_t)T * a * D);
@@ -264,9 +264,11 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int kvh = blockIdx.x, split = blockIdx.y;
-  // The position counter was advanced when the previous token ended, long before this launch; only the cache row of
-  // the newest position (and the queries) come from the kernel just before this one.
-  const int n = *pos + 1;
+  // The position counter was advanced by the previous token's task head, and the embedding kernel that opens a step
+  // lets no later kernel of the step start before that head has completed; only the cache row of the newest position
+  // (and the queries) come from the kernel just before this one.  Read through L2: the line may sit stale in this
+  // SM's L1 from the step before.
+  const int n = __ldcg(pos) + 1;
   // splits of at least 256 positions, and no more of them per kv head than keeps the grid within one wave of CTAs
   // (max_sph): a warp then walks several rounds of its split, the next half tile loading while one is multiplied
   const int lim = max(1, min(nsplit, max_sph));
@@ -531,11 +533,11 @@ cudaError_t launch_dec_t(const LaunchCtx& c, const float* q, const void* kc, con
                          int b, int max_seq, int nsplit, float* scratch, unsigned* tickets, float* o) {
   auto kern = decode_attn_mma_kernel<D>;
   const size_t smem = (size_t)DW * 2 * DKB * D * 2;  // >= merge buffers (16 DW + 8 DW D + grp * nsplit floats)
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_done;
+  if (!attr_done.get()) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   int sms = 148, dev = 0;
   cudaGetDevice(&dev);

@@ -366,11 +366,11 @@ cudaError_t launch_att_t(const LaunchCtx& c, const CUtensorMap& tmK, const CUten
                          int a, int b, void* O, int* err) {
   auto kern = prefill_attn_tc_kernel<MODE>;
   const size_t smem = ATT_SMEM + 1024;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_done;
+  if (!attr_done.get()) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   if (c.launches) ++*c.launches;
   cudaLaunchConfig_t cfg{};

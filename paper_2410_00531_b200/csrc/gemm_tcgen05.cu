@@ -175,11 +175,11 @@ static cudaError_t launch_tc_t(const LaunchCtx& c, const CUtensorMap& tmA, const
                                const GemmTcArgs& a, int n_batch) {
   auto kern = gemm_tc_kernel<BN, STAGES, SPLIT>;
   const size_t smem = (size_t)STAGES * ((1 + SPLIT) * kBM * kBK * 2 + BN * kBK * 2) + 1024;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_done;
+  if (!attr_done.get()) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   if (c.launches) ++*c.launches;
   cudaLaunchConfig_t cfg{};

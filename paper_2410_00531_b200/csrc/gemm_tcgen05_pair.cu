@@ -394,11 +394,11 @@ cudaError_t launch_pair_t(const LaunchCtx& c, const void* A, const void* Alo, in
   if (!make_map(&tmW, W, (uint64_t)a.K, w_rows, (uint64_t)a.K, BNT / 2)) return cudaErrorInvalidValue;
   auto kern = gemm_tc_pair_kernel<BNA, NACC, STAGES>;
   const size_t smem = (size_t)STAGES * pair_stage_bytes(BNT) + 1024;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_done;
+  if (!attr_done.get()) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   if (c.launches) ++*c.launches;
   cudaLaunchConfig_t cfg{};
@@ -480,11 +480,11 @@ cudaError_t launch_gemm_tc_rowsum(const LaunchCtx& c, const void* A_bf16, const 
   if (!make_map(&tmW, W_bf16, (uint64_t)K, w_rows, (uint64_t)K, RS_BN / 2)) return cudaErrorInvalidValue;
   auto kern = gemm_tc_pair_rowsum_kernel;
   const size_t smem = (size_t)RS_STAGES * RS_STAGE + 1024;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_done;
+  if (!attr_done.get()) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   if (c.launches) ++*c.launches;
   RowSumArgs a{X, ldx, T, n_out, K, n_shards, a_col_batch, w_row_batch, err};

@@ -1,6 +1,5 @@
-// Persistent weight-streaming GEMV bodies shared by the stand-alone kernels (kernels_decode.cu) and the
-// whole-token kernel (decode_mega.cu).  A body is written for CTA `cta` of `ncta` CTAs that are all
-// resident; `xs` is the CTA's dynamic shared memory (the staged activation vector).
+// Persistent weight-streaming GEMV bodies of the decode kernels (kernels_decode.cu).  A body is written for CTA
+// `cta` of `ncta` CTAs that are all resident; `xs` is the CTA's dynamic shared memory (the staged activation vector).
 #pragma once
 #include "common.cuh"
 

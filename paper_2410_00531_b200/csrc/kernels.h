@@ -16,6 +16,18 @@ enum { DT_F32 = 0, DT_BF16 = 1 };
 enum : int { DEVERR_NONE = 0, DEVERR_TOKEN_RANGE = 1, DEVERR_POS_RANGE = 2, DEVERR_WAIT_TIMEOUT = 3 };
 static inline size_t dt_size(int dt) { return dt == DT_BF16 ? 2 : 4; }
 
+// A function attribute (e.g. the dynamic shared memory limit) belongs to one device: this remembers, per device
+// ordinal, whether the current device already has it.
+struct PerDeviceOnce {
+  bool done[64] = {};
+  static int cur() {
+    int dev = 0;
+    return cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 ? dev : -1;
+  }
+  bool get() const { const int d = cur(); return d >= 0 && done[d]; }
+  void set() { const int d = cur(); if (d >= 0) done[d] = true; }
+};
+
 // Input of a GEMV that starts a block: x is either already normalised (ss_part == nullptr) or the
 // raw residual stream together with the producer's partial sums of squares, in which case the kernel
 // applies x * rsqrt(sum(ss_part) / h + eps) while staging; gain (may be null) is the block's norm gain.
@@ -165,42 +177,10 @@ cudaError_t launch_reduce_residual_norm_rows(const LaunchCtx& c, const float* pa
 cudaError_t launch_rmsnorm_stat_row(const LaunchCtx& c, const float* xrow, int h, float eps, float* x,
                                     float* xhat, float* ss_part, int n_parts, int* pos, int pos_value);
 
-// ---------------------------------------------------------------- whole-token decode kernel
-// One cooperative launch per decoded token (all weights resident).  The per-layer argument table lives in
-// device memory: mega_layer_table_bytes(L) bytes, filled on the host with mega_fill_layer and copied over.
-struct MegaLayerDesc {
-  const void *wqkv, *wo, *wgu, *wdown;     // shard-major weight matrices of the layer's two blocks
-  const float *gain_attn, *gain_ffn;
-  void *kc, *vc;                           // this layer's KV cache
-  float *tap_attn, *tap_ffn;               // may be null
-  float *x, *ss_part, *q, *o, *act;        // shared activation buffers
-  const int* pos;
-  const float2* rope;
-  int n_parts, h, a, b, d, s, n_shards, max_seq;
-  float eps;
-};
-struct MegaTokenDesc {
-  const void* layer_table_dev;
-  int n_layers, dt, vocab, max_seq, h, a, b, d, s, nsplit, n_parts;
-  float eps;
-  const void *emb, *head;
-  const float* gain_final;
-  float *x, *ss_part, *q, *o, *attn_scratch, *logits, *amax_val;
-  int* amax_idx;
-  unsigned *tickets, *bar;
-  int *tok_hist, *pos, *err;
-  unsigned long long* ts;  // optional phase-timing stamps (2 per barrier), may be null
-};
-size_t mega_layer_table_bytes(int n_layers);
-void mega_fill_layer(void* table_host, int l, const MegaLayerDesc& d);
-bool mega_supported(int dt, int h, int a, int b, int d, int s);
-size_t mega_smem_bytes(int dt, int h, int a, int b, int d, int s, int nsplit);
-cudaError_t launch_decode_token(const LaunchCtx& c, const MegaTokenDesc& t);
-
 // tuning knobs (0: CTAs per SM of the column-sharded GEMVs, 1: of the fused row-sharded GEMVs,
 // 2: L2 prefetch bytes per row before the dependency wait)
 void set_tuning(int key, int value);
-int get_tuning(int key);  // 4: whole-token kernel's L2 prefetch bytes per row
+int get_tuning(int key);
 
 // misc
 cudaError_t launch_fill_u32(const LaunchCtx& c, uint32_t* p, size_t n, uint32_t v);

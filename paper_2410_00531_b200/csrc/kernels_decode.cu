@@ -21,7 +21,6 @@ struct Tuning {
   int cps_rows = 4;          // CTAs per SM, fused row-sharded GEMVs
   int prefetch_bytes = 1024; // L2 prefetch per row issued before the dependency wait (more than ~2 KB measured slower)
   int warps = 0;             // 0: one CTA per SM with a balanced warp count; 8, 16, 32: that many warps, cps CTAs per SM
-  int mega_prefetch = 2048;  // whole-token kernel: bytes per row requested from L2 ahead of a barrier
 };
 static Tuning g_tune;
 void set_tuning(int key, int value) {
@@ -29,10 +28,9 @@ void set_tuning(int key, int value) {
   if (key == 1) g_tune.cps_rows = value;
   if (key == 2) g_tune.prefetch_bytes = value;
   if (key == 3) g_tune.warps = value;
-  if (key == 4) g_tune.mega_prefetch = value;
 }
 int get_tuning(int key) {
-  return key == 0 ? g_tune.cps_cols : key == 1 ? g_tune.cps_rows : key == 2 ? g_tune.prefetch_bytes : key == 3 ? g_tune.warps : g_tune.mega_prefetch;
+  return key == 0 ? g_tune.cps_cols : key == 1 ? g_tune.cps_rows : key == 2 ? g_tune.prefetch_bytes : key == 3 ? g_tune.warps : 0;
 }
 static int sm_count() {
   static int n = 0;
@@ -236,11 +234,11 @@ static cudaError_t launch_gemv_cols_w(const LaunchCtx& c, GemvArgs& A) {
     grid = g;
   }
   auto kern = gemv_cols_kernel<WT, EPI, WARPS>;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_done;
+  if (!attr_done.get()) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   return launch_kernel(c, kern, dim3((unsigned)grid), dim3(warps * 32), (size_t)A.K * sizeof(float), A);
 }
@@ -265,11 +263,11 @@ static cudaError_t launch_gemv_t(const LaunchCtx& c, GemvArgs& A) {
   const int bps = (A.items_per_shard + WARPS - 1) / WARPS;
   const size_t smem = (size_t)A.kc * sizeof(float);
   auto kern = gemv_kernel<WT, R, EPI, WARPS>;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_done;
+  if (!attr_done.get()) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   return launch_kernel(c, kern, dim3((unsigned)(bps * A.n_shards)), dim3(WARPS * 32), smem, A);
 }
@@ -371,11 +369,11 @@ bool rowshard_fused_supported(int Ks, int n_shards) { return (size_t)Ks * n_shar
 template <typename WT, int R, int NS, int WARPS>
 static cudaError_t launch_rowfused_w(const LaunchCtx& c, RowFusedArgs& A) {
   auto kern = gemv_rowshard_fused_kernel<WT, R, NS, WARPS>;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_done;
+  if (!attr_done.get()) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   const size_t smem = (size_t)A.Ks * A.n_shards * sizeof(float);
   int cps = g_tune.cps_rows < 1 ? 1 : (g_tune.cps_rows > 4 ? 4 : g_tune.cps_rows);
@@ -451,11 +449,11 @@ cudaError_t launch_gemv_rowshard_fused_unequal(const LaunchCtx& c, int dt, const
   auto go = [&](auto wt) -> cudaError_t {
     using WT = decltype(wt);
     auto kern = gemv_rowshard_fused_kernel<WT, 1, 0, 0>;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_done;
+    if (!attr_done.get()) {
       cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
       if (e != cudaSuccess) return e;
-      attr_done = true;
+      attr_done.set();
     }
     int grid, warps;
     balance_split(rows, &grid, &warps);
@@ -472,8 +470,11 @@ __global__ void __launch_bounds__(1024) embed_kernel(const WT* emb, const int* t
                                                     int vocab, int max_seq, int h, float eps, float* x,
                                                     float* xhat, float* ss_part, int n_parts, int* err) {
   __shared__ float red[32];
-  pdl_launch_dependents();
+  // The step's first kernel waits for the previous token's task head (which advances *pos) BEFORE it lets its
+  // dependents start: no kernel of this step can then be resident while the position is still the old one, which
+  // is what lets the attention kernel read *pos ahead of its own dependency wait.
   pdl_wait();
+  pdl_launch_dependents();
   const int p = *pos;
   int tok = (p >= 0 && p < max_seq) ? tok_hist[p] : -1;
   if (p < 0 || p >= max_seq) {
@@ -747,11 +748,11 @@ static cudaError_t launch_attn_t(const LaunchCtx& c, const float* q, const void*
   if (smem < (size_t)GRP * nsplit * sizeof(float)) smem = (size_t)GRP * nsplit * sizeof(float);
   if (smem < (size_t)2 * 256 * D) smem = (size_t)2 * 256 * D;  // K and V windows: 2 x CH x D x sizeof = 512 D bytes
   auto kern = decode_attn_kernel<KT, GRP, LPR>;
-  static bool attr_done = false;
-  if (smem > 48 * 1024 && !attr_done) {
+  static PerDeviceOnce attr_done;
+  if (smem > 48 * 1024 && !attr_done.get()) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   return launch_kernel(c, kern, dim3(b, nsplit), dim3(256), smem, q, (const KT*)kc, (const KT*)vc, pos,
                        max_seq, nsplit, scratch, tickets, o);

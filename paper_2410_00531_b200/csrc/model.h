@@ -54,8 +54,7 @@ struct tpi_model {
   char* host = nullptr;
   cudaStream_t cs = nullptr, ps = nullptr;
   bool own_cs = false, own_ps = false;
-  int opt_graph = 1, opt_pdl = 1, opt_profile = 0, opt_tensor = 1, opt_mega = 0;
-  bool mega_ready = false;  // the whole-token kernel's layer table is in device memory
+  int opt_graph = 1, opt_pdl = 1, opt_profile = 0, opt_tensor = 1;
   int position = 0;
   // window ring
   Ring ring;
@@ -124,5 +123,6 @@ int release_block(tpi_model* m, int block);
 void drop_graph(tpi_model* m);
 void harvest_profile(tpi_model* m);
 int check_device_error(tpi_model* m, const int* io_err);
+void recover_after_failed_step(tpi_model* m);  // after an enqueue that failed part-way
 
 #pragma GCC visibility pop

@@ -41,7 +41,6 @@ struct Plan {
   size_t emb, head, final_gain, rope, inv_freq, kcache, vcache, kv_layer_bytes;
   size_t x, xhat, ss_part, q, o, act, partials, logits, attn_scratch, amax_val, amax_idx, tickets, tok_hist, pos, err,
       taps;
-  size_t mega_table, mega_bar;  // argument table and barrier counter of the whole-token kernel
   size_t pX, pXn, pQKV, pQ, pO, pGU, pACT, pPART;
   size_t blocks;      // start of the weight-block region (resident images or window slots)
   size_t dev_fixed;   // bytes before the block region
@@ -72,7 +71,6 @@ static inline void make_plan(const tpi_config& c, int n_shards_max, int window_b
                s = c.ffn, v = c.vocab, L = c.n_layers, S = c.max_seq, T = c.max_prefill;
   p->bl = block_layout(c);
   p->nsplit = attn_nsplit(c);
-  if (head_blocks < 2048) head_blocks = 2048;  // the whole-token kernel uses one entry per CTA
   p->head_blocks = head_blocks;
   p->n_shards_max = n_shards_max;
   size_t o = 0;
@@ -101,8 +99,6 @@ static inline void make_plan(const tpi_config& c, int n_shards_max, int window_b
   p->pos = take(4);
   p->err = take(4);
   p->taps = take(L * 2 * h * 4);
-  p->mega_table = take(L * 1024);  // >= sizeof(MegaLayer) per layer (checked where the struct lives)
-  p->mega_bar = take(256);
   p->pX = take(T * h * 4);
   p->pXn = take(T * h * 4);
   p->pQKV = take(T * (a + 2 * b) * d * 4);

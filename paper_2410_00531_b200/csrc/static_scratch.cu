@@ -63,7 +63,10 @@ extern "C" size_t tpi_op_static_scratch_floats(void) { return TPI_STATIC_SCRATCH
 
 extern "C" int tpi_op_rowshard_project_static(int dtype, const void* W, const float* x_in, int rows, int Ks,
                                               int n_shards, float eps, float* x, float* xhat, void* stream) {
-  if (rows < 1 || n_shards < 1) return TPI_ERR_INVALID_ARG;
+  if (rows < 1 || n_shards < 1 || Ks < 1 || !W || !x_in || !x || !xhat) {
+    tpi_internal_set_error("tpi_op_rowshard_project_static: rows, Ks and n_shards must be >= 1 and no pointer may be null");
+    return TPI_ERR_INVALID_ARG;
+  }
   if ((size_t)n_shards * (size_t)rows > (size_t)TPI_STATIC_SCRATCH_FLOATS) {
     tpi_internal_set_error(
         "tpi_op_rowshard_project_static: n_shards * rows exceeds the built-in scratch of 65536 floats; "

@@ -1,86 +1,8 @@
 // The per-token step driver: the five kernels per layer (graph + programmatic dependent launch when all blocks are
-// resident, plain launches between the window's events otherwise), the optional whole-token kernel, tpi_decode_*.
+// resident, plain launches between the window's events otherwise), tpi_decode_*.
 #include "model.h"
 
-// Whole-token kernel: per-layer argument table (pointers into the resident block images and the arena).
-static int ensure_mega(tpi_model* m) {
-  if (m->mega_ready) return TPI_OK;
-  const tpi_config& c = m->cfg;
-  const Plan& p = m->plan;
-  const BlockLayout& bl = p.bl;
-  char* tab = m->host + p.h_stage;  // staging area is free outside of loading
-  const int n_parts = rowshard_fused_parts(c.hidden);
-  for (int l = 0; l < c.n_layers; ++l) {
-    char* ab = m->dev + p.blocks + (size_t)l * (bl.attn_bytes + bl.ffn_bytes);
-    char* fb = ab + bl.attn_bytes;
-    MegaLayerDesc d{};
-    d.wqkv = ab + bl.off_qkv; d.wo = ab + bl.off_wo; d.wgu = fb + bl.off_gu; d.wdown = fb + bl.off_down;
-    d.gain_attn = (const float*)ab; d.gain_ffn = (const float*)fb;
-    d.kc = m->dev + p.kcache + (size_t)l * p.kv_layer_bytes;
-    d.vc = m->dev + p.vcache + (size_t)l * p.kv_layer_bytes;
-    d.tap_attn = (float*)(m->dev + p.taps) + (size_t)(2 * l) * c.hidden;
-    d.tap_ffn = d.tap_attn + c.hidden;
-    d.x = (float*)(m->dev + p.x); d.ss_part = (float*)(m->dev + p.ss_part); d.q = (float*)(m->dev + p.q);
-    d.o = (float*)(m->dev + p.o); d.act = (float*)(m->dev + p.act);
-    d.pos = (const int*)(m->dev + p.pos); d.rope = (const float2*)(m->dev + p.rope);
-    d.n_parts = n_parts; d.h = c.hidden; d.a = c.n_heads; d.b = c.n_kv_heads; d.d = c.head_dim; d.s = c.ffn;
-    d.n_shards = m->N; d.max_seq = c.max_seq; d.eps = c.rms_eps;
-    mega_fill_layer(tab, l, d);
-  }
-  CK(cudaMemcpyAsync(m->dev + p.mega_table, tab, mega_layer_table_bytes(c.n_layers), cudaMemcpyHostToDevice, m->cs));
-  CK(cudaStreamSynchronize(m->cs));
-  m->mega_ready = true;
-  return TPI_OK;
-}
-
-static bool mega_usable(const tpi_model* m) {
-  const tpi_config& c = m->cfg;
-  return m->opt_mega && m->window <= 0 && !m->opt_profile && !m->unequal &&
-         mega_supported(c.dtype, c.hidden, c.n_heads, c.n_kv_heads, c.head_dim, c.ffn) &&
-         mega_layer_table_bytes(c.n_layers) <= m->plan.h_stage_bytes &&
-         mega_smem_bytes(c.dtype, c.hidden, c.n_heads, c.n_kv_heads, c.head_dim, c.ffn, m->plan.nsplit) <= 200 * 1024;
-}
-
-static int enqueue_decode_mega(tpi_model* m, LaunchCtx& lc) {
-  const tpi_config& c = m->cfg;
-  const Plan& p = m->plan;
-  MegaTokenDesc t{};
-  t.layer_table_dev = m->dev + p.mega_table;
-  t.n_layers = c.n_layers; t.dt = c.dtype; t.vocab = c.vocab; t.max_seq = c.max_seq; t.h = c.hidden; t.a = c.n_heads;
-  t.b = c.n_kv_heads; t.d = c.head_dim; t.s = c.ffn; t.nsplit = p.nsplit; t.n_parts = rowshard_fused_parts(c.hidden);
-  t.eps = c.rms_eps; t.emb = m->dev + p.emb; t.head = m->dev + p.head; t.gain_final = (const float*)(m->dev + p.final_gain);
-  t.x = (float*)(m->dev + p.x); t.ss_part = (float*)(m->dev + p.ss_part); t.q = (float*)(m->dev + p.q);
-  t.o = (float*)(m->dev + p.o); t.attn_scratch = (float*)(m->dev + p.attn_scratch); t.logits = (float*)(m->dev + p.logits);
-  t.amax_val = (float*)(m->dev + p.amax_val); t.amax_idx = (int*)(m->dev + p.amax_idx);
-  t.tickets = (unsigned*)(m->dev + p.tickets); t.bar = (unsigned*)(m->dev + p.mega_bar);
-  t.tok_hist = (int*)(m->dev + p.tok_hist); t.pos = (int*)(m->dev + p.pos); t.err = (int*)(m->dev + p.err);
-  static const bool want_ts = getenv("TPI_MEGA_TS") != nullptr;  // phase-timing aid: stamps go to the prefill scratch
-  t.ts = want_ts ? (unsigned long long*)(m->dev + p.pX) : nullptr;
-  CK(launch_decode_token(lc, t));
-  if (want_ts) {
-    const int nb = 1 + 5 * c.n_layers;
-    std::vector<unsigned long long> h(2 * nb);
-    CK(cudaMemcpyAsync(h.data(), t.ts, h.size() * 8, cudaMemcpyDeviceToHost, m->cs));
-    CK(cudaStreamSynchronize(m->cs));
-    // per phase kind: time from the previous barrier's release to CTA 0's arrival (work) and arrival -> release (wait)
-    double work[5] = {0, 0, 0, 0, 0}, wait[5] = {0, 0, 0, 0, 0};
-    for (int l = 0; l < c.n_layers; ++l)
-      for (int ph = 0; ph < 5; ++ph) {
-        const int k = 1 + 5 * l + ph;
-        work[ph] += (double)(h[2 * k] - h[2 * k - 1]);
-        wait[ph] += (double)(h[2 * k + 1] - h[2 * k]);
-      }
-    static const char* nm[5] = {"qkv", "attn", "oproj", "gateup", "down"};
-    for (int ph = 0; ph < 5; ++ph)
-      fprintf(stderr, "[mega] %-6s work %.2f us  barrier wait %.2f us (per layer)\n", nm[ph], work[ph] / c.n_layers * 1e-3,
-              wait[ph] / c.n_layers * 1e-3);
-    fprintf(stderr, "[mega] token %.1f us\n", (double)(h[2 * nb - 1] - h[0]) * 1e-3);
-  }
-  return TPI_OK;
-}
-
 void drop_graph(tpi_model* m) {
-  m->mega_ready = false;
   if (m->graph_exec) cudaGraphExecDestroy(m->graph_exec);
   m->graph_exec = nullptr;
 }
@@ -193,7 +115,23 @@ int check_device_error(tpi_model* m, const int* io_err) {
   cudaMemsetAsync(m->dev + m->plan.err, 0, 4, m->cs);
   cudaStreamSynchronize(m->cs);
   if (code == DEVERR_TOKEN_RANGE) return fail(TPI_ERR_TOKEN_RANGE, "a token id was outside [0, vocab)");
+  if (code == DEVERR_WAIT_TIMEOUT) return fail(TPI_ERR_TIMEOUT, "a bounded wait inside a kernel ran out (the kernel returned early)");
   return fail(TPI_ERR_DEVICE_CHECK, "device error word = %d", code);
+}
+
+// An enqueue that fails part-way leaves kernels of an unfinished step in the stream and, in window mode, the ring
+// between an acquire and its release: drain both streams, restart the ring at block 0 and put the device's position
+// counter back to the host's, so that the next call starts from a consistent state.
+void recover_after_failed_step(tpi_model* m) {
+  char saved[512];
+  snprintf(saved, sizeof saved, "%s", tpi_last_error());  // keep the original failure's message
+  cudaStreamSynchronize(m->cs);
+  cudaStreamSynchronize(m->ps);
+  cudaGetLastError();
+  if (m->sched_open) { m->sched_free.push_back(m->sched_open); m->sched_open = nullptr; }
+  if (m->window > 0) start_window(m);
+  write_position(m, m->position);
+  fail(0, "%s", saved);
 }
 
 // io layout (pinned): [0] scratch int, [1] device error word, [2..] token ids
@@ -207,23 +145,18 @@ static int run_decode(tpi_model* m, int32_t token_in, int n_steps, int32_t* toke
   const auto w0 = std::chrono::steady_clock::now();
   io[2] = token_in;
   CK(cudaMemcpyAsync(dptr<int>(m, p.tok_hist) + m->position, io + 2, 4, cudaMemcpyHostToDevice, m->cs));
-  const bool use_mega = mega_usable(m);
-  const bool use_graph = !use_mega && m->opt_graph && m->window <= 0 && !m->opt_profile;
-  if (use_mega) TRY(ensure_mega(m));
+  const bool use_graph = m->opt_graph && m->window <= 0 && !m->opt_profile;
   if (use_graph) TRY(ensure_graph(m));
   int launches = 0;
   CK(cudaEventRecord(m->ev_t0, m->cs));
   for (int i = 0; i < n_steps; ++i) {
-    if (use_mega) {
-      LaunchCtx lc{m->cs, false, &launches};
-      TRY(enqueue_decode_mega(m, lc));
-    } else if (use_graph) { CK(cudaGraphLaunch(m->graph_exec, m->cs)); launches += m->graph_launches; }
+    if (use_graph) { CK(cudaGraphLaunch(m->graph_exec, m->cs)); launches += m->graph_launches; }
     else {
       LaunchCtx lc{m->cs, m->opt_pdl != 0 && !m->opt_profile, &launches};
       m->sched_rec = m->opt_profile != 0;
       const int rc = enqueue_decode(m, lc);
       m->sched_rec = false;
-      TRY(rc);
+      if (rc) { recover_after_failed_step(m); return rc; }
     }
   }
   CK(cudaEventRecord(m->ev_t1, m->cs));
@@ -232,6 +165,11 @@ static int run_decode(tpi_model* m, int32_t token_in, int n_steps, int32_t* toke
   if (logits) CK(cudaMemcpyAsync(m->host + p.h_logits, m->dev + p.logits, (size_t)c.vocab * 4, cudaMemcpyDeviceToHost, m->cs));
   CK(cudaEventRecord(m->ev_done, m->cs));
   TRY(wait_event(m, m->ev_done));
+  if (io[1] != DEVERR_NONE) {  // the step's results are void: the host position stays, the device counter goes back to it
+    const int rc = check_device_error(m, io + 1);
+    write_position(m, m->position);
+    return rc;
+  }
   m->position += n_steps;
   memcpy(tokens_out, io + 3, (size_t)n_steps * 4);
   if (logits) memcpy(logits, m->host + p.h_logits, (size_t)c.vocab * 4);
@@ -241,7 +179,7 @@ static int run_decode(tpi_model* m, int32_t token_in, int n_steps, int32_t* toke
   m->st.last_decode_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - w0).count();
   m->st.kernel_launches_last = launches;
   if (m->opt_profile) harvest_profile(m);
-  return check_device_error(m, io + 1);
+  return TPI_OK;
 }
 
 extern "C" int tpi_decode_step(tpi_model* m, int32_t token_in, int32_t* token_out, float* logits_or_null) {

@@ -148,7 +148,8 @@ extern "C" int tpi_prefill(tpi_model* m, const int32_t* tokens, int n_tokens, in
     memcpy(io + 3, tokens + t0, (size_t)T * 4);
     CK(cudaMemcpyAsync(dptr<int>(m, p.tok_hist) + p_begin + t0, io + 3, (size_t)T * 4, cudaMemcpyHostToDevice, m->cs));
     CK(cudaEventRecord(m->ev_done, m->cs));
-    TRY(enqueue_prefill_chunk(m, lc, p_begin + t0, T, t0 + T == n_tokens));
+    const int rc = enqueue_prefill_chunk(m, lc, p_begin + t0, T, t0 + T == n_tokens);
+    if (rc) { recover_after_failed_step(m); return rc; }
   }
   CK(cudaEventRecord(m->ev_t1, m->cs));
   m->st.last_prefill_enqueue_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - w0).count();
@@ -157,6 +158,11 @@ extern "C" int tpi_prefill(tpi_model* m, const int32_t* tokens, int n_tokens, in
   if (logits_or_null) CK(cudaMemcpyAsync(m->host + p.h_logits, m->dev + p.logits, (size_t)c.vocab * 4, cudaMemcpyDeviceToHost, m->cs));
   CK(cudaEventRecord(m->ev_done, m->cs));
   TRY(wait_event(m, m->ev_done));
+  if (io[1] != DEVERR_NONE) {  // results are void: keep the host position and put the device counter back to it
+    const int rc = check_device_error(m, io + 1);
+    write_position(m, m->position);
+    return rc;
+  }
   m->position = p_begin + n_tokens;
   *first_token = io[2];
   if (logits_or_null) memcpy(logits_or_null, m->host + p.h_logits, (size_t)c.vocab * 4);
@@ -167,6 +173,6 @@ extern "C" int tpi_prefill(tpi_model* m, const int32_t* tokens, int n_tokens, in
   }
   m->st.kernel_launches_last = launches;
   if (m->opt_profile) harvest_profile(m);
-  return check_device_error(m, io + 1);
+  return TPI_OK;
 }
 
