@@ -35,6 +35,19 @@ def rel_l2(got, want) -> float:
     return float(np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-300))
 
 
+def close_elementwise(got, want, tol) -> bool:
+    """The vector bar plus an element bar: rel-L2 <= tol AND no entry further than 3 * tol * rms(want) from the
+    oracle's (a norm alone would let one entry of a long vector drift by a large multiple of the rms).
+    Raises with the measured numbers when a bar is missed; returns True otherwise."""
+    want = np.asarray(want, dtype=np.float64).ravel()
+    got = np.asarray(got, dtype=np.float64).ravel()
+    rms = float(np.sqrt(np.mean(want * want)))
+    r, worst = rel_l2(got, want), float(np.abs(got - want).max())
+    assert r <= tol, f"rel-L2 {r:.3e} > {tol:g}"
+    assert worst <= 3 * tol * max(rms, 1e-300), f"max |delta| {worst:.3e} > 3 * {tol:g} * rms {rms:.3e} (rel-L2 {r:.3e})"
+    return True
+
+
 TINY = S.ModelShape("tiny-test", 2, 32, 4, 2, 8, 48, 37, 1e-5, 10000.0, "f32", 7, 2, 5, 3)
 
 

@@ -5,12 +5,16 @@ import torch
 import pytest
 
 import tpi_synth as S
-from tests.helpers import check_logits, gpu_session, make_oracle, rel_l2, tol_for
+from tests.helpers import check_logits, close_elementwise, gpu_session, make_oracle, rel_l2, tol_for
 
 pytestmark = pytest.mark.gpu
 
 
-def _run_and_compare(shape, n_shards, window=0, n_decode=8, prompt_len=None, max_prefill=None, opts=()):
+def _run_and_compare(shape, n_shards, window=0, n_decode=8, prompt_len=None, max_prefill=None, opts=(), max_ambiguous=None):
+    """Prompt pass + teacher-forced decode against the oracle.  Every hidden state, cache row and logits vector must
+    meet the vector bar (rel-L2 <= tol) and the element bar (max |delta| <= 3 tol rms); every step must satisfy the
+    token rule.  Returns (tokens, mismatches, ambiguous steps): a mismatch is only ever accepted on a step whose
+    oracle top-2 gap is within twice the per-logit allowance, and the number of such steps is bounded by the caller."""
     import paper_2410_00531_b200 as P
     tol = tol_for(shape)
     toks = S.prompt_tokens(shape, prompt_len or shape.prompt_len)
@@ -21,29 +25,36 @@ def _run_and_compare(shape, n_shards, window=0, n_decode=8, prompt_len=None, max
             P.set_option(ses.h, o, v)
         tok, lg = P.prefill(ses.h, toks, shape.vocab)
         want = orc.forward(toks)
-        check_logits(lg, tok, want, tol)
+        ok, amb = check_logits(lg, tok, want, tol)
+        mismatches, ambiguous = int(not ok), int(amb)
         for l in range(shape.n_layers):
-            assert rel_l2(P.get_hidden(ses.h, l, 0, shape.hidden), orc.taps[(l, "attn")][-1]) <= tol
-            assert rel_l2(P.get_hidden(ses.h, l, 1, shape.hidden), orc.taps[(l, "ffn")][-1]) <= tol
+            assert close_elementwise(P.get_hidden(ses.h, l, 0, shape.hidden), orc.taps[(l, "attn")][-1], tol)
+            assert close_elementwise(P.get_hidden(ses.h, l, 1, shape.hidden), orc.taps[(l, "ffn")][-1], tol)
         # cache contents and indexing: slot p holds position p
         for l in range(shape.n_layers):
             for g in range(shape.n_kv_heads):
                 k, v = P.get_kv(ses.h, l, g, 0, T, shape.head_dim)
-                assert rel_l2(k, orc.cache.K[l][g]) <= tol and rel_l2(v, orc.cache.V[l][g]) <= tol
-        out_tokens, mismatches = [tok], 0
+                assert close_elementwise(k, orc.cache.K[l][g], tol) and close_elementwise(v, orc.cache.V[l][g], tol)
+        out_tokens = [tok]
         feed = int(np.argmax(want))
         for step in range(n_decode):
             tok, lg = P.decode_step(ses.h, feed, shape.vocab)   # teacher-forced with the oracle's token
             want = orc.forward([feed])
-            ok, _ = check_logits(lg, tok, want, tol)
+            ok, amb = check_logits(lg, tok, want, tol)
             mismatches += (not ok)
+            ambiguous += amb
             for l in range(shape.n_layers):
-                assert rel_l2(P.get_hidden(ses.h, l, 1, shape.hidden), orc.taps[(l, "ffn")][-1]) <= tol
+                assert close_elementwise(P.get_hidden(ses.h, l, 0, shape.hidden), orc.taps[(l, "attn")][-1], tol)
+                assert close_elementwise(P.get_hidden(ses.h, l, 1, shape.hidden), orc.taps[(l, "ffn")][-1], tol)
             feed = int(np.argmax(want))
             out_tokens.append(tok)
         assert P.position(ses.h) == T + n_decode
         k, v = P.get_kv(ses.h, shape.n_layers - 1, 0, T, n_decode, shape.head_dim)
-        assert rel_l2(k, orc.cache.K[-1][0][T:]) <= tol
+        assert close_elementwise(k, orc.cache.K[-1][0][T:], tol)
+        print(f"[parity] {shape.name} N={n_shards} T={T}: {mismatches} mismatches, {ambiguous} ambiguous of {n_decode + 1} steps")
+        assert mismatches <= ambiguous
+        if max_ambiguous is not None:
+            assert ambiguous <= max_ambiguous
         return out_tokens, mismatches
 
 
@@ -58,37 +69,12 @@ def test_c1_full_depth(n_shards):
 
 def test_c1_every_decode_driver():
     """The default is a CUDA graph of per-phase kernels with programmatic dependent launch; the same
-    kernels also run without PDL or as plain stream launches, and the whole step can run as one
-    cooperative kernel."""
+    kernels also run without PDL or as plain stream launches."""
     import paper_2410_00531_b200 as P
     shape = S.CONFIGS["C1"]
-    _run_and_compare(shape, 2, opts=((P.OPT_MEGA, 1),))
-    _run_and_compare(shape, 4, opts=((P.OPT_MEGA, 1),))
-    _run_and_compare(shape, 2, opts=((P.OPT_MEGA, 0), (P.OPT_GRAPH, 0), (P.OPT_PDL, 0)))
-    _run_and_compare(shape, 2, opts=((P.OPT_MEGA, 0), (P.OPT_GRAPH, 0), (P.OPT_PDL, 1)))
-    _run_and_compare(shape, 2, opts=((P.OPT_MEGA, 0), (P.OPT_GRAPH, 1), (P.OPT_PDL, 0)))
-
-
-@pytest.mark.parametrize("cfg,n_shards", [("C2", 4), ("C3", 8)])
-def test_whole_token_kernel_matches_per_phase_kernels(cfg, n_shards):
-    """Same greedy tokens and (nearly) the same logits from both decode drivers at full width."""
-    import paper_2410_00531_b200 as P
-    shape = S.CONFIGS[cfg].with_(n_layers=2, vocab=32000)
-    toks = S.prompt_tokens(shape, 150)
-    res = {}
-    with gpu_session(shape, 400, 150, n_shards) as ses:
-        for mega in (1, 0):
-            P.set_option(ses.h, P.OPT_MEGA, mega)
-            P.reset(ses.h)
-            t0, _ = P.prefill(ses.h, toks, 0)
-            seq = P.decode_run(ses.h, t0, 40)
-            t1, lg = P.decode_step(ses.h, int(seq[-1]), shape.vocab)
-            st = P.get_stats(ses.h)
-            assert st["kernel_launches_last"] == (1 if mega else 2 + 5 * shape.n_layers)
-            res[mega] = (t0, seq, t1, lg)
-    assert res[1][0] == res[0][0]
-    assert rel_l2(res[1][3], res[0][3]) < 1e-3 or (res[1][1] != res[0][1]).any()
-    assert (res[1][1][:8] == res[0][1][:8]).all()
+    _run_and_compare(shape, 2, opts=((P.OPT_GRAPH, 0), (P.OPT_PDL, 0)))
+    _run_and_compare(shape, 2, opts=((P.OPT_GRAPH, 0), (P.OPT_PDL, 1)))
+    _run_and_compare(shape, 2, opts=((P.OPT_GRAPH, 1), (P.OPT_PDL, 0)))
 
 
 def test_chunked_prefill_matches():
@@ -114,7 +100,6 @@ def test_streamed_is_bit_identical_to_resident(window):
     res = {}
     for w in (0, window):
         with gpu_session(shape, 64, 16, 2, w) as ses:
-            P.set_option(ses.h, P.OPT_MEGA, 0)      # same per-phase kernels in both runs: results must be the same bits
             t0, lg0 = P.prefill(ses.h, toks, shape.vocab)
             seq = P.decode_run(ses.h, t0, 6)
             t1, lg1 = P.decode_step(ses.h, int(seq[-1]), shape.vocab)
@@ -141,7 +126,6 @@ def test_block_retention_is_bit_identical_and_loads_less(window, T):
     for mode in ("resident", "streamed", "retained"):
         extra = n_keep * ffn_bytes if mode == "retained" else 0
         with gpu_session(shape, 64, 16, 2, 0 if mode == "resident" else window, extra_dev_bytes=extra) as ses:
-            P.set_option(ses.h, P.OPT_MEGA, 0)
             if mode == "retained":
                 P.set_retention(ses.h, T)
             t0, lg0 = P.prefill(ses.h, toks, shape.vocab)
@@ -319,7 +303,6 @@ def test_full_size_7b_shape_sampled_outputs_and_size_independent_properties():
         for key, n, w in (("n4", 4, 0), ("n1", 1, 0), ("n4w4", 4, 4)):
             P.set_shards(ses.h, n)
             P.set_window(ses.h, w)
-            P.set_option(ses.h, P.OPT_MEGA, 0)
             t0, lg = P.prefill(ses.h, toks, shape.vocab)
             h_attn, h_ffn = P.get_hidden(ses.h, 0, 0, shape.hidden), P.get_hidden(ses.h, 0, 1, shape.hidden)
             assert rel_l2(h_attn, one.taps[(0, "attn")][-1]) <= 1e-2 and rel_l2(h_ffn, one.taps[(0, "ffn")][-1]) <= 1e-2
