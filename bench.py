@@ -124,13 +124,33 @@ class ClockSampler(threading.Thread):
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def tpi_config(shape: S.ModelShape, max_seq: int, max_prefill: int):
+    import paper_2410_00531_b200 as P
+    return P.make_config(n_layers=shape.n_layers, hidden=shape.hidden, n_heads=shape.n_heads,
+                         n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim, ffn=shape.ffn,
+                         vocab=shape.vocab, max_seq=max_seq, max_prefill=max_prefill,
+                         rms_eps=shape.rms_eps, rope_base=shape.rope_base, dtype=shape.dtype)
+
+
+def make_oracle(shape: S.ModelShape):
+    """The CPU fp64 oracle on the generator's weights (only the CPU-baseline legs come here)."""
+    import functools
+    from oracle.llama_oracle import LlamaOracle, OracleConfig
+
+    @functools.lru_cache(maxsize=64)
+    def w(layer: int, tid: int):
+        return S.as_f64(S.gen_tensor(shape, layer, tid))
+    cfg = OracleConfig(shape.n_layers, shape.hidden, shape.n_heads, shape.n_kv_heads, shape.head_dim, shape.ffn,
+                       shape.vocab, shape.rms_eps, shape.rope_base, "bf16" if shape.dtype == "bf16" else "none")
+    return LlamaOracle(cfg, w)
+
+
 def oracle_sample(shape: S.ModelShape, n_tokens: int, l_red: int = 2, ctx: int = 16):
     """Time the CPU fp64 oracle, as it stands, on a bounded sample of the workload:
     `l_red` layers at full width + the task head, `n_tokens` decode steps after a `ctx`-token
     prompt; per-layer time is scaled linearly to the full depth.  Weight generation is excluded."""
-    from tests.helpers import make_oracle
     red = shape.with_(n_layers=l_red)
-    orc = make_oracle(red, cache=64)
+    orc = make_oracle(red)
     toks = S.prompt_tokens(red, ctx)
     orc.forward(toks)                       # also pulls every weight through the generator once
     t_steps = []
@@ -165,9 +185,12 @@ def run_reference(args, shape):
     steps = steps[args.warmup:]
     ms = float(np.mean(steps)) * 1e3
     out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-           "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / value, "higher_is_better": True,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": workload_name(shape, args), "sample_ms_per_step": ms},
+           "config": {"workload": workload_name(shape, args),
+                      "note": "ms_per_step is the timed step (a bounded sample: 2 layers + head); value is tokens/s "
+                              "with the per-layer time scaled to the full depth",
+                      "full_depth_ms_per_step_extrapolated": 1e3 / value},
            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0, "wall_s": time.perf_counter() - t0}
@@ -197,58 +220,62 @@ def whole_job_value(steps: int, ms: float, world: int) -> float:
 
 
 # ------------------------------------------------------------------ GPU arm
-def run_gpu(args, shape):
+def open_session(P, shape, local, max_seq, prefill_chunk, window=0, retain=0):
+    """Load a model (weights from the seeded generator) into fresh arenas; returns (session, seconds)."""
     import torch
-    import paper_2410_00531_b200 as P
-    from tests.helpers import tpi_config
-
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
-    torch.cuda.set_device(local)
-    K, W, T = args.steps, args.warmup, shape.prompt_len
-    max_seq = T + W + K + 8 + (K + 8 if args.window > 0 else 0)   # the streamed leg also decodes its e2e and diagnostic tokens
-    cfg = tpi_config(shape, max_seq, min(T, args.prefill_chunk))
-    t_load = time.perf_counter()
+    cfg = tpi_config(shape, max_seq, min(shape.prompt_len, prefill_chunk))
+    t0 = time.perf_counter()
     extra = 0
-    if args.window > 0 and args.retain > 0:      # room for the kept FFN blocks beside the window (Prop. 6)
-        extra = len(range(0, shape.n_layers, args.retain)) * P.block_bytes(cfg)[1]
-    elif args.window > 0 and args.retain == -1:  # as many as fit in what the GPU has free (leave 8 GiB of headroom)
-        import torch
+    if window > 0 and retain > 0:      # room for the kept FFN blocks beside the window (Prop. 6)
+        extra = len(range(0, shape.n_layers, retain)) * P.block_bytes(cfg)[1]
+    elif window > 0 and retain == -1:  # as many as fit in what the GPU has free (leave 8 GiB of headroom)
         free_b, _ = torch.cuda.mem_get_info(local)
-        base = P.query_arena(cfg, shape.n_shards, args.window, True)[0]
+        base = P.query_arena(cfg, shape.n_shards, window, True)[0]
         extra = max(0, min(shape.n_layers * P.block_bytes(cfg)[1], free_b - base - (8 << 30)))
-    ses = P.Session(cfg, S.synth_fill(shape), shape.n_shards, args.window, device=local, extra_dev_bytes=extra)
+    ses = P.Session(cfg, S.synth_fill(shape), shape.n_shards, window, device=local, extra_dev_bytes=extra)
     if extra:
-        P.set_retention(ses.h, args.retain)      # -1: the library picks the smallest T that fits the arena
-    t_load = time.perf_counter() - t_load
-    if args.window > 0:
-        return run_streamed(args, shape, ses, t_load, local, rank)
+        P.set_retention(ses.h, retain)           # -1: the library picks the smallest T that fits the arena
+    return ses, time.perf_counter() - t0
+
+
+def close_session(ses):
+    import torch
+    ses.close()
+    del ses
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
+def kv_bytes_per_token(shape, ctx):
+    B = 2 if shape.dtype == "bf16" else 4
+    return 2 * shape.n_layers * shape.n_kv_heads * shape.head_dim * B * (ctx + 1)
+
+
+def resident_decode(P, ses, shape, local, K, W, world=1, n_ttft=4):
+    """TTFT (best of n_ttft - 1 prompt passes after a warm one) and K device-chained decode steps after W warm-up
+    steps, timed with CUDA events on the launching stream between barriers, clocks sampled meanwhile."""
+    import torch
+    h, T = ses.h, shape.prompt_len
     toks = S.prompt_tokens(shape)
-    h = ses.h
 
     def barrier():
         if world > 1:
+            import torch.distributed as dist
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- TTFT: prompt pass (host wall time of the call incl. the token's D2H), best of 3 after a warm pass
     ttft = []
-    for _ in range(1 if args.quick else 4):
+    for _ in range(n_ttft):
         P.reset(h)
         t0 = time.perf_counter()
         first, _ = P.prefill(h, toks, 0)
         ttft.append((time.perf_counter() - t0) * 1e3)
     ttft_ms = min(ttft[1:]) if len(ttft) > 1 else ttft[0]
-
-    # ---- device-resident decode: W warm-up steps, then K timed steps in one enqueue
     tok = int(P.decode_run(h, first, W)[-1]) if W else first
     sampler = ClockSampler(local)
     sampler.start()
-    time.sleep(0.3)
+    time.sleep(0.5)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with torch.cuda.stream(ses.compute):
@@ -259,8 +286,154 @@ def run_gpu(args, shape):
     dev_ms = e0.elapsed_time(e1)
     clocks = sampler.stop()
     st = P.get_stats(h)
-    launches = st["kernel_launches_last"]
     dev_ms = max_over_ranks(dev_ms, f"cuda:{local}")
+    token_bytes = st["weight_bytes_per_token"] + kv_bytes_per_token(shape, T + W + K / 2)
+    return {"first": first, "out": out, "dev_ms": dev_ms, "clocks": clocks, "stats": st, "ttft_ms": ttft_ms,
+            "token_bytes": token_bytes, "token_gbs": token_bytes / (dev_ms / K * 1e-3) / 1e9, "barrier": barrier}
+
+
+def resident_leg(P, name, shape, local, K, W, prefill_chunk):
+    """One more resident workload in compact form (tokens/s, whole-token HBM fraction, TTFT and its fraction)."""
+    T = shape.prompt_len
+    ses, load_s = open_session(P, shape, local, T + W + K + 8, prefill_chunk)
+    try:
+        r = resident_decode(P, ses, shape, local, K, W, n_ttft=3)
+    finally:
+        close_session(ses)
+    peak, kind = measured_peaks()
+    tr = ttft_roofline(shape, T, r["ttft_ms"], r["stats"]["weight_bytes_per_token"], peak)
+    return {"workload": f"{name} {shape.name} N={shape.n_shards} resident", "steps": K, "warmup": W,
+            "context": f"{T + W}..{T + W + K}", "tokens_per_s": round(K / (r["dev_ms"] * 1e-3), 2),
+            "ms_per_step": round(r["dev_ms"] / K, 4), "bytes_per_token": int(r["token_bytes"]),
+            "hbm_gbs": round(r["token_gbs"], 1), "hbm_frac": round(r["token_gbs"] / peak, 4), "peak_kind": kind,
+            "ttft_ms": round(r["ttft_ms"], 3), "ttft_prompt_tokens": T, "ttft_bound": tr["bound"],
+            "ttft_frac": round(tr["frac"], 4), "graph": bool(r["stats"]["graph_active"]),
+            "gpu_launches": r["stats"]["kernel_launches_last"], "clocks": r["clocks"], "load_s": round(load_s, 1)}
+
+
+def host_link_peak(torch, local: int) -> float:
+    """Pinned host -> device copy rate of this machine (GB/s), 1 GiB, best of 4: the streamed runs' denominator."""
+    n = 1 << 30
+    hbuf = torch.empty(n, dtype=torch.uint8, pin_memory=True)
+    dbuf = torch.empty(n, dtype=torch.uint8, device=f"cuda:{local}")
+    best = 0.0
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        dbuf.copy_(hbuf, non_blocking=True)
+        e1.record()
+        torch.cuda.synchronize()
+        best = max(best, n / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    del hbuf, dbuf
+    return best
+
+
+def streamed_decode(P, ses, shape, local, K, W):
+    """Window-streamed decode in its steady state: after the prompt pass and W warm-up tokens the device is drained
+    (the window is then full and none of its bytes count), K tokens are enqueued in one call and the region ends when
+    both streams are idle again, so every block copy issued inside the region also completed inside it.  Tokens/s and
+    link GB/s are K tokens, resp. ALL bytes copied in the region, over the region's wall time."""
+    import torch
+    h = ses.h
+    toks = S.prompt_tokens(shape)
+    t0 = time.perf_counter()
+    first, _ = P.prefill(h, toks, 0)
+    ttft_ms = (time.perf_counter() - t0) * 1e3
+    tok = int(P.decode_run(h, first, W)[-1]) if W else first
+    sampler = ClockSampler(local)
+    sampler.start()
+    torch.cuda.synchronize()
+    st0 = P.get_stats(h)
+    t0 = time.perf_counter()
+    out = P.decode_run(h, tok, K)
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    clocks = sampler.stop()
+    st = P.get_stats(h)
+    region_bytes = st["link_bytes_total"] - st0["link_bytes_total"]
+    return {"out": out, "wall_s": wall, "clocks": clocks, "stats": st, "ttft_ms": ttft_ms,
+            "region_bytes": region_bytes, "link_gbs": region_bytes / wall / 1e9, "tokens_per_s": K / wall}
+
+
+def streamed_leg(P, name, shape, local, K, W, window, link_peak, retain=0):
+    ses, load_s = open_session(P, shape, local, shape.prompt_len + W + K + 16, 4096, window, retain)
+    try:
+        r = streamed_decode(P, ses, shape, local, K, W)
+        P.set_option(ses.h, P.OPT_PROFILE, 1)    # the paper's diagnostics on two more tokens, outside the timed region
+        P.scheduler_reset(ses.h)
+        P.decode_run(ses.h, int(r["out"][-1]), 2)
+        import torch
+        torch.cuda.synchronize()
+        sched = P.scheduler_report(ses.h)
+    finally:
+        close_session(ses)
+    st = r["stats"]
+    return {"workload": f"{name} {shape.name} L{shape.n_layers} N={shape.n_shards} streamed, window {window} blocks"
+                        + (f", retain T={sched['retain_every_T']}" if retain else ""),
+            "steps": K, "warmup": W, "tokens_per_s": round(r["tokens_per_s"], 4),
+            "ms_per_step": round(r["wall_s"] / K * 1e3, 2), "link_bytes_per_token": int(r["region_bytes"] / K),
+            "link_gbs": round(r["link_gbs"], 2), "link_peak_gbs": round(link_peak, 2),
+            "link_frac": round(r["link_gbs"] / link_peak, 4), "window_device_bytes": st["window_peak_bytes"],
+            "retained_blocks": st["retained_blocks"], "ttft_ms": round(r["ttft_ms"], 1),
+            "ttft_prompt_tokens": shape.prompt_len,
+            "sched": {k: (round(v, 3) if isinstance(v, float) else v) for k, v in sched.items()
+                      if k in ("t_attn_ms", "t_ffn_ms", "tau_attn_ms", "tau_ffn_ms", "tight_holds", "loose_holds", "retention_T")},
+            "clocks": r["clocks"], "load_s": round(load_s, 1)}
+
+
+def extra_legs(P, args, local):
+    """The other listed workloads, measured in the same process after the headline: the 8B shape at its 4096-token
+    context and the 70B shape, both resident; then the window-streamed path on 70B-shaped blocks, bf16 and fp32, at a
+    depth that keeps each run near half a minute (the bytes per block and the link rate are what is measured; depth
+    only scales the time per token)."""
+    import torch
+    legs = {}
+
+    def run(key, fn):
+        t0 = time.perf_counter()
+        try:
+            legs[key] = fn()
+            legs[key]["leg_s"] = round(time.perf_counter() - t0, 1)
+        except Exception as e:   # a leg that cannot run on this box (memory) must not take the headline down
+            legs[key] = {"error": f"{type(e).__name__}: {e}"[:300]}
+            torch.cuda.empty_cache()
+
+    want = set(args.legs.split(","))
+    if "C3" in want:
+        run("C3", lambda: resident_leg(P, "C3", S.CONFIGS["C3"], local, 256, 5, args.prefill_chunk))
+    if "C5" in want:
+        run("C5", lambda: resident_leg(P, "C5", S.CONFIGS["C5"], local, 32, 4, args.prefill_chunk))
+    if "S5" in want or "S4" in want:
+        link_peak = host_link_peak(torch, local)
+        if "S5" in want:
+            run("C5_streamed", lambda: streamed_leg(P, "C5-shaped", S.CONFIGS["C5"].with_(n_layers=10, prompt_len=64),
+                                                    local, 16, 2, 8, link_peak))
+        if "S4" in want:
+            run("C4_streamed", lambda: streamed_leg(P, "C4-shaped", S.CONFIGS["C4"].with_(n_layers=5, prompt_len=64),
+                                                    local, 16, 2, 8, link_peak))
+    return legs
+
+
+def run_gpu(args, shape):
+    import torch
+    import paper_2410_00531_b200 as P
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    K, W, T = args.steps, args.warmup, shape.prompt_len
+    if args.window > 0:
+        return run_streamed(args, shape, local, rank)
+    ses, t_load = open_session(P, shape, local, T + W + K + 8, args.prefill_chunk)
+    h = ses.h
+    toks = S.prompt_tokens(shape)
+    r = resident_decode(P, ses, shape, local, K, W, world, n_ttft=1 if args.quick else 4)
+    barrier, dev_ms, st, out = r["barrier"], r["dev_ms"], r["stats"], r["out"]
+    launches = st["kernel_launches_last"]
     value = whole_job_value(K, dev_ms, world)
 
     if args.quick:   # profiling aid: device-resident decode only
@@ -283,7 +456,8 @@ def run_gpu(args, shape):
     e2e_s = max_over_ranks(e2e_s, f"cuda:{local}")
     e2e = whole_job_value(K, e2e_s * 1e3, world)
 
-    # ---- roofline of the dominant kernel (gate/up GEMV), CUDA events around each launch
+    # ---- roofline of the dominant kernel (gate/up GEMV): CUDA events around each launch.  Profile mode runs the step
+    # as plain serialised stream launches (no graph, no programmatic dependent launch), so each launch is timed alone.
     P.set_option(h, P.OPT_PROFILE, 1)
     for _ in range(3):
         tok, _ = P.decode_step(h, tok, 0)
@@ -291,14 +465,8 @@ def run_gpu(args, shape):
     P.set_option(h, P.OPT_PROFILE, 0)
     peak, peak_kind = measured_peaks()
     achieved = sp["dominant_kernel_bytes"] / (sp["dominant_kernel_ms"] * 1e-3) / 1e9 if sp["dominant_kernel_ms"] else None
-    B = 2 if shape.dtype == "bf16" else 4
-    ctx_mid = T + W + K / 2
-    kv_bytes = 2 * shape.n_layers * shape.n_kv_heads * shape.head_dim * B * (ctx_mid + 1)
-    token_bytes = st["weight_bytes_per_token"] + kv_bytes
-    token_gbs = token_bytes / (dev_ms / K * 1e-3) / 1e9
-
+    close_session(ses)
     if rank != 0:
-        ses.close()
         return
     # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only)
     cpu = None
@@ -313,13 +481,13 @@ def run_gpu(args, shape):
                    "l2": "inputs larger than L2: every step streams %.2f GB of weights" % (st["weight_bytes_per_token"] / 1e9),
                    "parallelism": "replicas" if world > 1 else "single GPU, N shards emulated",
                    "graph": bool(st["graph_active"]), "load_s": round(t_load, 1)},
-        "clocks": clocks,
+        "clocks": r["clocks"],
         "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": 4, "d2h_bytes_per_step": 8},
         "gpu_launches": launches,
-        "ttft_ms": ttft_ms, "ttft_prompt_tokens": T,
-        "ttft_roofline": ttft_roofline(shape, T, ttft_ms, st["weight_bytes_per_token"], peak),
-        "token_roofline": {"bound": "hbm", "bytes_per_token": token_bytes, "achieved": token_gbs, "peak": peak,
-                           "unit": "GB/s", "frac": token_gbs / peak, "peak_kind": peak_kind},
+        "ttft_ms": r["ttft_ms"], "ttft_prompt_tokens": T,
+        "ttft_roofline": ttft_roofline(shape, T, r["ttft_ms"], st["weight_bytes_per_token"], peak),
+        "token_roofline": {"bound": "hbm", "bytes_per_token": r["token_bytes"], "achieved": r["token_gbs"], "peak": peak,
+                           "unit": "GB/s", "frac": r["token_gbs"] / peak, "peak_kind": peak_kind},
         "roofline": {"bound": "hbm", "kernel": "gemv_cols_kernel<bf16,EPI_SWIGLU> (gate/up + SwiGLU)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak if achieved else None, "traffic": traffic_from_profile(args.workload),
@@ -328,53 +496,27 @@ def run_gpu(args, shape):
         "cpu_baseline": cpu,
         "tokens_tail": [int(x) for x in out[-4:]],
     }
+    if world == 1 and args.legs and args.workload == "C2" and not (args.layers or args.prompt or args.shards):
+        line["legs"] = extra_legs(P, args, local)
     print(json.dumps(line), flush=True)
-    ses.close()
 
 
-def host_link_peak(torch, local: int) -> float:
-    """Pinned host -> device copy rate of this machine (GB/s), 1 GiB, best of 3: the streamed runs' denominator."""
-    n = 1 << 30
-    hbuf = torch.empty(n, dtype=torch.uint8, pin_memory=True)
-    dbuf = torch.empty(n, dtype=torch.uint8, device=f"cuda:{local}")
-    best = 0.0
-    for _ in range(4):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        dbuf.copy_(hbuf, non_blocking=True)
-        e1.record()
-        torch.cuda.synchronize()
-        best = max(best, n / (e0.elapsed_time(e1) * 1e-3) / 1e9)
-    return best
-
-
-def run_streamed(args, shape, ses, t_load, local, rank):
-    """Window-streamed decode: every layer block crosses the host link once per token."""
+def run_streamed(args, shape, local, rank):
+    """`--window W`: the streamed path as the headline of its own line (steady-state arithmetic as in the legs)."""
     import torch
     import paper_2410_00531_b200 as P
-    h = ses.h
     K, W, T = args.steps, args.warmup, shape.prompt_len
-    toks = S.prompt_tokens(shape)
-    t0 = time.perf_counter()
-    first, _ = P.prefill(h, toks, 0)
-    ttft_ms = (time.perf_counter() - t0) * 1e3
-    tok = int(P.decode_run(h, first, W)[-1]) if W else first
-    st0 = P.get_stats(h)
-    sampler = ClockSampler(local)
-    sampler.start()
+    ses, t_load = open_session(P, shape, local, T + W + 2 * K + 24, args.prefill_chunk, args.window, args.retain)
+    h = ses.h
+    r = streamed_decode(P, ses, shape, local, K, W)
+    st, out = r["stats"], r["out"]
+    # e2e: the per-token public call (same link bytes per step, one host round trip per token)
+    tok = int(out[-1])
     torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    out = P.decode_run(h, tok, K)
-    torch.cuda.synchronize()
-    wall = time.perf_counter() - t0
-    clocks = sampler.stop()
-    st = P.get_stats(h)
-    dev_ms = st["last_decode_dev_ms"]
-    link_bytes = (st["link_bytes_total"] - st0["link_bytes_total"]) / K
-    # e2e: per-token public call
     t0 = time.perf_counter()
     for _ in range(K):
-        tok, _ = P.decode_step(h, int(out[-1]) if _ == 0 else tok, 0)
+        tok, _ = P.decode_step(h, tok, 0)
+    torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     attn_b, ffn_b = P.block_bytes(ses.cfg)
     # the paper's scheduler diagnostics on a few extra tokens (event-timed per block: outside every timed region)
@@ -383,31 +525,28 @@ def run_streamed(args, shape, ses, t_load, local, rank):
     P.decode_run(h, tok, min(K, 4))
     torch.cuda.synchronize()
     sched = P.scheduler_report(h)
-    ses.close()
+    close_session(ses)
     peak = host_link_peak(torch, local)
-    # The window is full when the timed region starts (the loader ran ahead while the host was idle) and the
-    # loader is only one block ahead when it ends, so the copies that overlap the region are the K tokens'
-    # blocks minus one window.
-    timed_bytes = link_bytes * K - st["window_peak_bytes"]
-    gbs = timed_bytes / (dev_ms * 1e-3) / 1e9
+    link_bytes = r["region_bytes"] / K
     line = {
-        "metric": METRIC, "value": K / (dev_ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": W,
-        "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": r["tokens_per_s"], "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": W,
+        "ms_per_step": r["wall_s"] / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": shape.dtype, "data": "synthetic",
         "config": {"workload": workload_name(shape, args).replace("all weights resident", f"layer blocks streamed from pinned host memory, window {args.window} blocks"),
                    "l2": "inputs larger than L2 (every block is copied from host memory each token)",
+                   "timing": "wall time of K chained tokens between two device-wide synchronisations; every byte copied in the region counts",
                    "window_blocks": args.window, "window_device_bytes": st["window_peak_bytes"],
                    "retain_ffn_every": sched["retain_every_T"], "retained_blocks": st["retained_blocks"],
                    "retained_device_bytes": st["retained_bytes"],
                    "block_bytes": {"attention": attn_b, "ffn": ffn_b}, "load_s": round(t_load, 1)},
-        "clocks": clocks,
+        "clocks": r["clocks"],
         "e2e": {"value": K / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(link_bytes) + 4, "d2h_bytes_per_step": 8},
         "gpu_launches": st["kernel_launches_last"],
-        "ttft_ms": ttft_ms, "ttft_prompt_tokens": T, "wall_ms_per_step": wall / K * 1e3,
+        "ttft_ms": r["ttft_ms"], "ttft_prompt_tokens": T, "dev_ms_per_step": st["last_decode_dev_ms"] / K,
         "roofline": {"bound": "host_link", "kernel": "cudaMemcpyAsync of block images on the copy stream",
-                     "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                     "traffic": link_bytes, "bytes_in_timed_region": timed_bytes,
-                     "peak_kind": "pinned H2D copy (1 GiB, best of 4) measured in this run"},
+                     "achieved": r["link_gbs"], "peak": peak, "unit": "GB/s", "frac": r["link_gbs"] / peak,
+                     "traffic": link_bytes, "bytes_in_timed_region": r["region_bytes"],
+                     "peak_kind": "pinned H2D copy (1 GiB, best of 5) measured in this run"},
         "scheduler": sched,
         "cpu_baseline": None, "tokens_tail": [int(x) for x in out[-4:]],
     }
@@ -423,6 +562,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C2", choices=sorted(S.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--legs", default="C3,C5,S5,S4",
+                    help="extra workloads measured after the default headline and reported under `legs` (C3, C5: resident; "
+                         "S5, S4: 70B-shaped bf16 / fp32 blocks window-streamed); empty string = none")
     ap.add_argument("--retain", type=int, default=0,
                     help="with --window: keep one FFN block in every T resident beside the window (0 = none, -1 = as many as fit)")
     ap.add_argument("--window", type=int, default=0,
