@@ -16,6 +16,12 @@
  *  - Every call returns 0 (TPI_OK) or a negative tpi_status.  Nothing aborts.
  *  - A model is used by one host thread at a time.
  *  - Weights are [out][in] row-major, no biases (Table 5's counts have none).
+ *  - Debug aid: with TPI_DEBUG=1 in the environment when tpi_query_arena and
+ *    tpi_load_model are called, every buffer carved from the device arena is
+ *    followed by a 256-byte guard zone holding a known pattern, and a small
+ *    kernel compares all zones at the end of every tpi_prefill / tpi_decode_*
+ *    call: a kernel that wrote past its buffer makes the call return
+ *    TPI_ERR_DEVICE_CHECK, and tpi_last_error() names the zone.
  */
 #ifndef TPI_H
 #define TPI_H
@@ -228,8 +234,12 @@ int tpi_steady_conditions(double t_attn, double t_ffn, double t_all_reduce, doub
  * fp32 activation split into two bf16 values, hi + lo, so ~16 mantissa bits
  * survive; 2 = a single bf16 per activation: twice the tensor throughput, but
  * the rounding alone costs ~1e-2 relative error on the logits after two
- * layers of the synthetic workloads; 0 = fp32 SIMT GEMM everywhere; default 1). */
-enum { TPI_OPT_GRAPH = 0, TPI_OPT_PDL = 1, TPI_OPT_PROFILE = 2, TPI_OPT_TENSOR = 3 };
+ * layers of the synthetic workloads; 0 = fp32 SIMT GEMM everywhere; default 1),
+ * TPI_OPT_WAIT_DEADLINE_MS (value > 0: how long tpi_prefill / tpi_decode_* wait for the device
+ * before they give up with TPI_ERR_TIMEOUT; default 900000, or TPI_WAIT_DEADLINE_S seconds from the
+ * environment.  After a timeout the enqueued work still runs to its end on the device; the host
+ * position is unchanged, and tpi_reset / tpi_set_position drain the stream and re-synchronise). */
+enum { TPI_OPT_GRAPH = 0, TPI_OPT_PDL = 1, TPI_OPT_PROFILE = 2, TPI_OPT_TENSOR = 3, TPI_OPT_WAIT_DEADLINE_MS = 4 };
 int tpi_set_option(tpi_model *m, int option, int value);
 
 /* Host-only test hook (needs no GPU): drives the window scheduler's ordering
@@ -245,6 +255,17 @@ int tpi_ring_trace(int n_blocks, int w, int n_exec, int *ops, int max_ops);
 /* The same with block retention: the FFN block of layers 0, T, 2T, ... is retained; executing a
  * retained block is recorded as op 5 (slot -1) and touches neither queue. */
 int tpi_ring_trace_retained(int n_blocks, int w, int n_exec, int ffn_every_T, int *ops, int max_ops);
+
+/* Host-only test hook for the failure path of the window scheduler (needs no GPU): as
+ * tpi_ring_trace_retained, but the back end's block copy number `fail_copy` (0-based, counted over the
+ * whole run, the start-up loads included) fails once with `fail_status` (a negative tpi_status), the
+ * way a cudaMemcpyAsync that returns an error would.  retry == 0: the run stops where a decoder step
+ * would stop and the call returns fail_status (the failure propagates unchanged).  retry != 0: the
+ * failure is recorded as op 6 (slot = fail_status, block = the block being executed, -1 during
+ * start-up) and the interrupted operation is issued again; the ring must carry on as if nothing had
+ * happened: no block skipped or loaded twice into a live slot, loads still in execution order. */
+int tpi_ring_trace_faulty(int n_blocks, int w, int n_exec, int ffn_every_T, int fail_copy, int fail_status,
+                          int retry, int *ops, int max_ops);
 
 void tpi_free(tpi_model *m);
 const char *tpi_strerror(int code);

@@ -115,6 +115,15 @@ int tpi_op_gemm_bf16(const void *A, const void *A_lo, int lda, int a_col_batch, 
                      long long y_bs, int ldy, int T, int n_out, int K, int n_batch, int32_t *err_word,
                      void *stream);
 
+/* Failure-path check of the kernels' bounded waits (a test aid; the paper has no counterpart): launches the
+ * kernel of tpi_op_gemm_bf16 (single-CTA tiles, one batch, A without a low half) with its loader switched
+ * off and every wait limited to `wait_polls` polls (1..65536, about 0.1 us each), so that no operand ever
+ * arrives and every wait in the kernel runs out.  The kernel must then return by itself within
+ * milliseconds, store nothing to Y, release its tensor memory, and leave 3 (wait timeout) in *err_word;
+ * the device context stays usable.  Nothing in it can wait without a limit and nothing faults. */
+int tpi_op_gemm_bf16_starved(const void *A, int lda, const void *W, float *Y, int ldy, int T, int n_out, int K,
+                             int wait_polls, int32_t *err_word, void *stream);
+
 /* The gate/up projection of Eq. 2 for T positions with SwiGLU applied in the GEMM's epilogue:
  * ACT[t][j] = silu(y[t][2j]) * y[t][2j+1], y = A . Wgu^T, Wgu bf16 [2 s][K] with rows interleaved
  * gate_j, up_j (all shards, shard-major).  A, A_lo as tpi_op_gemm_bf16 (one batch).  ACT: bf16 [T][s];

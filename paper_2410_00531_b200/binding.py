@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtpi.so")
 
 TPI_F32, TPI_BF16 = 0, 1
-OPT_GRAPH, OPT_PDL, OPT_PROFILE, OPT_TENSOR = 0, 1, 2, 3
+OPT_GRAPH, OPT_PDL, OPT_PROFILE, OPT_TENSOR, OPT_WAIT_DEADLINE_MS = 0, 1, 2, 3, 4
 (T_EMB, T_HEAD, T_FINAL_NORM, T_ATTN_NORM, T_WQ, T_WK, T_WV, T_WO,
  T_FFN_NORM, T_WGATE, T_WUP, T_WDOWN) = range(12)
 
@@ -84,6 +84,7 @@ SYMBOLS = {
     "tpi_set_option": (C.c_int, [C.c_void_p, C.c_int, C.c_int]),
     "tpi_ring_trace": (C.c_int, [C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.c_int]),
     "tpi_ring_trace_retained": (C.c_int, [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.c_int]),
+    "tpi_ring_trace_faulty": (C.c_int, [C.c_int] * 7 + [C.POINTER(C.c_int), C.c_int]),
     "tpi_set_retention": (C.c_int, [C.c_void_p, C.c_int]),
     "tpi_set_partition": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
     "tpi_scheduler_report": (C.c_int, [C.c_void_p, C.c_void_p]),
@@ -258,6 +259,17 @@ def ring_trace(n_blocks: int, w: int, n_exec: int, max_ops: int = 1 << 16, ffn_e
     ops = np.zeros((max_ops, 3), np.int32)
     n = _check(lib().tpi_ring_trace_retained(n_blocks, w, n_exec, ffn_every_T,
                                              ops.ctypes.data_as(C.POINTER(C.c_int)), max_ops))
+    if n > max_ops:
+        raise ValueError("trace buffer too small")
+    return ops[:n]
+
+
+def ring_trace_faulty(n_blocks: int, w: int, n_exec: int, fail_copy: int, fail_status: int, retry: bool,
+                      ffn_every_T: int = 0, max_ops: int = 1 << 16) -> np.ndarray:
+    """The ring's ordering trace when block copy number `fail_copy` fails once; raises TpiError(fail_status) unless retry."""
+    ops = np.zeros((max_ops, 3), np.int32)
+    n = _check(lib().tpi_ring_trace_faulty(n_blocks, w, n_exec, ffn_every_T, fail_copy, fail_status, int(retry),
+                                           ops.ctypes.data_as(C.POINTER(C.c_int)), max_ops))
     if n > max_ops:
         raise ValueError("trace buffer too small")
     return ops[:n]

@@ -64,6 +64,30 @@ static int validate(const tpi_config* c, int N) {
   return TPI_OK;
 }
 
+// TPI_DEBUG=1 in the environment builds the device arena with guard zones (read at tpi_query_arena and tpi_load_model,
+// which must see the same setting).
+static bool debug_env() {
+  const char* e = getenv("TPI_DEBUG");
+  return e && e[0] && e[0] != '0';
+}
+
+static CanaryList canary_list(const tpi_model* m) {
+  CanaryList L{};
+  L.n = m->plan.n_canaries;
+  for (int i = 0; i < L.n; ++i) L.off[i] = m->plan.canary_off[i];
+  return L;
+}
+int fill_canaries(tpi_model* m) {
+  LaunchCtx lc{m->cs, false, nullptr};
+  CK(launch_canary_fill(lc, m->dev, canary_list(m)));
+  return TPI_OK;
+}
+int enqueue_canary_check(tpi_model* m, LaunchCtx& lc) {
+  if (m->plan.n_canaries < 1) return TPI_OK;
+  CK(launch_canary_check(lc, m->dev, canary_list(m), dptr<int>(m, m->plan.err)));
+  return TPI_OK;
+}
+
 extern "C" int tpi_query_arena(const tpi_config* cfg, int n_shards_max, int window_blocks, int keep_host_images,
                                size_t* dev_bytes, size_t* host_bytes) {
   TRY(validate(cfg, 1));
@@ -71,7 +95,7 @@ extern "C" int tpi_query_arena(const tpi_config* cfg, int n_shards_max, int wind
   if (n_shards_max < 8) n_shards_max = 8;  // tpi_load_model always plans for at least 8 shards
   Plan p;
   make_plan(*cfg, n_shards_max, window_blocks, keep_host_images, head_argmax_blocks(cfg->vocab), &p, dev_bytes,
-            host_bytes);
+            host_bytes, debug_env());
   return TPI_OK;
 }
 
@@ -93,7 +117,10 @@ int wait_event(tpi_model* m, cudaEvent_t ev) {
     if (spins > 2000) std::this_thread::yield();
     if ((spins & 1023) == 0) {
       const double s = std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count();
-      if (s > m->wait_deadline_s) return fail(TPI_ERR_TIMEOUT, "device did not finish within %.0f s", s);
+      if (s > m->wait_deadline_s) {
+        m->desync = true;  // the enqueued work is still running: host and device positions no longer agree
+        return fail(TPI_ERR_TIMEOUT, "device did not finish within %.3f s", s);
+      }
     }
   }
 }
@@ -303,6 +330,7 @@ static int init_device_state(tpi_model* m) {
   CK(cudaMemsetAsync(m->dev + p.pos, 0, 4, m->cs));
   CK(cudaMemsetAsync(m->dev + p.err, 0, 4, m->cs));
   CK(cudaMemsetAsync(m->dev + p.taps, 0, (size_t)c.n_layers * 2 * c.hidden * 4, m->cs));
+  TRY(fill_canaries(m));
   CK(cudaStreamSynchronize(m->cs));
   return TPI_OK;
 }
@@ -325,7 +353,7 @@ static int load_all(tpi_model* m) {
 static int check_arenas(tpi_model* m, int window, bool host_images, Plan* out) {
   size_t need_d, need_h;
   make_plan(m->cfg, m->plan.n_shards_max, window, host_images, head_argmax_blocks(m->cfg.vocab), out, &need_d,
-            &need_h);
+            &need_h, m->debug);
   if (need_d > m->res.dev_bytes)
     return fail(TPI_ERR_NOMEM, "device arena too small: need %zu bytes, have %zu", need_d, m->res.dev_bytes);
   if (need_h > m->res.host_bytes)
@@ -371,7 +399,8 @@ extern "C" int tpi_load_model(const tpi_config* cfg, const tpi_resources* res, t
   // keep host images when streaming, or when the host arena has room for them anyway
   Plan with_images;
   size_t nd, nh;
-  make_plan(*cfg, m->plan.n_shards_max, window_blocks, 1, head_argmax_blocks(cfg->vocab), &with_images, &nd, &nh);
+  m->debug = debug_env();
+  make_plan(*cfg, m->plan.n_shards_max, window_blocks, 1, head_argmax_blocks(cfg->vocab), &with_images, &nd, &nh, m->debug);
   m->host_images = window_blocks > 0 || nh <= res->host_bytes;
   int rc = check_arenas(m, window_blocks, m->host_images, &m->plan);
   if (rc) { delete m; return rc; }
@@ -422,6 +451,7 @@ int write_position(tpi_model* m, int p) {
   CK(cudaMemcpyAsync(m->dev + m->plan.pos, io, 4, cudaMemcpyHostToDevice, m->cs));
   CK(cudaStreamSynchronize(m->cs));
   m->position = p;
+  m->desync = false;
   return TPI_OK;
 }
 
@@ -528,6 +558,10 @@ extern "C" int tpi_set_option(tpi_model* m, int option, int value) {
     case TPI_OPT_GRAPH: m->opt_graph = value != 0; break;
     case TPI_OPT_PDL: m->opt_pdl = value != 0; break;
     case TPI_OPT_TENSOR: m->opt_tensor = value < 0 ? 0 : (value > 2 ? 2 : value); break;
+    case TPI_OPT_WAIT_DEADLINE_MS:
+      if (value < 1) return fail(TPI_ERR_INVALID_ARG, "the wait deadline must be at least 1 ms");
+      m->wait_deadline_s = value * 1e-3;
+      return TPI_OK;  // nothing about the launch sequence changes: the captured graph stays
     case TPI_OPT_PROFILE:
       m->opt_profile = value != 0;
       if (value && m->prof_ev.empty()) {

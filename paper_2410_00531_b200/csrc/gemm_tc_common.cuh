@@ -31,9 +31,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: about a quarter of a second at most, then the error word is set.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* err) {
-  for (int i = 0; i < (1 << 21); ++i) {
+// Bounded wait: `limit` polls (by default about a quarter of a second), then the error word is set.
+constexpr int kWaitPolls = 1 << 21;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* err, int limit = kWaitPolls) {
+  for (int i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (i > 128) __nanosleep(100);
   }
@@ -97,6 +98,9 @@ struct GemmTcArgs {
   __nv_bfloat16* act;
   long long act_lo_off;
   int act_ld, act_split;
+  // Failure-path test aid (both 0 in every product launch): wait_polls > 0 replaces the poll limit of every wait in
+  // the single-CTA-tile kernel; starve != 0 switches its loader off, so that nothing ever fills a stage.
+  int wait_polls, starve;
 };
 
 constexpr int kBK = 64;

@@ -43,6 +43,7 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * BN, m0 = blockIdx.y * kBM, batch = blockIdx.z;
   const int kblocks = a.K / kBK;
+  const int polls = a.wait_polls > 0 ? a.wait_polls : kWaitPolls;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -63,11 +64,11 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (warp == 0) {
-    if (lane == 0) {  // ---- TMA producer
+    if (lane == 0 && !a.starve) {  // ---- TMA producer
       for (int kb = 0; kb < kblocks; ++kb) {
         const int s = kb % STAGES;
         const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(&empty[s], ph ^ 1, a.err)) break;
+        if (!mbar_wait(&empty[s], ph ^ 1, a.err, polls)) break;
         uint8_t* sa = smem + (size_t)s * STAGE_BYTES;
         mbar_expect_tx(&full[s], STAGE_BYTES);
         tma_load_2d(sa, &tmA, &full[s], batch * a.a_col_batch + kb * kBK, m0);
@@ -83,7 +84,7 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
       for (int kb = 0; kb < kblocks && ok; ++kb) {
         const int s = kb % STAGES;
         const uint32_t ph = (kb / STAGES) & 1;
-        ok = mbar_wait(&full[s], ph, a.err);
+        ok = mbar_wait(&full[s], ph, a.err, polls);
         if (!ok) break;
         tc_fence_after();
         const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
@@ -98,11 +99,13 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
         }
         umma_commit(&empty[s]);  // the stage is free once these MMAs have read it
       }
-      umma_commit(&acc_ready);
+      // after a wait that ran out the accumulator is incomplete: leave acc_ready alone, so that the epilogue's own
+      // (bounded) wait runs out too and nothing is read back or stored
+      if (ok) umma_commit(&acc_ready);
     }
   } else {  // ---- epilogue: warps 2..5 cover the four 32-lane quarters of tensor memory
     const int q = warp & 3;
-    const bool ok = mbar_wait(&acc_ready, 0, a.err);
+    const bool ok = mbar_wait(&acc_ready, 0, a.err, polls);
     tc_fence_after();
     const int row = m0 + q * 32 + lane;
     float* yrow = a.Y + (size_t)batch * a.y_bs + (size_t)row * a.ldy + n0;
@@ -210,7 +213,7 @@ static bool gemm_pair_enabled() {
 static cudaError_t launch_gemm_tc_any(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
                                       const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T,
                                       int n_out, int K, int n_batch, int* err, void* act, int act_ld, long long act_lo_off,
-                                      int act_split) {
+                                      int act_split, int wait_polls = 0, int starve = 0) {
   // Tile width: one CTA computes 128 positions x BN outputs and, per 64-wide k-block, pulls the activation tile(s)
   // plus BN weight rows through shared memory; a CTA's ingest rate is what bounds it, so the cost of a choice is
   // (waves of CTAs over the SMs) x (bytes per k-block), and widths that leave SMs idle or spill into another wave lose.
@@ -233,7 +236,7 @@ static cudaError_t launch_gemm_tc_any(const LaunchCtx& c, const void* A_bf16, co
                                  : (double)waves * ((K / kBK) * tile_us[i] + 4.0 + bn / 64.0);
     if (cost < best - 1e-9) { best = cost; BN = bn; best_us = cost; }
   }
-  if (A_lo_bf16 && T > kBM && gemm_pair_enabled()) {  // a CTA pair (M = 256) pulls half the weight bytes per MMA
+  if (A_lo_bf16 && T > kBM && gemm_pair_enabled() && !starve) {  // a CTA pair (M = 256) pulls half the weight bytes per MMA
     double pair_us = 0;
     const int shape = gemm_tc_pair_choose(T, n_out, K, n_batch, nsm, &pair_us);
     if (shape >= 0 && pair_us < best_us)
@@ -246,7 +249,8 @@ static cudaError_t launch_gemm_tc_any(const LaunchCtx& c, const void* A_bf16, co
   if (!make_map(&tmAlo, A_lo_bf16 ? A_lo_bf16 : A_bf16, (uint64_t)lda, (uint64_t)T, (uint64_t)lda, kBM)) return cudaErrorInvalidValue;
   const uint64_t w_rows = (uint64_t)(n_batch - 1) * w_row_batch + n_out;
   if (!make_map(&tmW, W_bf16, (uint64_t)K, w_rows, (uint64_t)K, (uint32_t)BN)) return cudaErrorInvalidValue;
-  GemmTcArgs a{Y, y_batch_stride, ldy, T, n_out, K, a_col_batch, w_row_batch, err, (__nv_bfloat16*)act, act_lo_off, act_ld, act_split};
+  GemmTcArgs a{Y, y_batch_stride, ldy, T, n_out, K, a_col_batch, w_row_batch, err, (__nv_bfloat16*)act, act_lo_off, act_ld, act_split,
+               wait_polls, starve};
 #define TPI_TC(BNV) \
   return A_lo_bf16 ? launch_tc_t<BNV, stages_for(BNV, 1), 1>(c, tmA, tmAlo, tmW, a, n_batch) \
                    : launch_tc_t<BNV, stages_for(BNV, 0), 0>(c, tmA, tmAlo, tmW, a, n_batch)
@@ -264,6 +268,12 @@ cudaError_t launch_gemm_tc(const LaunchCtx& c, const void* A_bf16, const void* A
                            int n_out, int K, int n_batch, int* err) {
   return launch_gemm_tc_any(c, A_bf16, A_lo_bf16, lda, a_col_batch, W_bf16, w_row_batch, Y, y_batch_stride, ldy, T, n_out, K,
                             n_batch, err, nullptr, 0, 0, 0);
+}
+
+cudaError_t launch_gemm_tc_starved(const LaunchCtx& c, const void* A_bf16, int lda, const void* W_bf16, float* Y, int ldy, int T,
+                                   int n_out, int K, int* err, int wait_polls) {
+  if (wait_polls < 1 || wait_polls > (1 << 16)) return cudaErrorInvalidValue;
+  return launch_gemm_tc_any(c, A_bf16, nullptr, lda, 0, W_bf16, n_out, Y, 0, ldy, T, n_out, K, 1, err, nullptr, 0, 0, 0, wait_polls, 1);
 }
 
 bool gemm_tc_swiglu_supported(int K, int lda, int s) { return gemm_tc_supported(K, lda, 2 * s) && s % 16 == 0; }

@@ -13,7 +13,8 @@ struct LaunchCtx {
 
 enum { DT_F32 = 0, DT_BF16 = 1 };
 // codes written to the device error word by kernel self-checks (the host reads it after a step)
-enum : int { DEVERR_NONE = 0, DEVERR_TOKEN_RANGE = 1, DEVERR_POS_RANGE = 2, DEVERR_WAIT_TIMEOUT = 3 };
+// DEVERR_CANARY + i: the guard zone after the i-th carved arena buffer no longer holds its pattern (debug arenas)
+enum : int { DEVERR_NONE = 0, DEVERR_TOKEN_RANGE = 1, DEVERR_POS_RANGE = 2, DEVERR_WAIT_TIMEOUT = 3, DEVERR_CANARY = 100 };
 static inline size_t dt_size(int dt) { return dt == DT_BF16 ? 2 : 4; }
 
 // A function attribute (e.g. the dynamic shared memory limit) belongs to one device: this remembers, per device
@@ -141,6 +142,11 @@ bool gemm_tc_rowsum_supported(int T, int K, int a_cols_total, int n_out, int ldx
 cudaError_t launch_gemm_tc_rowsum(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
                                   const void* W_bf16, int w_row_batch, float* X, int ldx, int T, int n_out, int K, int n_shards,
                                   int* err);
+// Failure-path test aid: the single-CTA-tile kernel with its loader switched off and every wait cut to `wait_polls`
+// polls (1..65536).  Every wait runs out: the kernel must return by itself, leave Y alone, free its tensor memory and
+// report DEVERR_WAIT_TIMEOUT in *err.
+cudaError_t launch_gemm_tc_starved(const LaunchCtx& c, const void* A_bf16, int lda, const void* W_bf16, float* Y, int ldy, int T,
+                                   int n_out, int K, int* err, int wait_polls);
 bool gemm_tc_swiglu_supported(int K, int lda, int s);
 cudaError_t launch_gemm_tc_swiglu(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, const void* Wgu_bf16,
                                   void* ACT, int out_mode, int T, int s, int K, int* err);
@@ -181,6 +187,15 @@ cudaError_t launch_rmsnorm_stat_row(const LaunchCtx& c, const float* xrow, int h
 // 2: L2 prefetch bytes per row before the dependency wait)
 void set_tuning(int key, int value);
 int get_tuning(int key);
+
+// Guard zones of a debug arena: up to 64 zones of 256 bytes at base + off[i].  fill writes the pattern, check compares
+// it and reports the first damaged zone as DEVERR_CANARY + i in *err (one CTA per zone, no other effect).
+struct CanaryList {
+  int n;
+  unsigned long long off[64];
+};
+cudaError_t launch_canary_fill(const LaunchCtx& c, char* base, const CanaryList& L);
+cudaError_t launch_canary_check(const LaunchCtx& c, const char* base, const CanaryList& L, int* err);
 
 // misc
 cudaError_t launch_fill_u32(const LaunchCtx& c, uint32_t* p, size_t n, uint32_t v);

@@ -602,6 +602,25 @@ cudaError_t launch_fill_u32(const LaunchCtx& c, uint32_t* p, size_t n, uint32_t 
   return launch_kernel(nc, fill_u32_kernel, dim3(blocks ? blocks : 1), dim3(256), 0, p, n, v);
 }
 
+// ------------------------------------------------------------------ guard zones of a debug arena
+__device__ __forceinline__ uint32_t canary_word(int zone, int i) { return 0xC0DE0000u ^ ((uint32_t)zone << 8) ^ (uint32_t)i; }
+__global__ void canary_kernel(char* base, const CanaryList L, int* err, int fill) {
+  pdl_launch_dependents();
+  pdl_wait();  // everything the step wrote is in memory
+  const int z = blockIdx.x, i = threadIdx.x;  // 64 words per zone
+  uint32_t* w = reinterpret_cast<uint32_t*>(base + L.off[z]);
+  if (fill) w[i] = canary_word(z, i);
+  else if (__ldcg(w + i) != canary_word(z, i)) atomicCAS(err, DEVERR_NONE, DEVERR_CANARY + z);
+}
+cudaError_t launch_canary_fill(const LaunchCtx& c, char* base, const CanaryList& L) {
+  if (L.n < 1) return cudaSuccess;
+  return launch_kernel(c, canary_kernel, dim3(L.n), dim3(64), 0, base, L, (int*)nullptr, 1);
+}
+cudaError_t launch_canary_check(const LaunchCtx& c, const char* base, const CanaryList& L, int* err) {
+  if (L.n < 1) return cudaSuccess;
+  return launch_kernel(c, canary_kernel, dim3(L.n), dim3(64), 0, const_cast<char*>(base), L, err, 0);
+}
+
 template <typename WT, int TO_FLOAT>
 __global__ void kv_convert_kernel(WT* cache, float* f, size_t n) {
   pdl_launch_dependents();

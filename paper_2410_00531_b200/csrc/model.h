@@ -93,6 +93,8 @@ struct tpi_model {
   double stall_ms = 0;
   tpi_stats st{};
   double wait_deadline_s = 900.0;
+  bool debug = false;   // TPI_DEBUG=1 at load: guard zones after every arena buffer, checked after every step
+  bool desync = false;  // a host wait timed out with work in flight; cleared by tpi_reset / tpi_set_position
 };
 
 template <typename T>
@@ -109,6 +111,8 @@ char* resident_block(tpi_model* m, int block);
 char* slot_ptr(tpi_model* m, int slot);
 int quiesce(tpi_model* m);
 int write_position(tpi_model* m, int p);
+int fill_canaries(tpi_model* m);
+int enqueue_canary_check(tpi_model* m, LaunchCtx& lc);  // no-op unless the arena was built with guard zones
 // window.cu
 cudaEvent_t sched_event(tpi_model* m);
 void sched_harvest(tpi_model* m);

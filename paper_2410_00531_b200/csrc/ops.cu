@@ -119,6 +119,14 @@ extern "C" int tpi_op_gemm_bf16(const void* A, const void* A_lo, int lda, int a_
   return e == cudaErrorInvalidValue ? TPI_ERR_SHAPE : cu(e);
 }
 
+extern "C" int tpi_op_gemm_bf16_starved(const void* A, int lda, const void* W, float* Y, int ldy, int T, int n_out, int K,
+                                        int wait_polls, int32_t* err_word, void* stream) {
+  if (!A || !W || !Y || !err_word || T < 1 || n_out < 1 || K < 1 || wait_polls < 1 || wait_polls > 65536) return TPI_ERR_INVALID_ARG;
+  if (!gemm_tc_supported(K, lda, ldy)) return TPI_ERR_SHAPE;
+  const cudaError_t e = launch_gemm_tc_starved(ctx(stream), A, lda, W, Y, ldy, T, n_out, K, err_word, wait_polls);
+  return e == cudaErrorInvalidValue ? TPI_ERR_SHAPE : cu(e);
+}
+
 extern "C" int tpi_op_gemm_bf16_swiglu(const void* A, const void* A_lo, int lda, const void* Wgu, void* ACT, int split_out, int T,
                                        int s, int K, int32_t* err_word, void* stream) {
   if (!A || !Wgu || !ACT || !err_word || T < 1 || s < 1 || K < 1) return TPI_ERR_INVALID_ARG;

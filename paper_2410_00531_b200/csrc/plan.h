@@ -34,6 +34,9 @@ static inline BlockLayout block_layout(const tpi_config& c) {
   return b;
 }
 
+constexpr int kMaxCanaries = 64;
+constexpr size_t kCanaryBytes = 256;
+
 struct Plan {
   BlockLayout bl;
   int nsplit, head_blocks, n_shards_max;
@@ -46,6 +49,10 @@ struct Plan {
   size_t dev_fixed;   // bytes before the block region
   // host arena offsets
   size_t h_io, h_logits, h_stage, h_stage_bytes, h_bounce, h_images, host_fixed;
+  // debug build of the arena (TPI_DEBUG=1): a guard zone of kCanaryBytes follows every carved device buffer; the
+  // zones hold a known pattern that a check kernel compares after every step (an overrun of buffer i lands in zone i)
+  int n_canaries;
+  size_t canary_off[kMaxCanaries];
 };
 
 static inline int attn_nsplit(const tpi_config& c) {
@@ -66,7 +73,7 @@ constexpr size_t kMaxNormParts = 1024;
 
 // Fills `p`; returns the bytes needed in each arena for the given residency mode.
 static inline void make_plan(const tpi_config& c, int n_shards_max, int window_blocks, int keep_host,
-                             int head_blocks, Plan* p, size_t* dev_bytes, size_t* host_bytes) {
+                             int head_blocks, Plan* p, size_t* dev_bytes, size_t* host_bytes, bool canaries = false) {
   const size_t B = elem_size(c.dtype), h = c.hidden, d = c.head_dim, a = c.n_heads, b = c.n_kv_heads,
                s = c.ffn, v = c.vocab, L = c.n_layers, S = c.max_seq, T = c.max_prefill;
   p->bl = block_layout(c);
@@ -74,7 +81,13 @@ static inline void make_plan(const tpi_config& c, int n_shards_max, int window_b
   p->head_blocks = head_blocks;
   p->n_shards_max = n_shards_max;
   size_t o = 0;
-  auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
+  p->n_canaries = 0;
+  auto take = [&](size_t bytes) {
+    size_t r = o;
+    o = align_up(o + bytes, 256);
+    if (canaries && p->n_canaries < kMaxCanaries) { p->canary_off[p->n_canaries++] = o; o += kCanaryBytes; }
+    return r;
+  };
   p->emb = take(v * h * B);
   p->head = take(v * h * B);
   p->final_gain = take(h * 4);

@@ -75,7 +75,7 @@ static int enqueue_decode(tpi_model* m, LaunchCtx& lc) {
   CK(launch_head_argmax(lc, dt, m->dev + p.head, norm_in(dptr<float>(m, p.final_gain)), h, c.vocab,
                         dptr<float>(m, p.logits), dptr<float>(m, p.amax_val), dptr<int>(m, p.amax_idx),
                         tickets + b, tok_hist, pos, 1));
-  return TPI_OK;
+  return enqueue_canary_check(m, lc);
 }
 
 static int ensure_graph(tpi_model* m) {
@@ -116,6 +116,9 @@ int check_device_error(tpi_model* m, const int* io_err) {
   cudaStreamSynchronize(m->cs);
   if (code == DEVERR_TOKEN_RANGE) return fail(TPI_ERR_TOKEN_RANGE, "a token id was outside [0, vocab)");
   if (code == DEVERR_WAIT_TIMEOUT) return fail(TPI_ERR_TIMEOUT, "a bounded wait inside a kernel ran out (the kernel returned early)");
+  if (code >= DEVERR_CANARY)
+    return fail(TPI_ERR_DEVICE_CHECK, "guard zone %d of the device arena was overwritten (the buffer carved before it, at arena offset < %zu, was overrun)",
+                code - DEVERR_CANARY, code - DEVERR_CANARY < m->plan.n_canaries ? m->plan.canary_off[code - DEVERR_CANARY] : (size_t)0);
   return fail(TPI_ERR_DEVICE_CHECK, "device error word = %d", code);
 }
 
@@ -137,6 +140,7 @@ void recover_after_failed_step(tpi_model* m) {
 // io layout (pinned): [0] scratch int, [1] device error word, [2..] token ids
 static int run_decode(tpi_model* m, int32_t token_in, int n_steps, int32_t* tokens_out, float* logits) {
   if (!m || n_steps < 1 || !tokens_out) return fail(TPI_ERR_INVALID_ARG, "bad argument");
+  if (m->desync) return fail(TPI_ERR_STATE, "an earlier call timed out with work in flight: call tpi_reset or tpi_set_position first");
   const tpi_config& c = m->cfg;
   if (token_in < 0 || token_in >= c.vocab) return fail(TPI_ERR_TOKEN_RANGE, "token %d outside [0, %d)", token_in, c.vocab);
   if (m->position + n_steps > c.max_seq) return fail(TPI_ERR_SEQ_OVERFLOW, "position %d + %d steps exceeds max_seq %d", m->position, n_steps, c.max_seq);

@@ -124,12 +124,13 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
                           dptr<float>(m, p.logits), dptr<float>(m, p.amax_val), dptr<int>(m, p.amax_idx),
                           dptr<unsigned>(m, p.tickets) + b, dptr<int>(m, p.tok_hist), dptr<int>(m, p.pos), 1));
   }
-  return TPI_OK;
+  return enqueue_canary_check(m, lc);
 }
 
 extern "C" int tpi_prefill(tpi_model* m, const int32_t* tokens, int n_tokens, int32_t* first_token,
                            float* logits_or_null) {
   if (!m || !tokens || n_tokens < 1 || !first_token) return fail(TPI_ERR_INVALID_ARG, "bad argument");
+  if (m->desync) return fail(TPI_ERR_STATE, "an earlier call timed out with work in flight: call tpi_reset or tpi_set_position first");
   const tpi_config& c = m->cfg;
   const Plan& p = m->plan;
   if (m->position + n_tokens > c.max_seq) return fail(TPI_ERR_SEQ_OVERFLOW, "position %d + %d tokens exceeds max_seq %d", m->position, n_tokens, c.max_seq);

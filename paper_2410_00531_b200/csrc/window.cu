@@ -238,7 +238,6 @@ int tr_push(void* ctx, int op, int slot, int block) {
   return 0;
 }
 int tr_cwr(void* c, int s) { return tr_push(c, 0, s, -1); }
-int tr_cb(void* c, int s, int b) { return tr_push(c, 1, s, b); }
 int tr_crl(void* c, int s) { return tr_push(c, 2, s, -1); }
 int tr_xwl(void* c, int s) { return tr_push(c, 3, s, -1); }
 int tr_xrr(void* c, int s) { return tr_push(c, 4, s, -1); }
@@ -254,27 +253,64 @@ extern "C" int tpi_ring_trace(int n_blocks, int w, int n_exec, int* ops, int max
 }
 
 extern "C" int tpi_ring_trace_retained(int n_blocks, int w, int n_exec, int ffn_every_T, int* ops, int max_ops) {
+  return tpi_ring_trace_faulty(n_blocks, w, n_exec, ffn_every_T, -1, 0, 0, ops, max_ops);
+}
+
+namespace {
+struct FaultyCtx {
+  TraceCtx t;
+  int copies, fail_copy, fail_status;
+};
+int ft_cb(void* c, int s, int b) {
+  FaultyCtx* f = (FaultyCtx*)c;
+  if (f->copies++ == f->fail_copy) return f->fail_status;  // the copy was not issued: nothing is recorded
+  return tr_push(&f->t, 1, s, b);
+}
+}  // namespace
+
+extern "C" int tpi_ring_trace_faulty(int n_blocks, int w, int n_exec, int ffn_every_T, int fail_copy, int fail_status,
+                                     int retry, int* ops, int max_ops) {
+  if (fail_copy >= 0 && fail_status >= 0) return fail(TPI_ERR_INVALID_ARG, "fail_status must be a negative status");
   if (n_blocks < 2 || n_blocks % 2 || w < 1 || n_exec < 0 || ffn_every_T < 0 || (!ops && max_ops > 0))
     return fail(TPI_ERR_INVALID_ARG, "bad argument");
   std::vector<char> keep(n_blocks, 0);
   if (ffn_every_T > 0)
     for (int l = 0; l < n_blocks / 2; l += ffn_every_T) keep[2 * l + 1] = 1;
-  TraceCtx t{ops, max_ops, 0};
+  FaultyCtx f{{ops, max_ops, 0}, 0, fail_copy, fail_status};
+  TraceCtx& t = f.t;
   RingBackend be;
-  be.ctx = &t;
+  be.ctx = &f;  // TraceCtx is FaultyCtx's first member: the recording callbacks take the same pointer
   be.copy_wait_released = tr_cwr;
-  be.copy_block = tr_cb;
+  be.copy_block = ft_cb;
   be.copy_record_loaded = tr_crl;
   be.compute_wait_loaded = tr_xwl;
   be.compute_record_released = tr_xrr;
   Ring r;
   r.configure(n_blocks, w, be, keep.data());
-  if (r.pump()) return TPI_ERR_STATE;
+  // a failure surfaces from the call that pumped the loader; with `retry` that call's pending part is issued again
+  auto failed = [&](int rc, int blk) -> bool {  // true: give up with rc
+    if (rc != fail_status || !retry) return true;
+    tr_push(&t, 6, fail_status, blk);
+    return false;
+  };
+  int rc = r.pump();
+  if (rc) {
+    if (failed(rc, -1)) return rc < 0 ? rc : TPI_ERR_STATE;
+    if ((rc = r.pump())) return rc < 0 ? rc : TPI_ERR_STATE;
+  }
   for (int i = 0; i < n_exec; ++i) {
     const int blk = i % n_blocks;
     if (keep[blk]) { tr_push(&t, 5, -1, blk); continue; }  // a retained block runs without any window operation
-    if (r.acquire(blk) < 0) return TPI_ERR_STATE;
-    if (r.release(blk)) return TPI_ERR_STATE;
+    int s = r.acquire(blk);
+    if (s < 0) {
+      if (failed(s, blk)) return s == -1000 || s == -1001 ? TPI_ERR_STATE : s;
+      if ((s = r.acquire(blk)) < 0) return s == -1000 || s == -1001 ? TPI_ERR_STATE : s;
+    }
+    rc = r.release(blk);
+    if (rc) {  // the block itself was released before the loader was pumped: only the pump is repeated
+      if (failed(rc, blk)) return rc == -1000 ? TPI_ERR_STATE : rc;
+      if ((rc = r.pump())) return rc < 0 ? rc : TPI_ERR_STATE;
+    }
   }
   return t.n;
 }

@@ -27,6 +27,7 @@ OPS_SYMBOLS = {
     "tpi_op_head_argmax": (_I, [_I, _P, _P, _P, _I, _I, _P, _P, _P, _P, _P, _P]),
     "tpi_op_gemm": (_I, [_I, _P, _LL, _I, _P, _LL, _P, _LL, _I, _I, _I, _I, _I, _P]),
     "tpi_op_gemm_bf16": (_I, [_P, _P, _I, _I, _P, _I, _P, _LL, _I, _I, _I, _I, _I, _P, _P]),
+    "tpi_op_gemm_bf16_starved": (_I, [_P, _I, _P, _P, _I, _I, _I, _I, _I, _P, _P]),
     "tpi_op_prefill_attention": (_I, [_I, _P, _P, _P, _I, _I, _I, _I, _I, _I, _P, _P]),
     "tpi_op_gemm_bf16_swiglu": (_I, [_P, _P, _I, _P, _P, _I, _I, _I, _I, _P, _P]),
     "tpi_op_gemm_bf16_rowsum": (_I, [_P, _P, _I, _I, _P, _I, _P, _I, _I, _I, _I, _I, _P, _P]),
@@ -113,6 +114,10 @@ def gemm(dtype, X, x_bs, ldx, W, w_bs, Y, y_bs, ldy, T, n_out, K, n_batch, strea
 
 def gemm_bf16(A, lda, a_col_batch, W, w_row_batch, Y, y_bs, ldy, T, n_out, K, n_batch, err_word, stream=None, A_lo=None):
     _check(_ops().tpi_op_gemm_bf16(A, A_lo, lda, a_col_batch, W, w_row_batch, Y, y_bs, ldy, T, n_out, K, n_batch, err_word, stream))
+
+
+def gemm_bf16_starved(A, lda, W, Y, ldy, T, n_out, K, wait_polls, err_word, stream=None):
+    _check(_ops().tpi_op_gemm_bf16_starved(A, lda, W, Y, ldy, T, n_out, K, wait_polls, err_word, stream))
 
 
 def gemm_bf16_swiglu(A, lda, Wgu, ACT, split_out, T, s, K, err_word, stream=None, A_lo=None):

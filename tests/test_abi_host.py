@@ -193,6 +193,33 @@ def test_ring_invariants():
             assert n_attn == w // 2 and len(kinds) - n_attn == (w + 1) // 2
 
 
+@pytest.mark.parametrize("w,T", [(1, 0), (2, 0), (3, 0), (4, 2), (8, 0)])
+def test_a_failed_block_copy_propagates_and_leaves_the_ring_consistent(w, T):
+    """Failure injection on the host: the back end's k-th block copy fails once (what a cudaMemcpyAsync error looks
+    like to the scheduler).  Without a retry the status comes back unchanged from wherever the loader was pumped
+    (start-up, a block's wait, a block's release).  With a retry the ring must carry on as if nothing had happened:
+    the copies, waits and releases are exactly those of a fault-free run, in the same order."""
+    n_blocks, n_exec = 12, 40
+    clean = P.ring_trace(n_blocks, w, n_exec, ffn_every_T=T)
+    n_copies = int((clean[:, 0] == 1).sum())
+    essential = lambda ops: [tuple(o) for o in ops if o[0] in (1, 2, 3, 4, 5)]
+    for k in list(range(0, min(n_copies, 30))) + [n_copies - 1]:
+        for status in (-6, -7):                                   # TPI_ERR_CUDA, TPI_ERR_TIMEOUT
+            with pytest.raises(P.TpiError) as e:
+                P.ring_trace_faulty(n_blocks, w, n_exec, k, status, False, ffn_every_T=T)
+            assert e.value.code == status
+        ops = P.ring_trace_faulty(n_blocks, w, n_exec, k, -6, True, ffn_every_T=T)
+        marks = [tuple(o) for o in ops if o[0] == 6]
+        assert len(marks) == 1 and marks[0][1] == -6             # seen once, with the injected status
+        assert essential(ops) == essential(clean)
+        # the retried load waits for its slot's release again, never less often than the fault-free run
+        assert int((ops[:, 0] == 0).sum()) >= int((clean[:, 0] == 0).sum())
+    # a copy index beyond the run never fires
+    assert essential(P.ring_trace_faulty(n_blocks, w, n_exec, 10 ** 6, -6, False, ffn_every_T=T)) == essential(clean)
+    with pytest.raises(P.TpiError):
+        P.ring_trace_faulty(n_blocks, w, n_exec, 0, 3, True)      # a failure needs a negative status
+
+
 # ----------------------------------------------------------------- steady-state diagnostics (Prop. 3, 4, 6)
 def test_steady_conditions_match_the_oracle_and_the_worked_example():
     # the paper's worked example: tight fails, loose holds, so no retention is needed
