@@ -100,6 +100,7 @@ def test_guard_zones_catch_a_write_past_a_buffer(monkeypatch):
     import paper_2410_00531_b200 as P
     shape = S.CONFIGS["C1"]
     toks = S.prompt_tokens(shape)
+    monkeypatch.delenv("TPI_DEBUG", raising=False)
     with gpu_session(shape, 64, 16, 2) as ses:
         plain_bytes = ses.dev.numel()
         t_ref, _ = P.prefill(ses.h, toks, 0)
