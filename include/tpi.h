@@ -238,8 +238,13 @@ int tpi_steady_conditions(double t_attn, double t_ffn, double t_all_reduce, doub
  * TPI_OPT_WAIT_DEADLINE_MS (value > 0: how long tpi_prefill / tpi_decode_* wait for the device
  * before they give up with TPI_ERR_TIMEOUT; default 900000, or TPI_WAIT_DEADLINE_S seconds from the
  * environment.  After a timeout the enqueued work still runs to its end on the device; the host
- * position is unchanged, and tpi_reset / tpi_set_position drain the stream and re-synchronise). */
-enum { TPI_OPT_GRAPH = 0, TPI_OPT_PDL = 1, TPI_OPT_PROFILE = 2, TPI_OPT_TENSOR = 3, TPI_OPT_WAIT_DEADLINE_MS = 4 };
+ * position is unchanged, and tpi_reset / tpi_set_position drain the stream and re-synchronise),
+ * TPI_OPT_ROWSHARD_FUSED (default 1: a decode step's row-sharded projections keep the N partial sums
+ * in registers and add them in rank order in the same kernel; 0: the partial sums go through memory
+ * and a second kernel adds them - the same residual bits, the form whose norm statistics a group of
+ * real ranks (tpi_tp.h) reproduces bit for bit). */
+enum { TPI_OPT_GRAPH = 0, TPI_OPT_PDL = 1, TPI_OPT_PROFILE = 2, TPI_OPT_TENSOR = 3, TPI_OPT_WAIT_DEADLINE_MS = 4,
+       TPI_OPT_ROWSHARD_FUSED = 5 };
 int tpi_set_option(tpi_model *m, int option, int value);
 
 /* Host-only test hook (needs no GPU): drives the window scheduler's ordering

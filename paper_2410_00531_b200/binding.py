@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtpi.so")
 
 TPI_F32, TPI_BF16 = 0, 1
-OPT_GRAPH, OPT_PDL, OPT_PROFILE, OPT_TENSOR, OPT_WAIT_DEADLINE_MS = 0, 1, 2, 3, 4
+OPT_GRAPH, OPT_PDL, OPT_PROFILE, OPT_TENSOR, OPT_WAIT_DEADLINE_MS, OPT_ROWSHARD_FUSED = 0, 1, 2, 3, 4, 5
 (T_EMB, T_HEAD, T_FINAL_NORM, T_ATTN_NORM, T_WQ, T_WK, T_WV, T_WO,
  T_FFN_NORM, T_WGATE, T_WUP, T_WDOWN) = range(12)
 

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libtpi.so")
-SOURCES = ["api.cu", "window.cu", "step_decode.cu", "step_prefill.cu", "inspect.cu", "ops.cu", "static_scratch.cu", "kernels_decode.cu", "kernels_prefill.cu", "gemm_tcgen05.cu", "gemm_tcgen05_pair.cu", "attn_prefill_mma.cu", "attn_prefill_tc.cu"]
+SOURCES = ["api.cu", "window.cu", "step_decode.cu", "step_prefill.cu", "inspect.cu", "ops.cu", "static_scratch.cu", "kernels_decode.cu", "kernels_prefill.cu", "gemm_tcgen05.cu", "gemm_tcgen05_pair.cu", "attn_prefill_mma.cu", "attn_prefill_tc.cu", "tp_kernels.cu", "step_tp.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC,-fopenmp,-O3", "--use_fast_math=false"]
 
@@ -17,7 +17,7 @@ def _stale() -> bool:
     if not os.path.exists(OUT):
         return True
     t = os.path.getmtime(OUT)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(HERE, "..", "include", f) for f in ("tpi.h", "tpi_ops.h")]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(HERE, "..", "include", f) for f in ("tpi.h", "tpi_ops.h", "tpi_tp.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 

@@ -558,6 +558,7 @@ extern "C" int tpi_set_option(tpi_model* m, int option, int value) {
     case TPI_OPT_GRAPH: m->opt_graph = value != 0; break;
     case TPI_OPT_PDL: m->opt_pdl = value != 0; break;
     case TPI_OPT_TENSOR: m->opt_tensor = value < 0 ? 0 : (value > 2 ? 2 : value); break;
+    case TPI_OPT_ROWSHARD_FUSED: m->opt_rowshard_fused = value != 0; break;
     case TPI_OPT_WAIT_DEADLINE_MS:
       if (value < 1) return fail(TPI_ERR_INVALID_ARG, "the wait deadline must be at least 1 ms");
       m->wait_deadline_s = value * 1e-3;

@@ -188,6 +188,31 @@ cudaError_t launch_rmsnorm_stat_row(const LaunchCtx& c, const float* xrow, int h
 void set_tuning(int key, int value);
 int get_tuning(int key);
 
+// ---------------------------------------------------------------- one shard per rank: the exchange kernels
+// Every rank has, in its own memory, a receive area recv[2][R][h] (fp32) and flags[2][R] (int): parity of the rank's
+// exchange counter x source rank.  Exchange number c (0-based, counted per rank in *epoch) uses parity c & 1; source j
+// stores its h values into every destination's recv[c & 1][j] and then flags[c & 1][j] = c + 1.
+constexpr int TP_MAX_RANKS = 16;
+struct TpPeers {
+  int n_ranks, rank;
+  float* recv[TP_MAX_RANKS];  // destination ranks' receive areas (this rank's own included)
+  int* flags[TP_MAX_RANKS];
+};
+// This rank's partial sums of a row-sharded projection, P[r] = W[r, :] . x_in (W [rows][Ks], the rank's own columns),
+// stored into every rank's receive area, then published.  Same per-row arithmetic as launch_gemv_partials.
+// ticket: unsigned, zero between launches.  drop != 0: compute but never publish (failure injection).
+cudaError_t launch_tp_rowpush(const LaunchCtx& c, int dt, const void* W, const float* x_in, int rows, int Ks, const int* epoch,
+                              unsigned* ticket, const TpPeers& peers, int drop);
+// The master's broadcast of the embedded hidden state: x[h] into every rank's recv[c & 1][0], then the flags.
+cudaError_t launch_tp_bcast(const LaunchCtx& c, const float* x, int h, const int* epoch, const TpPeers& peers, int drop);
+// The consumer: waits (at most wait_polls polls per flag) until all sources of exchange *epoch have published, then
+// mode 0: x <- ((P_0 + P_1) + ... + P_{R-1}) + x (rank order, shortcut last); mode 1: x <- P_0 (broadcast).
+// Also tap (may be null) <- x, xhat, ss_part[0] = sum of squares (zeros in [1, n_parts)), ++*epoch, and
+// (pos_advance != null) ++*pos_advance.  A wait that runs out sets DEVERR_WAIT_TIMEOUT in *err and changes nothing.
+cudaError_t launch_tp_recv(const LaunchCtx& c, const float* recv, const int* flags, int* epoch, int n_ranks, int h, int mode,
+                           float eps, float* x, float* xhat, float* tap, float* ss_part, int n_parts, int* pos_advance,
+                           int* err, int wait_polls);
+
 // Guard zones of a debug arena: up to 64 zones of 256 bytes at base + off[i].  fill writes the pattern, check compares
 // it and reports the first damaged zone as DEVERR_CANARY + i in *err (one CTA per zone, no other effect).
 struct CanaryList {

@@ -54,7 +54,7 @@ struct tpi_model {
   char* host = nullptr;
   cudaStream_t cs = nullptr, ps = nullptr;
   bool own_cs = false, own_ps = false;
-  int opt_graph = 1, opt_pdl = 1, opt_profile = 0, opt_tensor = 1;
+  int opt_graph = 1, opt_pdl = 1, opt_profile = 0, opt_tensor = 1, opt_rowshard_fused = 1;
   int position = 0;
   // window ring
   Ring ring;

@@ -37,7 +37,7 @@ static int enqueue_decode(tpi_model* m, LaunchCtx& lc) {
   auto rowshard = [&](const void* W, const float* xin, int Ks, const int* k0, float* tap) -> int {
     if (m->unequal) {
       CK(launch_gemv_rowshard_fused_unequal(lc, dt, W, xin, h, k0, N, x, ss_part, tap));
-    } else if (rowshard_fused_supported(Ks, N)) {
+    } else if (m->opt_rowshard_fused && rowshard_fused_supported(Ks, N)) {
       CK(launch_gemv_rowshard_fused(lc, dt, W, (size_t)h * Ks, xin, h, Ks, N, x, ss_part, tap));
     } else {  // very long shard slices: partial sums through memory, then the sum kernel
       CK(launch_gemv_partials(lc, dt, W, (size_t)h * Ks, xin, h, Ks, N, partials));

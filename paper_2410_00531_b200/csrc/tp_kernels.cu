@@ -1,0 +1,199 @@
+// Exchange kernels of the one-shard-per-rank form (Sec. 3.2's star allreduce in its one-hop shape): a rank stores its
+// partial sums into every rank's receive area with plain stores and then sets one flag per destination; the consumer
+// waits for the flags with a limit, adds the partial sums in rank order and the shortcut last.  Remote memory is only
+// ever WRITTEN, never read; nothing here is a multicast.
+#include "common.cuh"
+#include "gemv_bodies.cuh"
+#include "kernels.h"
+#include "launch.cuh"
+
+namespace tpi {
+
+namespace {
+
+__device__ __forceinline__ void st_release_sys(int* p, int v) {
+  asm volatile("st.release.sys.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_sys(const int* p) {
+  int v;
+  asm volatile("ld.acquire.sys.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+int sm_count_tp() {
+  int dev = 0, n = 0;
+  cudaGetDevice(&dev);
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+  return n;
+}
+
+struct RowPushArgs {
+  const void* W;  // [rows][Ks]
+  const float* x_in;
+  int rows, Ks, seg_cap, drop;
+  const int* epoch;
+  unsigned* ticket;
+  TpPeers peers;
+};
+
+// Persistent: one CTA per SM, x_in staged once, CTA `cta` owns rows [rows * cta / ncta, rows * (cta + 1) / ncta); its
+// partial sums are collected in shared memory and leave as contiguous runs, one run per destination rank.
+template <typename WT>
+__global__ void __launch_bounds__(1024) tp_rowpush_kernel(const RowPushArgs A) {
+  extern __shared__ __align__(16) float xs[];  // [Ks] staged inputs | [seg_cap] this CTA's partial sums
+  __shared__ bool s_last;
+  float* seg = xs + A.Ks;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const int cta = blockIdx.x, ncta = gridDim.x;
+  const int lo = (int)((long long)A.rows * cta / ncta), hi = (int)((long long)A.rows * (cta + 1) / ncta);
+  const WT* Wall = reinterpret_cast<const WT*>(A.W);
+  pdl_wait();  // x_in and the exchange counter come from the kernels before
+  pdl_launch_dependents();
+  for (int k = threadIdx.x * 4; k < A.Ks; k += blockDim.x * 4)
+    *reinterpret_cast<float4*>(xs + k) = *reinterpret_cast<const float4*>(A.x_in + k);
+  __syncthreads();
+  const int nvec = A.Ks / Elem<WT>::VEC;
+  for (int g = lo + warp; g < hi; g += nw) {
+    const uint4* wp[1] = {reinterpret_cast<const uint4*>(Wall + (size_t)g * A.Ks)};
+    float acc[1] = {0.f};
+    warp_dot<WT, 1>(wp, 0, xs, nvec, lane, acc);
+    const float p = warp_sum(acc[0]);
+    if (lane == 0) seg[g - lo] = p;
+  }
+  __syncthreads();
+  const int c = __ldcg(A.epoch), parity = c & 1, R = A.peers.n_ranks;
+  if (!A.drop) {
+    for (int j = 0; j < R; ++j) {
+      float* dst = A.peers.recv[j] + ((size_t)(parity * R + A.peers.rank) * A.rows + lo);
+      for (int i = threadIdx.x; i < hi - lo; i += blockDim.x) dst[i] = seg[i];
+    }
+  }
+  __threadfence_system();  // this CTA's stores are performed before its ticket
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned t = atomicAdd(A.ticket, 1u);
+    s_last = (t == (unsigned)ncta - 1);
+  }
+  __syncthreads();
+  if (s_last && threadIdx.x == 0) {  // every CTA's stores are out: publish
+    __threadfence_system();
+    if (!A.drop)
+      for (int j = 0; j < R; ++j) st_release_sys(A.peers.flags[j] + parity * R + A.peers.rank, c + 1);
+    *A.ticket = 0u;
+  }
+}
+
+__global__ void __launch_bounds__(1024) tp_bcast_kernel(const float* x, int h, const int* epoch, const TpPeers P, int drop) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int c = __ldcg(epoch), parity = c & 1, R = P.n_ranks;
+  if (drop) return;
+  for (int j = 0; j < R; ++j) {
+    float* dst = P.recv[j] + (size_t)(parity * R + 0) * h;
+    for (int k = threadIdx.x; k < h; k += blockDim.x) dst[k] = x[k];
+  }
+  __threadfence_system();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence_system();
+    for (int j = 0; j < R; ++j) st_release_sys(P.flags[j] + parity * R + 0, c + 1);
+  }
+}
+
+struct RecvArgs {
+  const float* recv;
+  const int* flags;
+  int* epoch;
+  int n_ranks, h, mode, n_parts, wait_polls;
+  float eps;
+  float *x, *xhat, *tap, *ss_part;
+  int* pos_advance;
+  int* err;
+};
+
+__global__ void __launch_bounds__(1024) tp_recv_kernel(const RecvArgs A) {
+  __shared__ float red[32];
+  __shared__ int s_ok;
+  pdl_wait();  // the counter was advanced by this rank's previous consumer
+  pdl_launch_dependents();
+  const int c = __ldcg(A.epoch), parity = c & 1, R = A.n_ranks;
+  const int n_src = A.mode == 1 ? 1 : R;
+  if (threadIdx.x == 0) s_ok = 1;
+  __syncthreads();
+  if ((int)threadIdx.x < n_src) {  // one thread per source; every wait has a limit
+    const int* f = A.flags + parity * R + threadIdx.x;
+    bool got = false;
+    for (int i = 0; i < A.wait_polls; ++i) {
+      if (ld_acquire_sys(f) == c + 1) { got = true; break; }
+      if (i > 64) __nanosleep(100);
+    }
+    if (!got) {
+      atomicCAS(A.err, DEVERR_NONE, DEVERR_WAIT_TIMEOUT);
+      s_ok = 0;
+    }
+  }
+  __syncthreads();
+  if (!s_ok) return;  // nothing is changed: the host sees the error word and resets the group
+  const float* P = A.recv + (size_t)parity * R * A.h;
+  float ss = 0.f;
+  for (int k = threadIdx.x; k < A.h; k += blockDim.x) {
+    float s = __ldcg(P + k);  // the master's own partial (rank 0) ...
+    if (A.mode == 0) {
+      for (int i = 1; i < R; ++i) s += __ldcg(P + (size_t)i * A.h + k);  // ... plus the workers', rank order
+      s += A.x[k];            // shortcut is added after the allreduce (Eq. 1-2)
+    }
+    A.x[k] = s;
+    if (A.tap) A.tap[k] = s;
+    ss = fmaf(s, s, ss);
+  }
+  ss = block_sum(ss, red);
+  const float r = rsqrtf(ss / (float)A.h + A.eps);
+  for (int k = threadIdx.x; k < A.h; k += blockDim.x) A.xhat[k] = A.x[k] * r;
+  for (int i = threadIdx.x; i < A.n_parts; i += blockDim.x) A.ss_part[i] = i ? 0.f : ss;
+  if (threadIdx.x == 0) {
+    *A.epoch = c + 1;
+    if (A.pos_advance) *A.pos_advance += 1;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_tp_rowpush(const LaunchCtx& c, int dt, const void* W, const float* x_in, int rows, int Ks, const int* epoch,
+                              unsigned* ticket, const TpPeers& peers, int drop) {
+  const int vec = dt == DT_BF16 ? 8 : 4;
+  if (rows < 1 || Ks < vec || Ks % vec || peers.n_ranks < 1 || peers.n_ranks > TP_MAX_RANKS) return cudaErrorInvalidValue;
+  int grid = sm_count_tp();
+  if (grid > rows) grid = rows;
+  const int per = (rows + grid - 1) / grid;
+  int warps = per < 32 ? per : 32;
+  if (warps < 4) warps = 4;
+  RowPushArgs A{W, x_in, rows, Ks, per + 1, drop, epoch, ticket, peers};
+  const size_t smem = ((size_t)Ks + per + 1) * sizeof(float);
+  if (smem > 200 * 1024) return cudaErrorInvalidValue;
+  auto go = [&](auto wt) -> cudaError_t {
+    using WT = decltype(wt);
+    auto kern = tp_rowpush_kernel<WT>;
+    static PerDeviceOnce attr_done;
+    if (!attr_done.get()) {
+      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+      if (e != cudaSuccess) return e;
+      attr_done.set();
+    }
+    return launch_kernel(c, kern, dim3(grid), dim3(warps * 32), smem, A);
+  };
+  return dt == DT_BF16 ? go(__nv_bfloat16{}) : go(float{});
+}
+
+cudaError_t launch_tp_bcast(const LaunchCtx& c, const float* x, int h, const int* epoch, const TpPeers& peers, int drop) {
+  return launch_kernel(c, tp_bcast_kernel, dim3(1), dim3(1024), 0, x, h, epoch, peers, drop);
+}
+
+cudaError_t launch_tp_recv(const LaunchCtx& c, const float* recv, const int* flags, int* epoch, int n_ranks, int h, int mode,
+                           float eps, float* x, float* xhat, float* tap, float* ss_part, int n_parts, int* pos_advance,
+                           int* err, int wait_polls) {
+  if (n_ranks < 1 || n_ranks > TP_MAX_RANKS || wait_polls < 1 || !err) return cudaErrorInvalidValue;
+  RecvArgs A{recv, flags, epoch, n_ranks, h, mode, n_parts, wait_polls, eps, x, xhat, tap, ss_part, pos_advance, err};
+  return launch_kernel(c, tp_recv_kernel, dim3(1), dim3(1024), 0, A);
+}
+
+}  // namespace tpi

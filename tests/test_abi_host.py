@@ -20,7 +20,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 def declared_functions():
     names = []
-    for hdr in ("tpi.h", "tpi_ops.h"):
+    for hdr in ("tpi.h", "tpi_ops.h", "tpi_tp.h"):
         src = open(os.path.join(ROOT, "include", hdr)).read()
         src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
         names += re.findall(r"\b(tpi_[a-z0-9_]+)\s*\(", src)
@@ -33,7 +33,8 @@ def test_library_exports_every_declared_symbol():
     assert len(decl) >= 30
     for name in decl:
         assert hasattr(lib, name), f"{name} declared in include/ but not exported"
-    bound = set(P.binding.SYMBOLS) | set(K.OPS_SYMBOLS)
+    import paper_2410_00531_b200.tp as TP
+    bound = set(P.binding.SYMBOLS) | set(K.OPS_SYMBOLS) | set(TP.TP_SYMBOLS)
     assert set(decl) <= bound, set(decl) - bound
 
 
