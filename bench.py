@@ -381,6 +381,49 @@ def streamed_leg(P, name, shape, local, K, W, window, link_peak, retain=0):
             "clocks": r["clocks"], "load_s": round(load_s, 1)}
 
 
+def tp_one_gpu_leg(P, shape, local, R, K, W):
+    """The one-shard-per-rank form with all R ranks on THIS GPU (they take turns on it; every exchange is ordered by
+    events): shows that the path runs at the workload's full size and what its launch sequence costs when nothing runs
+    in parallel.  Not a multi-GPU measurement."""
+    import torch
+    import paper_2410_00531_b200.tp as TP
+    T = shape.prompt_len
+    cfg = tpi_config(shape, T + W + K + 8, T)
+    t0 = time.perf_counter()
+    g = TP.Group(cfg, S.synth_fill(shape), R, 0, device=local)
+    load_s = time.perf_counter() - t0
+    try:
+        toks = S.prompt_tokens(shape)
+        g.prefill(toks, 0)
+        g.reset()
+        t0 = time.perf_counter()
+        first, _ = g.prefill(toks, 0)
+        ttft_ms = (time.perf_counter() - t0) * 1e3
+        tok = int(g.decode_run(first, W)[-1])
+        sampler = ClockSampler(local)
+        sampler.start()
+        time.sleep(0.5)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        out = g.decode_run(tok, K)
+        torch.cuda.synchronize()
+        wall = time.perf_counter() - t0
+        clocks = sampler.stop()
+        st = g.stats()
+    finally:
+        g.close()
+        import gc
+        gc.collect()
+        torch.cuda.empty_cache()
+    return {"workload": f"{shape.name}: {R} ranks with one shard each, ALL ON ONE GPU (time-shared, events between streams; "
+                        "functional, not a multi-GPU number)", "steps": K, "warmup": W,
+            "tokens_per_s": round(K / wall, 2), "ms_per_step": round(wall / K * 1e3, 3), "ttft_ms": round(ttft_ms, 2),
+            "ttft_prompt_tokens": T, "kernel_launches_per_token": st["kernel_launches_last"] // K,
+            "exchange_bytes_per_token_per_rank": st["exchange_bytes_per_token"],
+            "weight_bytes_per_token_worker": st["weight_bytes_worker"], "tokens_tail": [int(x) for x in out[-2:]],
+            "clocks": clocks, "load_s": round(load_s, 1)}
+
+
 def extra_legs(P, args, local):
     """The other listed workloads, measured in the same process after the headline: the 8B shape at its 4096-token
     context and the 70B shape, both resident; then the window-streamed path on 70B-shaped blocks, bf16 and fp32, at a
@@ -403,6 +446,8 @@ def extra_legs(P, args, local):
         run("C3", lambda: resident_leg(P, "C3", S.CONFIGS["C3"], local, 256, 5, args.prefill_chunk))
     if "C5" in want:
         run("C5", lambda: resident_leg(P, "C5", S.CONFIGS["C5"], local, 32, 4, args.prefill_chunk))
+    if "TP" in want:
+        run("C2_4_ranks_one_gpu", lambda: tp_one_gpu_leg(P, S.CONFIGS["C2"], local, 4, 32, 4))
     if "S5" in want or "S4" in want:
         link_peak = host_link_peak(torch, local)
         if "S5" in want:
@@ -562,9 +607,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C2", choices=sorted(S.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--legs", default="C3,C5,S5,S4",
+    ap.add_argument("--legs", default="C3,C5,TP,S5,S4",
                     help="extra workloads measured after the default headline and reported under `legs` (C3, C5: resident; "
-                         "S5, S4: 70B-shaped bf16 / fp32 blocks window-streamed); empty string = none")
+                         "TP: the 7B shape as 4 ranks with one shard each on this one GPU; S5, S4: 70B-shaped bf16 / fp32 "
+                         "blocks window-streamed); empty string = none")
     ap.add_argument("--retain", type=int, default=0,
                     help="with --window: keep one FFN block in every T resident beside the window (0 = none, -1 = as many as fit)")
     ap.add_argument("--window", type=int, default=0,

@@ -35,8 +35,11 @@
  * group of R ranks gives the same bits as an emulated model with N = R shards
  * run with TPI_OPT_ROWSHARD_FUSED = 0.
  *
- * The prompt is fed one position at a time through the decode kernels (the
- * batched prompt pass of tpi.h is not part of this form yet).
+ * A prompt is processed in chunks of up to cfg.max_prefill positions per pass
+ * over the weights, with the kernels of tpi.h's prompt pass on every rank's
+ * slices; the partial sums of a chunk (positions x hidden, fp32) travel the same
+ * way.  TPI_TP_OPT_BATCHED_PROMPT = 0 feeds the prompt one position at a time
+ * through the decode kernels instead.
  */
 #ifndef TPI_TP_H
 #define TPI_TP_H
@@ -101,8 +104,9 @@ int tpi_tp_get_kv(tpi_tp_group *g, int layer, int kv_head, int pos0, int n, floa
  * never publishes them (a rank that "never joins"); the other ranks' waits then
  * run out and the call returns TPI_ERR_TIMEOUT; one-shot, 0 clears it.
  * TPI_TP_OPT_PDL: programmatic dependent launch between a rank's kernels
- * (default 1). */
-enum { TPI_TP_OPT_EVENTS = 0, TPI_TP_OPT_WAIT_POLLS = 1, TPI_TP_OPT_DROP_PUSH = 2, TPI_TP_OPT_PDL = 3 };
+ * (default 1).  TPI_TP_OPT_BATCHED_PROMPT (default 1): see above. */
+enum { TPI_TP_OPT_EVENTS = 0, TPI_TP_OPT_WAIT_POLLS = 1, TPI_TP_OPT_DROP_PUSH = 2, TPI_TP_OPT_PDL = 3,
+       TPI_TP_OPT_BATCHED_PROMPT = 4 };
 int tpi_tp_set_option(tpi_tp_group *g, int option, int value);
 
 typedef struct {

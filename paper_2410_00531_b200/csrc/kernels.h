@@ -189,12 +189,15 @@ void set_tuning(int key, int value);
 int get_tuning(int key);
 
 // ---------------------------------------------------------------- one shard per rank: the exchange kernels
-// Every rank has, in its own memory, a receive area recv[2][R][h] (fp32) and flags[2][R] (int): parity of the rank's
-// exchange counter x source rank.  Exchange number c (0-based, counted per rank in *epoch) uses parity c & 1; source j
-// stores its h values into every destination's recv[c & 1][j] and then flags[c & 1][j] = c + 1.
+// Every rank has, in its own memory, a receive area of two halves of `half` floats each (fp32) and flags[2][R] (int):
+// parity of the rank's exchange counter, then the R sources side by side, n floats each (n = h for a decode step,
+// T * h for a prompt pass of T positions; R * n <= half).  Exchange number c (0-based, counted per rank in *epoch)
+// uses parity c & 1; source j stores its n values at recv + (c & 1) * half + j * n of every destination and then sets
+// flags[c & 1][j] = c + 1.
 constexpr int TP_MAX_RANKS = 16;
 struct TpPeers {
   int n_ranks, rank;
+  long long half;             // floats per parity half of a receive area
   float* recv[TP_MAX_RANKS];  // destination ranks' receive areas (this rank's own included)
   int* flags[TP_MAX_RANKS];
 };
@@ -209,9 +212,15 @@ cudaError_t launch_tp_bcast(const LaunchCtx& c, const float* x, int h, const int
 // mode 0: x <- ((P_0 + P_1) + ... + P_{R-1}) + x (rank order, shortcut last); mode 1: x <- P_0 (broadcast).
 // Also tap (may be null) <- x, xhat, ss_part[0] = sum of squares (zeros in [1, n_parts)), ++*epoch, and
 // (pos_advance != null) ++*pos_advance.  A wait that runs out sets DEVERR_WAIT_TIMEOUT in *err and changes nothing.
-cudaError_t launch_tp_recv(const LaunchCtx& c, const float* recv, const int* flags, int* epoch, int n_ranks, int h, int mode,
-                           float eps, float* x, float* xhat, float* tap, float* ss_part, int n_parts, int* pos_advance,
+cudaError_t launch_tp_recv(const LaunchCtx& c, const float* recv, long long half, const int* flags, int* epoch, int n_ranks, int h,
+                           int mode, float eps, float* x, float* xhat, float* tap, float* ss_part, int n_parts, int* pos_advance,
                            int* err, int wait_polls);
+// Prompt pass: n floats of src (T x h partial sums, or the embedded rows with as_rank0 != 0) into every rank's slot of
+// this source, then the flags; and the consumer's wait alone (n_src sources, 1 for the broadcast), which also advances
+// the counter, so that the ordinary row kernels can read the receive area afterwards.
+cudaError_t launch_tp_push_rows(const LaunchCtx& c, const float* src, size_t n, const int* epoch, unsigned* ticket,
+                                const TpPeers& peers, int as_rank0, int drop);
+cudaError_t launch_tp_wait(const LaunchCtx& c, const int* flags, int* epoch, int n_ranks, int n_src, int* err, int wait_polls);
 
 // Guard zones of a debug arena: up to 64 zones of 256 bytes at base + off[i].  fill writes the pattern, check compares
 // it and reports the first damaged zone as DEVERR_CANARY + i in *err (one CTA per zone, no other effect).

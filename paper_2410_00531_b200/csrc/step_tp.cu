@@ -28,7 +28,10 @@ struct TpRank {
   cudaEvent_t ev_push = nullptr, ev_done = nullptr;
 };
 
-size_t tp_tail_bytes(const tpi_config& c, int R) { return align_up((size_t)2 * R * c.hidden * 4, 256) + 3 * 256; }
+// floats of one parity half of a rank's receive area: R sources x (one position's hidden state for a decode step, up
+// to max_prefill positions for a prompt pass)
+size_t tp_half_floats(const tpi_config& c, int R) { return (size_t)R * c.max_prefill * c.hidden; }
+size_t tp_tail_bytes(const tpi_config& c, int R) { return align_up((size_t)2 * tp_half_floats(c, R) * 4, 256) + 3 * 256; }
 
 int slice_of(const tpi_config& c, int R, int rank, int tid, int64_t* row0, int64_t* n_rows, int64_t* col0, int64_t* n_cols) {
   if (R < 1 || R > TPI_TP_MAX_RANKS || rank < 0 || rank >= R) return fail(TPI_ERR_INVALID_ARG, "rank %d of %d", rank, R);
@@ -86,7 +89,6 @@ tpi_config local_cfg(const tpi_config& c, int R, int rank) {
   l.n_kv_heads = c.n_kv_heads / R;
   l.ffn = c.ffn / R;
   if (rank != 0) l.vocab = 1;  // workers hold no embedding and no head (Sec. 3.1: they reside on the master)
-  l.max_prefill = 1;           // the prompt goes through the decode kernels, one position at a time
   return l;
 }
 
@@ -96,7 +98,7 @@ struct tpi_tp_group {
   tpi_config cfg{};
   int R = 0, window = 0;
   std::vector<TpRank> ranks;
-  int events = 1, wait_polls = 1 << 21, drop_rank = -1, pdl = 1;
+  int events = 1, wait_polls = 1 << 21, drop_rank = -1, pdl = 1, batched_prompt = 1;
   int position = 0, launches_last = 0;
   bool broken = false;  // a call failed or timed out: tpi_tp_reset first
   uint64_t exchanges = 0;
@@ -115,6 +117,7 @@ TpPeers peers_of(const tpi_tp_group* g, int rank) {
   TpPeers P{};
   P.n_ranks = g->R;
   P.rank = rank;
+  P.half = (long long)tp_half_floats(g->cfg, g->R);
   for (int j = 0; j < g->R; ++j) { P.recv[j] = g->ranks[j].recv; P.flags[j] = g->ranks[j].flags; }
   return P;
 }
@@ -153,7 +156,7 @@ int enqueue_step(tpi_tp_group* g, bool with_head, int* launches) {
       LaunchCtx lc = ctx(r);
       float* tap = layer_tap >= 0 ? dptr<float>(m, p.taps) + (size_t)layer_tap * h : nullptr;
       const bool adv = advance_workers && !(i == 0 && with_head);
-      CK(launch_tp_recv(lc, r.recv, r.flags, r.epoch, R, h, mode, c.rms_eps, dptr<float>(m, p.x), dptr<float>(m, p.xhat), tap,
+      CK(launch_tp_recv(lc, r.recv, (long long)tp_half_floats(c, R), r.flags, r.epoch, R, h, mode, c.rms_eps, dptr<float>(m, p.x), dptr<float>(m, p.xhat), tap,
                         dptr<float>(m, p.ss_part), rowshard_fused_parts(h), adv ? dptr<int>(m, p.pos) : nullptr,
                         dptr<int>(m, p.err), g->wait_polls));
     }
@@ -217,6 +220,214 @@ int enqueue_step(tpi_tp_group* g, bool with_head, int* launches) {
                           h, c.vocab, dptr<float>(m, p.logits), dptr<float>(m, p.amax_val), dptr<int>(m, p.amax_idx),
                           dptr<unsigned>(m, p.tickets) + bl_, dptr<int>(m, p.tok_hist), dptr<int>(m, p.pos), 1));
   }
+  return TPI_OK;
+}
+
+// T prompt positions [pos0, pos0 + T) through all ranks at once (enqueue only): Algorithm 1's loop body with T
+// positions per rank, every rank on its own heads and FFN columns.  The row-sharded projections leave T x h partial
+// sums per rank, which go to every rank's receive area (tp_push_rows_kernel); the consumer is the wait kernel followed
+// by the ordinary row kernel that adds R partial sums in rank order and the shortcut (and applies the next RMSNorm).
+// The host addresses the receive area by the parity of its own exchange count, which equals the device counter as long
+// as no wait ran out (after one, the call fails and tpi_tp_reset puts both back to zero).
+int enqueue_prompt_chunk(tpi_tp_group* g, int pos0, int T, bool last, int* launches) {
+  const tpi_config& c = g->cfg;
+  const int R = g->R, h = c.hidden, d = c.head_dim, dt = c.dtype, L = c.n_layers;
+  const int al = c.n_heads / R, bl_ = c.n_kv_heads / R, sl = c.ffn / R;
+  const int qkv_cols = (al + 2 * bl_) * d;
+  const size_t half = tp_half_floats(c, R);
+  auto ctx = [&](TpRank& r) { return LaunchCtx{r.m->cs, g->pdl != 0, launches}; };
+  auto drop_now = [&](int rank) {
+    if (g->drop_rank != rank) return 0;
+    g->drop_rank = -1;
+    return 1;
+  };
+  const bool tc = dt == TPI_BF16 && g->ranks[0].m->opt_tensor && gemm_tc_supported(h, h, qkv_cols) && gemm_tc_supported(h, h, 2 * sl) &&
+                  gemm_tc_supported(al * d, al * d, h) && gemm_tc_supported(sl, sl, h);
+  const int act_mode = tc ? 2 : 0;  // split bf16 activations on the tensor cores, fp32 otherwise
+  const bool fuse_norm = g->window <= 0;  // a streamed rank may not hold the next block's gain yet
+  auto gemm = [&](TpRank& r, LaunchCtx& lc, const float* A, int lda, const void* W, float* Y, int ldy, int n_out, int K) -> int {
+    if (tc) {
+      const __nv_bfloat16* hi = reinterpret_cast<const __nv_bfloat16*>(A);
+      CK(launch_gemm_tc(lc, hi, hi + (size_t)T * lda, lda, 0, W, n_out, Y, 0, ldy, T, n_out, K, 1, dptr<int>(r.m, r.m->plan.err)));
+    } else {
+      CK(launch_gemm_simt(lc, dt, A, 0, lda, W, 0, Y, 0, ldy, T, n_out, K, 1));
+    }
+    return TPI_OK;
+  };
+  // every rank waits for `n_src` sources of the current exchange; returns the receive parity in *parity
+  auto wait_all = [&](int n_src) -> int {
+    for (int i = 0; i < R; ++i) {
+      TpRank& r = g->ranks[i];
+      CK(cudaSetDevice(r.device));
+      if (g->events)
+        for (int j = 0; j < (n_src == 1 ? 1 : R); ++j)
+          if (j != i) CK(cudaStreamWaitEvent(r.m->cs, g->ranks[j].ev_push, 0));
+      LaunchCtx lc = ctx(r);
+      CK(launch_tp_wait(lc, r.flags, r.epoch, R, n_src, dptr<int>(r.m, r.m->plan.err), g->wait_polls));
+    }
+    return TPI_OK;
+  };
+  // ---- the master embeds the T tokens and sends the rows to every rank
+  {
+    TpRank& r = g->ranks[0];
+    tpi_model* m = r.m;
+    const Plan& p = m->plan;
+    CK(cudaSetDevice(r.device));
+    LaunchCtx lc = ctx(r);
+    CK(launch_embed_rows(lc, dt, m->dev + p.emb, dptr<int>(m, p.tok_hist), pos0, T, c.vocab, h, dptr<float>(m, p.pX), dptr<int>(m, p.err)));
+    CK(launch_tp_push_rows(lc, dptr<float>(m, p.pX), (size_t)T * h, r.epoch, r.ticket, peers_of(g, 0), 1, drop_now(0)));
+    if (g->events) CK(cudaEventRecord(r.ev_push, m->cs));
+  }
+  {
+    const int parity = (int)(g->exchanges & 1);
+    TRY(wait_all(1));
+    for (int i = 1; i < R; ++i) {  // the workers take the rows out of the master's slot
+      TpRank& r = g->ranks[i];
+      CK(cudaSetDevice(r.device));
+      CK(cudaMemcpyAsync(dptr<float>(r.m, r.m->plan.pX), r.recv + (size_t)parity * half, (size_t)T * h * 4,
+                         cudaMemcpyDeviceToDevice, r.m->cs));
+    }
+    ++g->exchanges;
+  }
+  std::vector<char> normed(R, 0);  // Xn already holds the input of the block about to start
+  for (int l = 0; l < L; ++l) {
+    for (int blk = 0; blk < 2; ++blk) {
+      for (int i = 0; i < R; ++i) {
+        TpRank& r = g->ranks[i];
+        tpi_model* m = r.m;
+        const Plan& p = m->plan;
+        const BlockLayout& bl = p.bl;
+        CK(cudaSetDevice(r.device));
+        LaunchCtx lc = ctx(r);
+        float *X = dptr<float>(m, p.pX), *Xn = dptr<float>(m, p.pXn), *PART = dptr<float>(m, p.pPART);
+        BlockRef br;
+        TRY(acquire_block(m, 2 * l + blk, &br));
+        if (!normed[i]) CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, act_mode));
+        if (blk == 0) {
+          float *QKV = dptr<float>(m, p.pQKV), *Q = dptr<float>(m, p.pQ), *O = dptr<float>(m, p.pO);
+          void* kc = m->dev + p.kcache + (size_t)l * p.kv_layer_bytes;
+          void* vc = m->dev + p.vcache + (size_t)l * p.kv_layer_bytes;
+          TRY(gemm(r, lc, Xn, h, br.base + bl.off_qkv, QKV, qkv_cols, qkv_cols, h));
+          CK(launch_rope_kv_rows(lc, dt, QKV, T, pos0, 1, al, bl_, d, c.max_seq, dptr<float2>(m, p.rope), Q, kc, vc));
+          if (m->opt_tensor && prefill_attention_tc_supported(dt, d, T))
+            CK(launch_prefill_attention_tc(lc, Q, kc, vc, T, pos0, al, bl_, c.max_seq, O, act_mode, dptr<int>(m, p.err)));
+          else if (m->opt_tensor && prefill_attention_mma_supported(dt, d))
+            CK(launch_prefill_attention_mma(lc, Q, kc, vc, T, pos0, al, bl_, d, c.max_seq, O, act_mode));
+          else
+            CK(launch_prefill_attention(lc, dt, Q, kc, vc, T, pos0, al, bl_, d, c.max_seq, O, act_mode));
+          TRY(gemm(r, lc, O, al * d, br.base + bl.off_wo, PART, h, h, al * d));
+        } else {
+          float *GU = dptr<float>(m, p.pGU), *ACT = dptr<float>(m, p.pACT);
+          if (tc && gemm_tc_swiglu_supported(h, h, sl)) {
+            const __nv_bfloat16* hi = reinterpret_cast<const __nv_bfloat16*>(Xn);
+            CK(launch_gemm_tc_swiglu(lc, hi, hi + (size_t)T * h, h, br.base + bl.off_gu, ACT, act_mode, T, sl, h, dptr<int>(m, p.err)));
+          } else {
+            TRY(gemm(r, lc, Xn, h, br.base + bl.off_gu, GU, 2 * sl, 2 * sl, h));
+            CK(launch_swiglu_rows(lc, GU, T, sl, ACT, act_mode));
+          }
+          TRY(gemm(r, lc, ACT, sl, br.base + bl.off_down, PART, h, h, sl));
+        }
+        CK(launch_tp_push_rows(lc, PART, (size_t)T * h, r.epoch, r.ticket, peers_of(g, i), 0, drop_now(i)));
+        TRY(release_block(m, 2 * l + blk));
+        if (g->events) CK(cudaEventRecord(r.ev_push, m->cs));
+      }
+      const int parity = (int)(g->exchanges & 1);
+      TRY(wait_all(R));
+      const bool more = !(l == L - 1 && blk == 1);
+      for (int i = 0; i < R; ++i) {  // ((P_0 + P_1) + ...) + X for T rows, and the next block's norm where its gain is at hand
+        TpRank& r = g->ranks[i];
+        tpi_model* m = r.m;
+        const Plan& p = m->plan;
+        CK(cudaSetDevice(r.device));
+        LaunchCtx lc = ctx(r);
+        const float* parts = r.recv + (size_t)parity * half;  // [R][T][h]: source j's rows at j * T * h
+        float* tap = last ? dptr<float>(m, p.taps) + (size_t)(2 * l + blk) * h : nullptr;
+        normed[i] = fuse_norm && more;
+        if (normed[i])
+          CK(launch_reduce_residual_norm_rows(lc, parts, R, T, h, dptr<float>(m, p.pX), tap, (const float*)resident_block(m, 2 * l + blk + 1),
+                                              c.rms_eps, dptr<float>(m, p.pXn), act_mode));
+        else
+          CK(launch_reduce_residual_rows(lc, parts, R, T, h, dptr<float>(m, p.pX), tap));
+      }
+      ++g->exchanges;
+    }
+  }
+  if (last) {
+    TpRank& r = g->ranks[0];
+    tpi_model* m = r.m;
+    const Plan& p = m->plan;
+    CK(cudaSetDevice(r.device));
+    LaunchCtx lc = ctx(r);
+    const int n_parts = rowshard_fused_parts(h);
+    CK(launch_rmsnorm_stat_row(lc, dptr<float>(m, p.pX) + (size_t)(T - 1) * h, h, c.rms_eps, dptr<float>(m, p.x), dptr<float>(m, p.xhat),
+                               dptr<float>(m, p.ss_part), n_parts, dptr<int>(m, p.pos), pos0 + T - 1));
+    CK(launch_head_argmax(lc, dt, m->dev + p.head,
+                          NormIn{dptr<float>(m, p.x), dptr<float>(m, p.final_gain), dptr<float>(m, p.ss_part), n_parts, c.rms_eps}, h,
+                          c.vocab, dptr<float>(m, p.logits), dptr<float>(m, p.amax_val), dptr<int>(m, p.amax_idx),
+                          dptr<unsigned>(m, p.tickets) + bl_, dptr<int>(m, p.tok_hist), dptr<int>(m, p.pos), 1));
+  }
+  return TPI_OK;
+}
+
+// The prompt in chunks of max_prefill positions through enqueue_prompt_chunk.
+int run_prompt(tpi_tp_group* g, const int32_t* tokens, int n, int32_t* first, float* logits) {
+  if (g->broken) return fail(TPI_ERR_STATE, "an earlier call failed or timed out: call tpi_tp_reset first");
+  const tpi_config& c = g->cfg;
+  if (g->position + n > c.max_seq) return fail(TPI_ERR_SEQ_OVERFLOW, "position %d + %d exceeds max_seq %d", g->position, n, c.max_seq);
+  for (int i = 0; i < n; ++i)
+    if (tokens[i] < 0 || tokens[i] >= c.vocab) return fail(TPI_ERR_TOKEN_RANGE, "token %d outside [0, %d)", tokens[i], c.vocab);
+  DeviceGuard guard;
+  const auto w0 = std::chrono::steady_clock::now();
+  tpi_model* m0 = g->ranks[0].m;
+  int* io0 = (int*)(m0->host + m0->plan.h_io);
+  int launches = 0;
+  g->broken = true;
+  const int p_begin = g->position;
+  for (int t0 = 0; t0 < n; t0 += c.max_prefill) {
+    const int T = n - t0 < c.max_prefill ? n - t0 : c.max_prefill;
+    CK(cudaSetDevice(g->ranks[0].device));
+    if (t0) TRY(wait_event(m0, g->ranks[0].ev_done));  // the pinned token area is free again
+    memcpy(io0 + 3, tokens + t0, (size_t)T * 4);
+    CK(cudaMemcpyAsync(dptr<int>(m0, m0->plan.tok_hist) + p_begin + t0, io0 + 3, (size_t)T * 4, cudaMemcpyHostToDevice, m0->cs));
+    CK(cudaEventRecord(g->ranks[0].ev_done, m0->cs));
+    TRY(enqueue_prompt_chunk(g, p_begin + t0, T, t0 + T == n, &launches));
+  }
+  for (int i = 1; i < g->R; ++i) {  // the workers' position counters (the master's was set by its head)
+    TpRank& r = g->ranks[i];
+    int* io = (int*)(r.m->host + r.m->plan.h_io);
+    io[0] = p_begin + n;
+    CK(cudaSetDevice(r.device));
+    CK(cudaMemcpyAsync(r.m->dev + r.m->plan.pos, io, 4, cudaMemcpyHostToDevice, r.m->cs));
+  }
+  CK(cudaSetDevice(g->ranks[0].device));
+  CK(cudaMemcpyAsync(io0 + 2, dptr<int>(m0, m0->plan.tok_hist) + p_begin + n, 4, cudaMemcpyDeviceToHost, m0->cs));
+  if (logits) CK(cudaMemcpyAsync(m0->host + m0->plan.h_logits, m0->dev + m0->plan.logits, (size_t)c.vocab * 4, cudaMemcpyDeviceToHost, m0->cs));
+  for (int i = 0; i < g->R; ++i) {
+    TpRank& r = g->ranks[i];
+    int* io = (int*)(r.m->host + r.m->plan.h_io);
+    CK(cudaSetDevice(r.device));
+    CK(cudaMemcpyAsync(io + 1, r.m->dev + r.m->plan.err, 4, cudaMemcpyDeviceToHost, r.m->cs));
+    CK(cudaEventRecord(r.ev_done, r.m->cs));
+  }
+  for (int i = 0; i < g->R; ++i) {
+    CK(cudaSetDevice(g->ranks[i].device));
+    TRY(wait_event(g->ranks[i].m, g->ranks[i].ev_done));
+  }
+  for (int i = 0; i < g->R; ++i) {
+    const int code = ((int*)(g->ranks[i].m->host + g->ranks[i].m->plan.h_io))[1];
+    if (code == DEVERR_NONE) continue;
+    if (code == DEVERR_WAIT_TIMEOUT)
+      return fail(TPI_ERR_TIMEOUT, "rank %d gave up waiting for another rank's partial sums (bounded wait ran out); call tpi_tp_reset", i);
+    if (code == DEVERR_TOKEN_RANGE) return fail(TPI_ERR_TOKEN_RANGE, "a token id was outside [0, vocab)");
+    return fail(TPI_ERR_DEVICE_CHECK, "rank %d: device error word = %d", i, code);
+  }
+  g->broken = false;
+  g->position = p_begin + n;
+  for (auto& r : g->ranks) r.m->position = g->position;
+  *first = io0[2];
+  if (logits) memcpy(logits, m0->host + m0->plan.h_logits, (size_t)c.vocab * 4);
+  g->launches_last = launches;
+  g->last_decode_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - w0).count();
   return TPI_OK;
 }
 
@@ -352,7 +563,7 @@ extern "C" int tpi_tp_create(const tpi_config* cfg, int n_ranks, const tpi_resou
     r.rf.tmp.clear();
     r.rf.tmp.shrink_to_fit();
     r.recv = (float*)r.tail;
-    char* t = r.tail + align_up((size_t)2 * n_ranks * cfg->hidden * 4, 256);
+    char* t = r.tail + align_up((size_t)2 * tp_half_floats(*cfg, n_ranks) * 4, 256);
     r.flags = (int*)t;
     r.epoch = (int*)(t + 256);
     r.ticket = (unsigned*)(t + 512);
@@ -368,6 +579,7 @@ extern "C" int tpi_tp_create(const tpi_config* cfg, int n_ranks, const tpi_resou
 
 extern "C" int tpi_tp_prefill(tpi_tp_group* g, const int32_t* tokens, int n_tokens, int32_t* first_token, float* logits_or_null) {
   if (!g || !tokens || n_tokens < 1 || !first_token) return fail(TPI_ERR_INVALID_ARG, "bad argument");
+  if (g->batched_prompt) return run_prompt(g, tokens, n_tokens, first_token, logits_or_null);
   return run_positions(g, tokens, n_tokens, n_tokens, false, first_token, 1, logits_or_null);
 }
 extern "C" int tpi_tp_decode_step(tpi_tp_group* g, int32_t token_in, int32_t* token_out, float* logits_or_null) {
@@ -396,6 +608,7 @@ extern "C" int tpi_tp_reset(tpi_tp_group* g) {
     TRY(write_position(r.m, 0));
   }
   g->position = 0;
+  g->exchanges = 0;
   g->broken = false;
   g->drop_rank = -1;
   return TPI_OK;
@@ -436,6 +649,7 @@ extern "C" int tpi_tp_set_option(tpi_tp_group* g, int option, int value) {
       g->drop_rank = value - 1;
       return TPI_OK;
     case TPI_TP_OPT_PDL: g->pdl = value != 0; return TPI_OK;
+    case TPI_TP_OPT_BATCHED_PROMPT: g->batched_prompt = value != 0; return TPI_OK;
     default: return fail(TPI_ERR_INVALID_ARG, "unknown option %d", option);
   }
 }

@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(1024) tp_rowpush_kernel(const RowPushArgs A) {
   const int c = __ldcg(A.epoch), parity = c & 1, R = A.peers.n_ranks;
   if (!A.drop) {
     for (int j = 0; j < R; ++j) {
-      float* dst = A.peers.recv[j] + ((size_t)(parity * R + A.peers.rank) * A.rows + lo);
+      float* dst = A.peers.recv[j] + ((size_t)parity * A.peers.half + (size_t)A.peers.rank * A.rows + lo);
       for (int i = threadIdx.x; i < hi - lo; i += blockDim.x) dst[i] = seg[i];
     }
   }
@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(1024) tp_bcast_kernel(const float* x, int h, c
   const int c = __ldcg(epoch), parity = c & 1, R = P.n_ranks;
   if (drop) return;
   for (int j = 0; j < R; ++j) {
-    float* dst = P.recv[j] + (size_t)(parity * R + 0) * h;
+    float* dst = P.recv[j] + (size_t)parity * P.half;  // source 0
     for (int k = threadIdx.x; k < h; k += blockDim.x) dst[k] = x[k];
   }
   __threadfence_system();
@@ -102,6 +102,7 @@ __global__ void __launch_bounds__(1024) tp_bcast_kernel(const float* x, int h, c
 
 struct RecvArgs {
   const float* recv;
+  long long half;
   const int* flags;
   int* epoch;
   int n_ranks, h, mode, n_parts, wait_polls;
@@ -134,7 +135,7 @@ __global__ void __launch_bounds__(1024) tp_recv_kernel(const RecvArgs A) {
   }
   __syncthreads();
   if (!s_ok) return;  // nothing is changed: the host sees the error word and resets the group
-  const float* P = A.recv + (size_t)parity * R * A.h;
+  const float* P = A.recv + (size_t)parity * A.half;
   float ss = 0.f;
   for (int k = threadIdx.x; k < A.h; k += blockDim.x) {
     float s = __ldcg(P + k);  // the master's own partial (rank 0) ...
@@ -154,6 +155,62 @@ __global__ void __launch_bounds__(1024) tp_recv_kernel(const RecvArgs A) {
     *A.epoch = c + 1;
     if (A.pos_advance) *A.pos_advance += 1;
   }
+}
+
+
+// Prompt pass: a block of n floats (T x h) goes to every rank's slot of this source.  Many CTAs copy, the last to
+// finish publishes the flags.
+__global__ void __launch_bounds__(256) tp_push_rows_kernel(const float* src, size_t n, const int* epoch, unsigned* ticket,
+                                                           const TpPeers P, int src_rank, int drop) {
+  __shared__ bool s_last;
+  pdl_wait();
+  pdl_launch_dependents();
+  const int c = __ldcg(epoch), parity = c & 1, R = P.n_ranks;
+  if (!drop) {
+    const size_t n4 = n >> 2;
+    for (int j = 0; j < R; ++j) {
+      float4* dst = reinterpret_cast<float4*>(P.recv[j] + (size_t)parity * P.half + (size_t)src_rank * n);
+      const float4* s4 = reinterpret_cast<const float4*>(src);
+      for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) dst[i] = s4[i];
+    }
+  }
+  __threadfence_system();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned t = atomicAdd(ticket, 1u);
+    s_last = (t == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (s_last && threadIdx.x == 0) {
+    __threadfence_system();
+    if (!drop)
+      for (int j = 0; j < R; ++j) st_release_sys(P.flags[j] + parity * R + src_rank, c + 1);
+    *ticket = 0u;
+  }
+}
+
+// The consumer's wait alone: one thread per source, bounded; then the counter moves on.
+__global__ void tp_wait_kernel(const int* flags, int* epoch, int n_ranks, int n_src, int* err, int wait_polls) {
+  __shared__ int s_ok;
+  pdl_wait();
+  pdl_launch_dependents();
+  const int c = __ldcg(epoch), parity = c & 1;
+  if (threadIdx.x == 0) s_ok = 1;
+  __syncthreads();
+  if ((int)threadIdx.x < n_src) {
+    const int* f = flags + parity * n_ranks + threadIdx.x;
+    bool got = false;
+    for (int i = 0; i < wait_polls; ++i) {
+      if (ld_acquire_sys(f) == c + 1) { got = true; break; }
+      if (i > 64) __nanosleep(100);
+    }
+    if (!got) {
+      atomicCAS(err, DEVERR_NONE, DEVERR_WAIT_TIMEOUT);
+      s_ok = 0;
+    }
+  }
+  __syncthreads();
+  if (s_ok && threadIdx.x == 0) *epoch = c + 1;
 }
 
 }  // namespace
@@ -184,15 +241,30 @@ cudaError_t launch_tp_rowpush(const LaunchCtx& c, int dt, const void* W, const f
   return dt == DT_BF16 ? go(__nv_bfloat16{}) : go(float{});
 }
 
+cudaError_t launch_tp_push_rows(const LaunchCtx& c, const float* src, size_t n, const int* epoch, unsigned* ticket,
+                                const TpPeers& peers, int as_rank0, int drop) {
+  if (n < 4 || n % 4 || (long long)(n * peers.n_ranks) > peers.half) return cudaErrorInvalidValue;
+  size_t blocks = (n / 4 + 255) / 256;
+  const size_t cap = (size_t)sm_count_tp() * 4;
+  if (blocks > cap) blocks = cap;
+  return launch_kernel(c, tp_push_rows_kernel, dim3((unsigned)blocks), dim3(256), 0, src, n, epoch, ticket, peers,
+                       as_rank0 ? 0 : peers.rank, drop);
+}
+
+cudaError_t launch_tp_wait(const LaunchCtx& c, const int* flags, int* epoch, int n_ranks, int n_src, int* err, int wait_polls) {
+  if (n_ranks < 1 || n_ranks > TP_MAX_RANKS || n_src < 1 || n_src > n_ranks || wait_polls < 1 || !err) return cudaErrorInvalidValue;
+  return launch_kernel(c, tp_wait_kernel, dim3(1), dim3(32), 0, flags, epoch, n_ranks, n_src, err, wait_polls);
+}
+
 cudaError_t launch_tp_bcast(const LaunchCtx& c, const float* x, int h, const int* epoch, const TpPeers& peers, int drop) {
   return launch_kernel(c, tp_bcast_kernel, dim3(1), dim3(1024), 0, x, h, epoch, peers, drop);
 }
 
-cudaError_t launch_tp_recv(const LaunchCtx& c, const float* recv, const int* flags, int* epoch, int n_ranks, int h, int mode,
-                           float eps, float* x, float* xhat, float* tap, float* ss_part, int n_parts, int* pos_advance,
+cudaError_t launch_tp_recv(const LaunchCtx& c, const float* recv, long long half, const int* flags, int* epoch, int n_ranks, int h,
+                           int mode, float eps, float* x, float* xhat, float* tap, float* ss_part, int n_parts, int* pos_advance,
                            int* err, int wait_polls) {
-  if (n_ranks < 1 || n_ranks > TP_MAX_RANKS || wait_polls < 1 || !err) return cudaErrorInvalidValue;
-  RecvArgs A{recv, flags, epoch, n_ranks, h, mode, n_parts, wait_polls, eps, x, xhat, tap, ss_part, pos_advance, err};
+  if (n_ranks < 1 || n_ranks > TP_MAX_RANKS || wait_polls < 1 || !err || half < (long long)n_ranks * h) return cudaErrorInvalidValue;
+  RecvArgs A{recv, half, flags, epoch, n_ranks, h, mode, n_parts, wait_polls, eps, x, xhat, tap, ss_part, pos_advance, err};
   return launch_kernel(c, tp_recv_kernel, dim3(1), dim3(1024), 0, A);
 }
 

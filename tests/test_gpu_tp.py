@@ -11,9 +11,9 @@ from tests.helpers import check_logits, close_elementwise, gpu_session, make_ora
 pytestmark = pytest.mark.gpu
 
 
-def _group(shape, R, max_seq, window=0):
+def _group(shape, R, max_seq, window=0, max_prefill=None):
     import paper_2410_00531_b200.tp as TP
-    return TP.Group(tpi_config(shape, max_seq, 1), S.synth_fill(shape), R, window)
+    return TP.Group(tpi_config(shape, max_seq, max_prefill or max_seq), S.synth_fill(shape), R, window)
 
 
 CASES = {
@@ -21,6 +21,8 @@ CASES = {
     "c1_r4": (S.CONFIGS["C1"], 4, 12, 5),
     "bf16_gqa_r2": (S.CONFIGS["C1"].with_(dtype="bf16", n_heads=8, n_kv_heads=2, head_dim=32, seed=77, rope_base=500000.0), 2, 10, 4),
     "c3_widths_r8": (S.CONFIGS["C3"].with_(n_layers=2, vocab=32000), 8, 20, 3),
+    "c3_widths_r8_long": (S.CONFIGS["C3"].with_(n_layers=2, vocab=32000), 8, 300, 2),
+    "c5_widths_r2": (S.CONFIGS["C5"].with_(n_layers=1, vocab=32000), 2, 140, 2),
     "c2_widths_r4": (S.CONFIGS["C2"].with_(n_layers=2), 4, 12, 3),
     "f32_gqa_r1": (S.CONFIGS["C1"].with_(n_heads=8, n_kv_heads=4, head_dim=32), 1, 8, 3),
 }
@@ -28,8 +30,8 @@ CASES = {
 
 @pytest.mark.parametrize("case", sorted(CASES))
 def test_ranks_match_the_oracle_s_per_device_form(case):
-    """Prompt (one position at a time) + teacher-forced decode against `forward(n_shards=R)`: logits and token rule on the
-    master, H_attn / H_ffn of every layer on EVERY rank (all ranks must hold the same bits after an allreduce), cache
+    """Prompt pass (all positions per pass, every rank on its slices; 300 positions take the CTA-pair GEMMs and the
+    tcgen05 attention) + teacher-forced decode against `forward(n_shards=R)`: logits and token rule on the master, H_attn / H_ffn of every layer on EVERY rank (all ranks must hold the same bits after an allreduce), cache
     rows of every kv head on the rank that owns it."""
     shape, R, T, n_dec = CASES[case]
     tol = tol_for(shape)
@@ -71,9 +73,11 @@ def test_ranks_give_the_emulated_shard_model_s_bits(case):
     the two-kernel form (partial sums through memory, then the rank-ordered sum) and is fed the prompt one position at a
     time through the same decode kernels.  Contexts stay within one attention split (256 positions)."""
     import paper_2410_00531_b200 as P
+    import paper_2410_00531_b200.tp as TP
     shape, R, T, n_dec = CASES[case]
     toks = S.prompt_tokens(shape, T)
     with _group(shape, R, T + n_dec + 2) as g:
+        g.set_option(TP.OPT_BATCHED_PROMPT, 0)                   # the prompt through the decode kernels, like the model below
         t_tp, lg_tp = g.prefill(toks, shape.vocab)
         seq_tp = g.decode_run(t_tp, n_dec)
         h_tp = [g.get_hidden(R - 1, l, w) for l in range(shape.n_layers) for w in (0, 1)]
@@ -89,13 +93,37 @@ def test_ranks_give_the_emulated_shard_model_s_bits(case):
         assert np.array_equal(a, b)
 
 
+@pytest.mark.parametrize("case,chunk", [("c1_r2", None), ("c1_r4", 5), ("bf16_gqa_r2", None), ("c3_widths_r8", None),
+                                        ("c3_widths_r8_long", None), ("c3_widths_r8_long", 128)])
+def test_prompt_pass_of_the_ranks_gives_the_emulated_model_s_prompt_pass_bits(case, chunk):
+    """The batched prompt pass on R ranks against the emulated model's (N = R): the same GEMM, attention and row kernels
+    run on slices instead of on the whole, every output element is accumulated in the same order, and the partial
+    sums are added in rank order on both sides, so first token, logits and the last position's hidden states agree
+    bit for bit; chunked prompts (a last chunk shorter than the others) included."""
+    import paper_2410_00531_b200 as P
+    shape, R, T, _ = CASES[case]
+    toks = S.prompt_tokens(shape, T)
+    with _group(shape, R, T + 4, max_prefill=chunk) as g:
+        t_tp, lg_tp = g.prefill(toks, shape.vocab)
+        h_tp = [g.get_hidden(0, l, w) for l in range(shape.n_layers) for w in (0, 1)]
+        kv_tp = g.get_kv(shape.n_layers - 1, shape.n_kv_heads - 1, 0, T)
+    with gpu_session(shape, T + 4, chunk or T, R) as ses:
+        t_em, lg_em = P.prefill(ses.h, toks, shape.vocab)
+        h_em = [P.get_hidden(ses.h, l, w, shape.hidden) for l in range(shape.n_layers) for w in (0, 1)]
+        kv_em = P.get_kv(ses.h, shape.n_layers - 1, shape.n_kv_heads - 1, 0, T, shape.head_dim)
+    assert t_tp == t_em and np.array_equal(lg_tp, lg_em)
+    for a, b in zip(h_tp, h_em):
+        assert np.array_equal(a, b)
+    assert np.array_equal(kv_tp[0], kv_em[0]) and np.array_equal(kv_tp[1], kv_em[1])
+
+
 def test_streamed_ranks_give_the_resident_ranks_bits():
     """Every rank streams its own blocks through its own window (Sec. 3.3 runs on every device)."""
     shape = S.CONFIGS["C1"].with_(n_layers=4)
     toks = S.prompt_tokens(shape, 9)
     res = {}
     for w in (0, 2, 3):
-        with _group(shape, 2, 32, w) as g:
+        with _group(shape, 2, 32, w, max_prefill=4) as g:        # 9 prompt positions in chunks of 4 + 4 + 1
             t0, lg = g.prefill(toks, shape.vocab)
             res[w] = (t0, lg, g.decode_run(t0, 5))
     for w in (2, 3):
@@ -126,6 +154,12 @@ def test_a_rank_that_never_publishes_ends_in_a_timeout_status_and_reset_recovers
             with pytest.raises(P.TpiError) as e:
                 g.decode_step(int(seq0[-1]), 0)                  # refused until the group is reset
             assert e.value.code == -9
+            g.reset()
+            # the same failure inside a prompt pass
+            g.set_option(TP.OPT_DROP_PUSH, victim + 1)
+            with pytest.raises(P.TpiError) as e:
+                g.prefill(toks, 0)
+            assert e.value.code == -7
             g.reset()
             g.set_option(TP.OPT_WAIT_POLLS, 1 << 21)
             t1, lg1 = g.prefill(toks, shape.vocab)
