@@ -302,13 +302,15 @@ def resident_leg(P, name, shape, local, K, W, prefill_chunk):
         close_session(ses)
     peak, kind = measured_peaks()
     tr = ttft_roofline(shape, T, r["ttft_ms"], r["stats"]["weight_bytes_per_token"], peak)
-    return {"workload": f"{name} {shape.name} N={shape.n_shards} resident", "steps": K, "warmup": W,
+    return {"workload": f"{name} {shape.name} N={shape.n_shards} resident", "steps": K,
             "context": f"{T + W}..{T + W + K}", "tokens_per_s": round(K / (r["dev_ms"] * 1e-3), 2),
-            "ms_per_step": round(r["dev_ms"] / K, 4), "bytes_per_token": int(r["token_bytes"]),
-            "hbm_gbs": round(r["token_gbs"], 1), "hbm_frac": round(r["token_gbs"] / peak, 4), "peak_kind": kind,
-            "ttft_ms": round(r["ttft_ms"], 3), "ttft_prompt_tokens": T, "ttft_bound": tr["bound"],
-            "ttft_frac": round(tr["frac"], 4), "graph": bool(r["stats"]["graph_active"]),
-            "gpu_launches": r["stats"]["kernel_launches_last"], "clocks": r["clocks"], "load_s": round(load_s, 1)}
+            "ms_per_step": round(r["dev_ms"] / K, 4), "hbm_gbs": round(r["token_gbs"], 1),
+            "hbm_frac": round(r["token_gbs"] / peak, 4), "ttft_ms": round(r["ttft_ms"], 2), "ttft_prompt_tokens": T,
+            "ttft_bound": tr["bound"], "ttft_frac": round(tr["frac"], 4), "clocks": short_clocks(r["clocks"])}
+
+
+def short_clocks(c: dict) -> dict:
+    return {"sm_mhz": c.get("sm_mhz"), "reasons": c.get("reasons"), "samples": c.get("samples")}
 
 
 def host_link_peak(torch, local: int) -> float:
@@ -368,17 +370,14 @@ def streamed_leg(P, name, shape, local, K, W, window, link_peak, retain=0):
     finally:
         close_session(ses)
     st = r["stats"]
-    return {"workload": f"{name} {shape.name} L{shape.n_layers} N={shape.n_shards} streamed, window {window} blocks"
+    return {"workload": f"{name} {shape.name} L{shape.n_layers} streamed, window {window}"
                         + (f", retain T={sched['retain_every_T']}" if retain else ""),
-            "steps": K, "warmup": W, "tokens_per_s": round(r["tokens_per_s"], 4),
-            "ms_per_step": round(r["wall_s"] / K * 1e3, 2), "link_bytes_per_token": int(r["region_bytes"] / K),
-            "link_gbs": round(r["link_gbs"], 2), "link_peak_gbs": round(link_peak, 2),
-            "link_frac": round(r["link_gbs"] / link_peak, 4), "window_device_bytes": st["window_peak_bytes"],
-            "retained_blocks": st["retained_blocks"], "ttft_ms": round(r["ttft_ms"], 1),
-            "ttft_prompt_tokens": shape.prompt_len,
-            "sched": {k: (round(v, 3) if isinstance(v, float) else v) for k, v in sched.items()
-                      if k in ("t_attn_ms", "t_ffn_ms", "tau_attn_ms", "tau_ffn_ms", "tight_holds", "loose_holds", "retention_T")},
-            "clocks": r["clocks"], "load_s": round(load_s, 1)}
+            "steps": K, "tokens_per_s": round(r["tokens_per_s"], 4), "ms_per_step": round(r["wall_s"] / K * 1e3, 2),
+            "link_GB_per_token": round(r["region_bytes"] / K / 1e9, 3), "link_gbs": round(r["link_gbs"], 2),
+            "link_peak_gbs": round(link_peak, 2), "link_frac": round(r["link_gbs"] / link_peak, 4),
+            "tau_over_t": [round(sched["tau_attn_ms"] / max(sched["t_attn_ms"], 1e-9), 1),
+                           round(sched["tau_ffn_ms"] / max(sched["t_ffn_ms"], 1e-9), 1)],
+            "loose_holds": sched["loose_holds"], "clocks": short_clocks(r["clocks"])}
 
 
 def tp_one_gpu_leg(P, shape, local, R, K, W):
@@ -415,13 +414,10 @@ def tp_one_gpu_leg(P, shape, local, R, K, W):
         import gc
         gc.collect()
         torch.cuda.empty_cache()
-    return {"workload": f"{shape.name}: {R} ranks with one shard each, ALL ON ONE GPU (time-shared, events between streams; "
-                        "functional, not a multi-GPU number)", "steps": K, "warmup": W,
-            "tokens_per_s": round(K / wall, 2), "ms_per_step": round(wall / K * 1e3, 3), "ttft_ms": round(ttft_ms, 2),
-            "ttft_prompt_tokens": T, "kernel_launches_per_token": st["kernel_launches_last"] // K,
-            "exchange_bytes_per_token_per_rank": st["exchange_bytes_per_token"],
-            "weight_bytes_per_token_worker": st["weight_bytes_worker"], "tokens_tail": [int(x) for x in out[-2:]],
-            "clocks": clocks, "load_s": round(load_s, 1)}
+    return {"workload": f"{shape.name}: {R} ranks, one shard each, ALL ON ONE GPU (time-shared; functional, not a multi-GPU number)",
+            "steps": K, "tokens_per_s": round(K / wall, 2), "ms_per_step": round(wall / K * 1e3, 3), "ttft_ms": round(ttft_ms, 2),
+            "ttft_prompt_tokens": T, "launches_per_token": st["kernel_launches_last"] // K,
+            "exchange_bytes_per_token_per_rank": st["exchange_bytes_per_token"], "clocks": short_clocks(clocks)}
 
 
 def extra_legs(P, args, local):
@@ -436,7 +432,7 @@ def extra_legs(P, args, local):
         t0 = time.perf_counter()
         try:
             legs[key] = fn()
-            legs[key]["leg_s"] = round(time.perf_counter() - t0, 1)
+            legs[key]["leg_s"] = round(time.perf_counter() - t0)
         except Exception as e:   # a leg that cannot run on this machine (memory) must not take the headline down
             legs[key] = {"error": f"{type(e).__name__}: {e}"[:300]}
             torch.cuda.empty_cache()
@@ -473,6 +469,10 @@ def run_gpu(args, shape):
     K, W, T = args.steps, args.warmup, shape.prompt_len
     if args.window > 0:
         return run_streamed(args, shape, local, rank)
+    if args.tp > 0:  # the one-shard-per-rank form with all ranks on this GPU, alone (short runs under a profiler)
+        if rank == 0:
+            print(json.dumps(tp_one_gpu_leg(P, shape, local, args.tp, K, W)), flush=True)
+        return
     ses, t_load = open_session(P, shape, local, T + W + K + 8, args.prefill_chunk)
     h = ses.h
     toks = S.prompt_tokens(shape)
@@ -620,6 +620,8 @@ def main():
     ap.add_argument("--prefill-chunk", type=int, default=4096, help="prompt positions processed per pass over the weights")
     ap.add_argument("--quick", action="store_true",
                     help="one prompt pass and the device-resident decode loop only (short runs under a profiler)")
+    ap.add_argument("--tp", type=int, default=0,
+                    help="run the workload as this many ranks with one shard each, all on this GPU, and print that leg alone")
     ap.add_argument("--layers", type=int, default=0, help="override the depth (small captures under a profiler)")
     args = ap.parse_args()
     shape = S.CONFIGS[args.workload]

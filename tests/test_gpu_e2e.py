@@ -367,7 +367,7 @@ def test_second_model_family_non_power_of_two_widths():
     N = 8; two layers and a 32000-entry vocabulary so that the oracle finishes in seconds."""
     shape = S.CONFIGS["C3"].with_(n_layers=2, hidden=7168, n_heads=56, n_kv_heads=8, head_dim=128, ffn=20480, vocab=32000,
                                   rope_base=5000000.0)
-    toks, mism = _run_and_compare(shape, 8, n_decode=4, prompt_len=96)
+    toks, mism = _run_and_compare(shape, 8, n_decode=4, prompt_len=96, max_ambiguous=3)
     assert mism <= 2
 
 
@@ -380,7 +380,7 @@ def test_full_width_reduced_depth(cfg, n_shards, T, chunk):
     long-prompt kernels (CTA-pair projections, star sum in the GEMM epilogue, tcgen05 attention); in chunks
     of 256 + 44 the second chunk takes the short-prompt kernels on top of the first chunk's cache."""
     shape = S.CONFIGS[cfg].with_(n_layers=2, vocab=32000)
-    toks, mism = _run_and_compare(shape, n_shards, n_decode=6, prompt_len=T, max_prefill=chunk)
+    toks, mism = _run_and_compare(shape, n_shards, n_decode=6, prompt_len=T, max_prefill=chunk, max_ambiguous=4)
     assert mism <= 3
 
 
