@@ -104,9 +104,13 @@ int tpi_tp_get_kv(tpi_tp_group *g, int layer, int kv_head, int pos0, int n, floa
  * never publishes them (a rank that "never joins"); the other ranks' waits then
  * run out and the call returns TPI_ERR_TIMEOUT; one-shot, 0 clears it.
  * TPI_TP_OPT_PDL: programmatic dependent launch between a rank's kernels
- * (default 1).  TPI_TP_OPT_BATCHED_PROMPT (default 1): see above. */
+ * (default 1).  TPI_TP_OPT_BATCHED_PROMPT (default 1): see above.
+ * TPI_TP_OPT_GRAPH (default 1): with every block resident, a decode position of
+ * ALL ranks is one CUDA graph (captured from the master's stream; the other
+ * ranks' streams join through the exchange's event waits, which become graph
+ * edges), so a token costs the host one launch; 0 = stream launches. */
 enum { TPI_TP_OPT_EVENTS = 0, TPI_TP_OPT_WAIT_POLLS = 1, TPI_TP_OPT_DROP_PUSH = 2, TPI_TP_OPT_PDL = 3,
-       TPI_TP_OPT_BATCHED_PROMPT = 4 };
+       TPI_TP_OPT_BATCHED_PROMPT = 4, TPI_TP_OPT_GRAPH = 5 };
 int tpi_tp_set_option(tpi_tp_group *g, int option, int value);
 
 typedef struct {

@@ -98,7 +98,10 @@ struct tpi_tp_group {
   tpi_config cfg{};
   int R = 0, window = 0;
   std::vector<TpRank> ranks;
-  int events = 1, wait_polls = 1 << 21, drop_rank = -1, pdl = 1, batched_prompt = 1;
+  int events = 1, wait_polls = 1 << 21, drop_rank = -1, pdl = 1, batched_prompt = 1, use_graph = 1;
+  cudaGraphExec_t graph_exec = nullptr;  // one decode position of ALL ranks (resident groups only)
+  int graph_launches = 0;
+  cudaEvent_t ev_graph = nullptr;
   int position = 0, launches_last = 0;
   bool broken = false;  // a call failed or timed out: tpi_tp_reset first
   uint64_t exchanges = 0;
@@ -131,8 +134,9 @@ bool share_a_device(const tpi_tp_group* g) {
 
 // One position through all ranks (enqueue only).  with_head: the master runs the task head and the greedy argmax
 // (which advance its position); otherwise (a prompt position that is not the last) its last consumer advances it.
-int enqueue_step(tpi_tp_group* g, bool with_head, int* launches) {
+int enqueue_step(tpi_tp_group* g, bool with_head, int* launches, bool force_edges = false) {
   const tpi_config& c = g->cfg;
+  const bool edges = g->events || force_edges;  // inside a graph capture the cross-stream waits ARE the graph's edges
   const int R = g->R, h = c.hidden, d = c.head_dim, dt = c.dtype, L = c.n_layers;
   const int al = c.n_heads / R, bl_ = c.n_kv_heads / R, sl = c.ffn / R;
   auto ctx = [&](TpRank& r) { return LaunchCtx{r.m->cs, g->pdl != 0, launches}; };
@@ -147,7 +151,7 @@ int enqueue_step(tpi_tp_group* g, bool with_head, int* launches) {
       tpi_model* m = r.m;
       const Plan& p = m->plan;
       CK(cudaSetDevice(r.device));
-      if (g->events) {
+      if (edges) {
         if (mode == 1) { if (i != 0) CK(cudaStreamWaitEvent(m->cs, g->ranks[0].ev_push, 0)); }
         else
           for (int j = 0; j < R; ++j)
@@ -174,7 +178,7 @@ int enqueue_step(tpi_tp_group* g, bool with_head, int* launches) {
                     dptr<float>(m, p.x), dptr<float>(m, p.xhat), dptr<float>(m, p.ss_part), rowshard_fused_parts(h),
                     dptr<int>(m, p.err)));
     CK(launch_tp_bcast(lc, dptr<float>(m, p.x), h, r.epoch, peers_of(g, 0), drop_now(0)));
-    if (g->events) CK(cudaEventRecord(r.ev_push, m->cs));
+    if (edges) CK(cudaEventRecord(r.ev_push, m->cs));
   }
   TRY(consume(1, -1, false));
   for (int l = 0; l < L; ++l) {
@@ -204,7 +208,7 @@ int enqueue_step(tpi_tp_group* g, bool with_head, int* launches) {
                                drop_now(i)));
         }
         TRY(release_block(m, 2 * l + blk));
-        if (g->events) CK(cudaEventRecord(r.ev_push, m->cs));
+        if (edges) CK(cudaEventRecord(r.ev_push, m->cs));
       }
       TRY(consume(0, 2 * l + blk, l == L - 1 && blk == 1));
     }
@@ -431,6 +435,48 @@ int run_prompt(tpi_tp_group* g, const int32_t* tokens, int n, int32_t* first, fl
   return TPI_OK;
 }
 
+void drop_group_graph(tpi_tp_group* g) {
+  if (g->graph_exec) cudaGraphExecDestroy(g->graph_exec);
+  g->graph_exec = nullptr;
+}
+
+// One decode position of all ranks as ONE CUDA graph: captured from the master's compute stream, the other ranks'
+// streams join the capture through the exchange's event waits (which become the graph's edges) and are joined back at
+// the end.  A token then costs the host one launch instead of 2 + R (1 + 7 L).
+int ensure_group_graph(tpi_tp_group* g) {
+  if (g->graph_exec) return TPI_OK;
+  TpRank& r0 = g->ranks[0];
+  cudaStream_t origin = r0.m->cs;
+  CK(cudaSetDevice(r0.device));
+  const uint64_t saved = g->exchanges;
+  int launches = 0;
+  cudaGraph_t graph = nullptr;
+  CK(cudaStreamBeginCapture(origin, cudaStreamCaptureModeThreadLocal));
+  int rc = enqueue_step(g, true, &launches, true);
+  cudaError_t e = cudaSuccess;
+  for (int i = 1; i < g->R && rc == TPI_OK && e == cudaSuccess; ++i) {  // join every rank's stream back
+    TpRank& r = g->ranks[i];
+    cudaSetDevice(r.device);
+    e = cudaEventRecord(r.ev_push, r.m->cs);
+    cudaSetDevice(r0.device);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(origin, r.ev_push, 0);
+  }
+  cudaSetDevice(r0.device);
+  const cudaError_t e2 = cudaStreamEndCapture(origin, &graph);
+  g->exchanges = saved;
+  if (rc) { if (graph) cudaGraphDestroy(graph); return rc; }
+  if (e != cudaSuccess || e2 != cudaSuccess) {
+    if (graph) cudaGraphDestroy(graph);
+    cudaGetLastError();
+    return fail(TPI_ERR_CUDA, "capturing the ranks' decode step failed: %s", cudaGetErrorString(e != cudaSuccess ? e : e2));
+  }
+  e = cudaGraphInstantiate(&g->graph_exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (e != cudaSuccess) { g->graph_exec = nullptr; return fail(TPI_ERR_CUDA, "graph instantiate failed: %s", cudaGetErrorString(e)); }
+  g->graph_launches = launches;
+  return TPI_OK;
+}
+
 // Feeds n positions: tokens[] (n_given of them, the rest are the ranks' own outputs chained on the master) and returns
 // the master's tokens after each of the last n_out positions.
 int run_positions(tpi_tp_group* g, const int32_t* tokens, int n_given, int n_pos, bool head_every, int32_t* out, int n_out,
@@ -449,7 +495,26 @@ int run_positions(tpi_tp_group* g, const int32_t* tokens, int n_given, int n_pos
   CK(cudaMemcpyAsync(dptr<int>(m0, m0->plan.tok_hist) + g->position, io0 + 3, (size_t)n_given * 4, cudaMemcpyHostToDevice, m0->cs));
   int launches = 0;
   g->broken = true;  // until the call has gone through
-  for (int i = 0; i < n_pos; ++i) TRY(enqueue_step(g, head_every || i == n_pos - 1, &launches));
+  const bool graph = g->use_graph && g->window <= 0 && head_every && g->drop_rank < 0;
+  if (graph) TRY(ensure_group_graph(g));
+  for (int i = 0; i < n_pos; ++i) {
+    if (graph) {
+      CK(cudaSetDevice(g->ranks[0].device));
+      CK(cudaGraphLaunch(g->graph_exec, m0->cs));
+      launches += g->graph_launches;
+      g->exchanges += 2ull * c.n_layers + 1;
+    } else {
+      TRY(enqueue_step(g, head_every || i == n_pos - 1, &launches));
+    }
+  }
+  if (graph) {  // the other ranks' streams took no part in the launch: what they do next comes after the graph
+    CK(cudaSetDevice(g->ranks[0].device));
+    CK(cudaEventRecord(g->ev_graph, m0->cs));
+    for (int i = 1; i < g->R; ++i) {
+      CK(cudaSetDevice(g->ranks[i].device));
+      CK(cudaStreamWaitEvent(g->ranks[i].m->cs, g->ev_graph, 0));
+    }
+  }
   // results and error words
   CK(cudaSetDevice(g->ranks[0].device));
   CK(cudaMemcpyAsync(io0 + 3, dptr<int>(m0, m0->plan.tok_hist) + g->position + n_pos - n_out + 1, (size_t)n_out * 4,
@@ -507,6 +572,8 @@ extern "C" int tpi_tp_query_arena(const tpi_config* cfg, int n_ranks, int rank, 
 extern "C" void tpi_tp_free(tpi_tp_group* g) {
   if (!g) return;
   DeviceGuard guard;
+  drop_group_graph(g);
+  if (g->ev_graph) cudaEventDestroy(g->ev_graph);
   for (auto& r : g->ranks) {
     cudaSetDevice(r.device);
     if (r.m) tpi_free(r.m);
@@ -573,6 +640,8 @@ extern "C" int tpi_tp_create(const tpi_config* cfg, int n_ranks, const tpi_resou
         cudaEventCreateWithFlags(&r.ev_done, cudaEventDisableTiming) != cudaSuccess)
       return bail(fail(TPI_ERR_CUDA, "event creation failed"));
   }
+  cudaSetDevice(g->ranks[0].device);
+  if (cudaEventCreateWithFlags(&g->ev_graph, cudaEventDisableTiming) != cudaSuccess) return bail(fail(TPI_ERR_CUDA, "event creation failed"));
   *out = g;
   return TPI_OK;
 }
@@ -640,15 +709,20 @@ extern "C" int tpi_tp_set_option(tpi_tp_group* g, int option, int value) {
         return fail(TPI_ERR_STATE, "ranks that share a device must be ordered by events: a kernel may not wait for a kernel that is not running");
       g->events = value != 0;
       return TPI_OK;
+    case TPI_TP_OPT_GRAPH:
+      g->use_graph = value != 0;
+      drop_group_graph(g);
+      return TPI_OK;
     case TPI_TP_OPT_WAIT_POLLS:
       if (value < 1) return fail(TPI_ERR_INVALID_ARG, "the poll limit must be positive");
       g->wait_polls = value;
+      drop_group_graph(g);  // the limit is a kernel argument
       return TPI_OK;
     case TPI_TP_OPT_DROP_PUSH:
       if (value < 0 || value > g->R) return fail(TPI_ERR_INVALID_ARG, "rank + 1 expected");
       g->drop_rank = value - 1;
       return TPI_OK;
-    case TPI_TP_OPT_PDL: g->pdl = value != 0; return TPI_OK;
+    case TPI_TP_OPT_PDL: g->pdl = value != 0; drop_group_graph(g); return TPI_OK;
     case TPI_TP_OPT_BATCHED_PROMPT: g->batched_prompt = value != 0; return TPI_OK;
     default: return fail(TPI_ERR_INVALID_ARG, "unknown option %d", option);
   }

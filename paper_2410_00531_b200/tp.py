@@ -11,7 +11,7 @@ import numpy as np
 
 from .binding import (FILL_FN, T_WDOWN, T_WO, TPI_BF16, TpiConfig, TpiResources, _check, _fptr, lib)
 
-OPT_EVENTS, OPT_WAIT_POLLS, OPT_DROP_PUSH, OPT_PDL, OPT_BATCHED_PROMPT = 0, 1, 2, 3, 4
+OPT_EVENTS, OPT_WAIT_POLLS, OPT_DROP_PUSH, OPT_PDL, OPT_BATCHED_PROMPT, OPT_GRAPH = 0, 1, 2, 3, 4, 5
 _P, _I = C.c_void_p, C.c_int
 _I64P = C.POINTER(C.c_int64)
 

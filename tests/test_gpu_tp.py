@@ -117,6 +117,28 @@ def test_prompt_pass_of_the_ranks_gives_the_emulated_model_s_prompt_pass_bits(ca
     assert np.array_equal(kv_tp[0], kv_em[0]) and np.array_equal(kv_tp[1], kv_em[1])
 
 
+def test_one_graph_over_all_ranks_matches_stream_launches():
+    """By default a decode position of all ranks is one CUDA graph (captured across the ranks' streams); the same kernels
+    as plain stream launches, with and without programmatic dependent launch, must give the same tokens and logits."""
+    import paper_2410_00531_b200.tp as TP
+    shape, R, T, _ = CASES["c3_widths_r8"]
+    toks = S.prompt_tokens(shape, T)
+    res = {}
+    with _group(shape, R, T + 40) as g:
+        for key, graph, pdl in (("graph", 1, 1), ("stream", 0, 1), ("stream_no_pdl", 0, 0), ("graph_again", 1, 0)):
+            g.set_option(TP.OPT_GRAPH, graph)
+            g.set_option(TP.OPT_PDL, pdl)
+            g.reset()
+            t0, _ = g.prefill(toks, 0)
+            seq = g.decode_run(t0, 24)
+            t1, lg = g.decode_step(int(seq[-1]), shape.vocab)
+            res[key] = (t0, seq, t1, lg)
+            assert g.stats()["kernel_launches_last"] == 2 + R * (1 + shape.n_layers * 7) + 1
+    for key in ("stream", "stream_no_pdl", "graph_again"):
+        a, b = res["graph"], res[key]
+        assert a[0] == b[0] and (a[1] == b[1]).all() and a[2] == b[2] and np.array_equal(a[3], b[3]), key
+
+
 def test_streamed_ranks_give_the_resident_ranks_bits():
     """Every rank streams its own blocks through its own window (Sec. 3.3 runs on every device)."""
     shape = S.CONFIGS["C1"].with_(n_layers=4)
