@@ -75,6 +75,24 @@ def test_prop5_worker_peak_counts_blocks():
     assert W.block_params("attn", h, v, a, b, s, p) == attn
 
 
+def test_prop5_peaks_add_up_table5_s_printed_block_sizes():
+    """Prop. 5 against numbers the paper prints, not against the formula typed again: Table 5 gives the blocks of
+    Llama 2-7B with n = 4, p = 0.25 in FP32 as 500 / 64 / 129 / 500 MB, and Prop. 5 says which of them a window of w
+    blocks holds: a worker floor(w/2) attention + ceil(w/2) FFN blocks (w = 1: the larger, FFN); the master its
+    pre/postprocess blocks first (w = 1: the postprocess block, w = 2: both) and the layer blocks in what is left."""
+    import os
+    rows = [ln.split() for ln in open(os.path.join(os.path.dirname(__file__), "golden", "table5_block_sizes.txt")) if ln[0] != "#"]
+    mb = {k: float(v) for k, v in rows}
+    h, v, a, b, s, p = 4096, 32000, 32, 32, 11008, 0.25
+    MiB = 2.0 ** 20 / 4          # parameters per printed MB (FP32)
+    for w, want in ((1, mb["ffn"]), (2, mb["attn"] + mb["ffn"]), (3, mb["attn"] + 2 * mb["ffn"]),
+                    (4, 2 * mb["attn"] + 2 * mb["ffn"]), (8, 4 * (mb["attn"] + mb["ffn"]))):
+        assert abs(W.worker_peak(w, h, a, b, s, p) / MiB - want) < 0.5 * w, w        # the printed sizes are rounded to 1 MB
+    for w, want in ((1, mb["post"]), (2, mb["pre"] + mb["post"]), (3, mb["pre"] + mb["post"] + mb["ffn"]),
+                    (4, mb["pre"] + mb["post"] + mb["attn"] + mb["ffn"]), (6, mb["pre"] + mb["post"] + 2 * (mb["attn"] + mb["ffn"]))):
+        assert abs(W.master_peak(w, h, v, a, b, s, p) / MiB - want) < 0.5 * w, w
+
+
 def test_retention_slot_expressions_and_prop6():
     """Appendix A.6's time-slot expressions evaluated by hand on the paper's measured latencies
     (t_attn 11, t_ffn 17, tau_attn 18, tau_ffn 30; allreduce 14 as in the worked example) with T = 2."""
