@@ -224,6 +224,13 @@ int enqueue_step(tpi_tp_group* g, bool with_head, int* launches, bool force_edge
                           h, c.vocab, dptr<float>(m, p.logits), dptr<float>(m, p.amax_val), dptr<int>(m, p.amax_idx),
                           dptr<unsigned>(m, p.tickets) + bl_, dptr<int>(m, p.tok_hist), dptr<int>(m, p.pos), 1));
   }
+  for (int i = 0; i < R; ++i) {  // debug arenas (TPI_DEBUG=1): every rank's guard zones are compared after the step
+    TpRank& r = g->ranks[i];
+    if (r.m->plan.n_canaries < 1) break;
+    CK(cudaSetDevice(r.device));
+    LaunchCtx lc = ctx(r);
+    TRY(enqueue_canary_check(r.m, lc));
+  }
   return TPI_OK;
 }
 
@@ -369,6 +376,13 @@ int enqueue_prompt_chunk(tpi_tp_group* g, int pos0, int T, bool last, int* launc
                           NormIn{dptr<float>(m, p.x), dptr<float>(m, p.final_gain), dptr<float>(m, p.ss_part), n_parts, c.rms_eps}, h,
                           c.vocab, dptr<float>(m, p.logits), dptr<float>(m, p.amax_val), dptr<int>(m, p.amax_idx),
                           dptr<unsigned>(m, p.tickets) + bl_, dptr<int>(m, p.tok_hist), dptr<int>(m, p.pos), 1));
+  }
+  for (int i = 0; i < R; ++i) {  // debug arenas (TPI_DEBUG=1): every rank's guard zones are compared after the step
+    TpRank& r = g->ranks[i];
+    if (r.m->plan.n_canaries < 1) break;
+    CK(cudaSetDevice(r.device));
+    LaunchCtx lc = ctx(r);
+    TRY(enqueue_canary_check(r.m, lc));
   }
   return TPI_OK;
 }

