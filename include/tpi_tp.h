@@ -63,10 +63,24 @@ typedef struct tpi_tp_group tpi_tp_group; /* opaque */
 int tpi_tp_rank_slice(const tpi_config *cfg, int n_ranks, int rank, int tensor_id, int64_t *row0, int64_t *n_rows,
                       int64_t *col0, int64_t *n_cols);
 
+/* The same for a heterogeneous partition (Sec. 3.1: device i takes the
+ * proportion p_i of the heads and FFN columns, stronger devices more): rank i
+ * owns kv_heads_per_rank[i] kv heads with their query-head groups and
+ * ffn_cols_per_rank[i] FFN columns, in rank order; both lists have n_ranks
+ * entries >= 1 that add up to n_kv_heads and ffn, and a rank's heads * head_dim
+ * and FFN columns are multiples of 16 bytes of weights (TPI_ERR_SHAPE
+ * otherwise).  NULL lists = the uniform partition. */
+int tpi_tp_rank_slice_p(const tpi_config *cfg, int n_ranks, int rank, const int32_t *kv_heads_per_rank,
+                        const int32_t *ffn_cols_per_rank, int tensor_id, int64_t *row0, int64_t *n_rows, int64_t *col0,
+                        int64_t *n_cols);
+
 /* Arena sizes rank `rank` needs (its slice of the model, its KV heads, its
  * receive buffers).  Pure host arithmetic. */
 int tpi_tp_query_arena(const tpi_config *cfg, int n_ranks, int rank, int window_blocks, size_t *dev_bytes,
                        size_t *host_bytes);
+
+int tpi_tp_query_arena_p(const tpi_config *cfg, int n_ranks, int rank, const int32_t *kv_heads_per_rank,
+                         const int32_t *ffn_cols_per_rank, int window_blocks, size_t *dev_bytes, size_t *host_bytes);
 
 /* Builds the R ranks.  res: HOST array of n_ranks resource sets (arenas on the
  * rank's device, streams of that device; both streams required).  devices: HOST
@@ -76,6 +90,10 @@ int tpi_tp_query_arena(const tpi_config *cfg, int n_ranks, int rank, int window_
  * devices, peer access between them must be possible (it is enabled here). */
 int tpi_tp_create(const tpi_config *cfg, int n_ranks, const tpi_resources *res, const int *devices, tpi_fill_fn fill,
                   void *user, int window_blocks, tpi_tp_group **out);
+/* The same with a heterogeneous partition (lists as in tpi_tp_rank_slice_p). */
+int tpi_tp_create_p(const tpi_config *cfg, int n_ranks, const int32_t *kv_heads_per_rank, const int32_t *ffn_cols_per_rank,
+                    const tpi_resources *res, const int *devices, tpi_fill_fn fill, void *user, int window_blocks,
+                    tpi_tp_group **out);
 void tpi_tp_free(tpi_tp_group *g);
 
 /* Algorithm 1 / 2 for a prompt and for one position; arguments as tpi_prefill /

@@ -6,11 +6,18 @@
 
 namespace {
 
+// Sec. 3.1 Step 1: rank i takes the proportion p_i of the attention heads (whole kv-head groups) and of the FFN columns.
+// Prefix sums over the ranks, R + 1 entries each.
+struct Partition {
+  std::vector<int> kv0, f0;
+};
+
 struct RankFill {  // the weight source as rank `rank` sees it: local tensors cut out of the unsharded ones
   tpi_fill_fn fill = nullptr;
   void* user = nullptr;
   tpi_config cfg{};  // the unsharded model
   int R = 1, rank = 0;
+  Partition part;
   std::vector<char> tmp;
 };
 
@@ -33,21 +40,49 @@ struct TpRank {
 size_t tp_half_floats(const tpi_config& c, int R) { return (size_t)R * c.max_prefill * c.hidden; }
 size_t tp_tail_bytes(const tpi_config& c, int R) { return align_up((size_t)2 * tp_half_floats(c, R) * 4, 256) + 3 * 256; }
 
-int slice_of(const tpi_config& c, int R, int rank, int tid, int64_t* row0, int64_t* n_rows, int64_t* col0, int64_t* n_cols) {
-  if (R < 1 || R > TPI_TP_MAX_RANKS || rank < 0 || rank >= R) return fail(TPI_ERR_INVALID_ARG, "rank %d of %d", rank, R);
-  if (c.n_heads % R || c.n_kv_heads % R || c.ffn % R)
-    return fail(TPI_ERR_SHAPE, "n_ranks=%d must divide heads (%d), kv heads (%d) and ffn (%d)", R, c.n_heads, c.n_kv_heads, c.ffn);
-  const int64_t h = c.hidden, d = c.head_dim, al = c.n_heads / R, bl = c.n_kv_heads / R, sl = c.ffn / R;
+// The uniform partition p_i = 1/R (lists null), or the given one; validated.
+int make_partition(const tpi_config& c, int R, const int32_t* kv_heads, const int32_t* ffn_cols, Partition* out) {
+  if (R < 1 || R > TPI_TP_MAX_RANKS) return fail(TPI_ERR_INVALID_ARG, "n_ranks must be in [1, %d]", TPI_TP_MAX_RANKS);
+  if ((kv_heads == nullptr) != (ffn_cols == nullptr)) return fail(TPI_ERR_INVALID_ARG, "give both lists or neither");
+  if (c.n_heads % c.n_kv_heads) return fail(TPI_ERR_SHAPE, "kv heads must divide heads");
+  out->kv0.assign(R + 1, 0);
+  out->f0.assign(R + 1, 0);
+  if (!kv_heads) {
+    if (c.n_heads % R || c.n_kv_heads % R || c.ffn % R)
+      return fail(TPI_ERR_SHAPE, "n_ranks=%d must divide heads (%d), kv heads (%d) and ffn (%d)", R, c.n_heads, c.n_kv_heads, c.ffn);
+    for (int i = 0; i <= R; ++i) { out->kv0[i] = c.n_kv_heads / R * i; out->f0[i] = c.ffn / R * i; }
+    return TPI_OK;
+  }
+  const int vec = c.dtype == TPI_BF16 ? 8 : 4, grp = c.n_heads / c.n_kv_heads;
+  for (int i = 0; i < R; ++i) {
+    if (kv_heads[i] < 1 || ffn_cols[i] < 1) return fail(TPI_ERR_SHAPE, "every rank needs at least one kv head and one FFN column");
+    if (ffn_cols[i] % vec || (kv_heads[i] * grp * c.head_dim) % vec)
+      return fail(TPI_ERR_SHAPE, "a rank's FFN columns and heads*d must be multiples of %d elements (16 bytes)", vec);
+    out->kv0[i + 1] = out->kv0[i] + kv_heads[i];
+    out->f0[i + 1] = out->f0[i] + ffn_cols[i];
+  }
+  if (out->kv0[R] != c.n_kv_heads || out->f0[R] != c.ffn)
+    return fail(TPI_ERR_SHAPE, "the ranks' kv heads (%d of %d) and FFN columns (%d of %d) must add up", out->kv0[R], c.n_kv_heads, out->f0[R], c.ffn);
+  return TPI_OK;
+}
+
+int slice_of(const tpi_config& c, const Partition& part, int rank, int tid, int64_t* row0, int64_t* n_rows, int64_t* col0, int64_t* n_cols) {
+  const int R = (int)part.kv0.size() - 1;
+  if (rank < 0 || rank >= R) return fail(TPI_ERR_INVALID_ARG, "rank %d of %d", rank, R);
+  const int64_t h = c.hidden, d = c.head_dim, grp = c.n_heads / c.n_kv_heads;
+  const int64_t q0 = (int64_t)part.kv0[rank] * grp * d, qn = (int64_t)(part.kv0[rank + 1] - part.kv0[rank]) * grp * d;  // query rows
+  const int64_t k0 = (int64_t)part.kv0[rank] * d, kn = (int64_t)(part.kv0[rank + 1] - part.kv0[rank]) * d;              // key / value rows
+  const int64_t s0 = part.f0[rank], sn = part.f0[rank + 1] - part.f0[rank];                                                // FFN columns
   int64_t r0 = 0, nr = 0, c0 = 0, nc = h;
   switch (tid) {
     case TPI_T_EMB: case TPI_T_HEAD: nr = rank == 0 ? c.vocab : 0; break;
     case TPI_T_FINAL_NORM: nr = rank == 0 ? 1 : 0; break;
     case TPI_T_ATTN_NORM: case TPI_T_FFN_NORM: nr = 1; break;
-    case TPI_T_WQ: r0 = rank * al * d; nr = al * d; break;
-    case TPI_T_WK: case TPI_T_WV: r0 = rank * bl * d; nr = bl * d; break;
-    case TPI_T_WO: nr = h; c0 = rank * al * d; nc = al * d; break;
-    case TPI_T_WGATE: case TPI_T_WUP: r0 = rank * sl; nr = sl; break;
-    case TPI_T_WDOWN: nr = h; c0 = rank * sl; nc = sl; break;
+    case TPI_T_WQ: r0 = q0; nr = qn; break;
+    case TPI_T_WK: case TPI_T_WV: r0 = k0; nr = kn; break;
+    case TPI_T_WO: nr = h; c0 = q0; nc = qn; break;
+    case TPI_T_WGATE: case TPI_T_WUP: r0 = s0; nr = sn; break;
+    case TPI_T_WDOWN: nr = h; c0 = s0; nc = sn; break;
     default: return fail(TPI_ERR_INVALID_ARG, "unknown tensor id %d", tid);
   }
   if (row0) *row0 = r0;
@@ -63,7 +98,7 @@ int rank_fill(void* user, int tid, int layer, int64_t row0, int64_t n, void* dst
   const tpi_config& c = f->cfg;
   const size_t B = elem_size(c.dtype);
   int64_t r0, nr, c0, nc;
-  if (slice_of(c, f->R, f->rank, tid, &r0, &nr, &c0, &nc)) return 1;
+  if (slice_of(c, f->part, f->rank, tid, &r0, &nr, &c0, &nc)) return 1;
   if (nr == 0) {  // a tensor this rank does not hold (workers: embedding, head, final norm): a one-row placeholder
     memset(dst, 0, (size_t)n * nc * B);
     return 0;
@@ -83,11 +118,11 @@ int rank_fill(void* user, int tid, int layer, int64_t row0, int64_t n, void* dst
   return 0;
 }
 
-tpi_config local_cfg(const tpi_config& c, int R, int rank) {
+tpi_config local_cfg(const tpi_config& c, const Partition& part, int rank) {
   tpi_config l = c;
-  l.n_heads = c.n_heads / R;
-  l.n_kv_heads = c.n_kv_heads / R;
-  l.ffn = c.ffn / R;
+  l.n_kv_heads = part.kv0[rank + 1] - part.kv0[rank];
+  l.n_heads = l.n_kv_heads * (c.n_heads / c.n_kv_heads);
+  l.ffn = part.f0[rank + 1] - part.f0[rank];
   if (rank != 0) l.vocab = 1;  // workers hold no embedding and no head (Sec. 3.1: they reside on the master)
   return l;
 }
@@ -97,6 +132,7 @@ tpi_config local_cfg(const tpi_config& c, int R, int rank) {
 struct tpi_tp_group {
   tpi_config cfg{};
   int R = 0, window = 0;
+  Partition part;
   std::vector<TpRank> ranks;
   int events = 1, wait_polls = 1 << 21, drop_rank = -1, pdl = 1, batched_prompt = 1, use_graph = 1;
   cudaGraphExec_t graph_exec = nullptr;  // one decode position of ALL ranks (resident groups only)
@@ -138,7 +174,6 @@ int enqueue_step(tpi_tp_group* g, bool with_head, int* launches, bool force_edge
   const tpi_config& c = g->cfg;
   const bool edges = g->events || force_edges;  // inside a graph capture the cross-stream waits ARE the graph's edges
   const int R = g->R, h = c.hidden, d = c.head_dim, dt = c.dtype, L = c.n_layers;
-  const int al = c.n_heads / R, bl_ = c.n_kv_heads / R, sl = c.ffn / R;
   auto ctx = [&](TpRank& r) { return LaunchCtx{r.m->cs, g->pdl != 0, launches}; };
   auto drop_now = [&](int rank) {  // one-shot failure injection: this rank computes but never publishes
     if (g->drop_rank != rank) return 0;
@@ -190,6 +225,7 @@ int enqueue_step(tpi_tp_group* g, bool with_head, int* launches, bool force_edge
         const BlockLayout& bl = p.bl;
         CK(cudaSetDevice(r.device));
         LaunchCtx lc = ctx(r);
+        const int al = r.lcfg.n_heads, bl_ = r.lcfg.n_kv_heads, sl = r.lcfg.ffn;  // this rank's share
         BlockRef br;
         TRY(acquire_block(m, 2 * l + blk, &br));
         const NormIn in{dptr<float>(m, p.x), (const float*)br.base, dptr<float>(m, p.ss_part), rowshard_fused_parts(h), c.rms_eps};
@@ -222,7 +258,7 @@ int enqueue_step(tpi_tp_group* g, bool with_head, int* launches, bool force_edge
     CK(launch_head_argmax(lc, dt, m->dev + p.head,
                           NormIn{dptr<float>(m, p.x), dptr<float>(m, p.final_gain), dptr<float>(m, p.ss_part), rowshard_fused_parts(h), c.rms_eps},
                           h, c.vocab, dptr<float>(m, p.logits), dptr<float>(m, p.amax_val), dptr<int>(m, p.amax_idx),
-                          dptr<unsigned>(m, p.tickets) + bl_, dptr<int>(m, p.tok_hist), dptr<int>(m, p.pos), 1));
+                          dptr<unsigned>(m, p.tickets) + r.lcfg.n_kv_heads, dptr<int>(m, p.tok_hist), dptr<int>(m, p.pos), 1));
   }
   for (int i = 0; i < R; ++i) {  // debug arenas (TPI_DEBUG=1): every rank's guard zones are compared after the step
     TpRank& r = g->ranks[i];
@@ -243,8 +279,6 @@ int enqueue_step(tpi_tp_group* g, bool with_head, int* launches, bool force_edge
 int enqueue_prompt_chunk(tpi_tp_group* g, int pos0, int T, bool last, int* launches) {
   const tpi_config& c = g->cfg;
   const int R = g->R, h = c.hidden, d = c.head_dim, dt = c.dtype, L = c.n_layers;
-  const int al = c.n_heads / R, bl_ = c.n_kv_heads / R, sl = c.ffn / R;
-  const int qkv_cols = (al + 2 * bl_) * d;
   const size_t half = tp_half_floats(c, R);
   auto ctx = [&](TpRank& r) { return LaunchCtx{r.m->cs, g->pdl != 0, launches}; };
   auto drop_now = [&](int rank) {
@@ -252,9 +286,15 @@ int enqueue_prompt_chunk(tpi_tp_group* g, int pos0, int T, bool last, int* launc
     g->drop_rank = -1;
     return 1;
   };
-  const bool tc = dt == TPI_BF16 && g->ranks[0].m->opt_tensor && gemm_tc_supported(h, h, qkv_cols) && gemm_tc_supported(h, h, 2 * sl) &&
-                  gemm_tc_supported(al * d, al * d, h) && gemm_tc_supported(sl, sl, h);
-  const int act_mode = tc ? 2 : 0;  // split bf16 activations on the tensor cores, fp32 otherwise
+  // split bf16 activations on the tensor cores where every contraction of EVERY rank qualifies (all ranks use the same
+  // arithmetic, so that the partition does not change which kernels run), fp32 SIMT otherwise
+  bool tc = dt == TPI_BF16 && g->ranks[0].m->opt_tensor;
+  for (int i = 0; i < R && tc; ++i) {
+    const tpi_config& lc_ = g->ranks[i].lcfg;
+    tc = gemm_tc_supported(h, h, (lc_.n_heads + 2 * lc_.n_kv_heads) * d) && gemm_tc_supported(h, h, 2 * lc_.ffn) &&
+         gemm_tc_supported(lc_.n_heads * d, lc_.n_heads * d, h) && gemm_tc_supported(lc_.ffn, lc_.ffn, h);
+  }
+  const int act_mode = tc ? 2 : 0;
   const bool fuse_norm = g->window <= 0;  // a streamed rank may not hold the next block's gain yet
   auto gemm = [&](TpRank& r, LaunchCtx& lc, const float* A, int lda, const void* W, float* Y, int ldy, int n_out, int K) -> int {
     if (tc) {
@@ -310,6 +350,7 @@ int enqueue_prompt_chunk(tpi_tp_group* g, int pos0, int T, bool last, int* launc
         const BlockLayout& bl = p.bl;
         CK(cudaSetDevice(r.device));
         LaunchCtx lc = ctx(r);
+        const int al = r.lcfg.n_heads, bl_ = r.lcfg.n_kv_heads, sl = r.lcfg.ffn, qkv_cols = (al + 2 * bl_) * d;
         float *X = dptr<float>(m, p.pX), *Xn = dptr<float>(m, p.pXn), *PART = dptr<float>(m, p.pPART);
         BlockRef br;
         TRY(acquire_block(m, 2 * l + blk, &br));
@@ -375,7 +416,7 @@ int enqueue_prompt_chunk(tpi_tp_group* g, int pos0, int T, bool last, int* launc
     CK(launch_head_argmax(lc, dt, m->dev + p.head,
                           NormIn{dptr<float>(m, p.x), dptr<float>(m, p.final_gain), dptr<float>(m, p.ss_part), n_parts, c.rms_eps}, h,
                           c.vocab, dptr<float>(m, p.logits), dptr<float>(m, p.amax_val), dptr<int>(m, p.amax_idx),
-                          dptr<unsigned>(m, p.tickets) + bl_, dptr<int>(m, p.tok_hist), dptr<int>(m, p.pos), 1));
+                          dptr<unsigned>(m, p.tickets) + r.lcfg.n_kv_heads, dptr<int>(m, p.tok_hist), dptr<int>(m, p.pos), 1));
   }
   for (int i = 0; i < R; ++i) {  // debug arenas (TPI_DEBUG=1): every rank's guard zones are compared after the step
     TpRank& r = g->ranks[i];
@@ -565,17 +606,30 @@ int run_positions(tpi_tp_group* g, const int32_t* tokens, int n_given, int n_pos
 
 }  // namespace
 
+extern "C" int tpi_tp_rank_slice_p(const tpi_config* cfg, int n_ranks, int rank, const int32_t* kv_heads_per_rank,
+                                   const int32_t* ffn_cols_per_rank, int tensor_id, int64_t* row0, int64_t* n_rows, int64_t* col0,
+                                   int64_t* n_cols) {
+  if (!cfg) return fail(TPI_ERR_INVALID_ARG, "null config");
+  Partition part;
+  TRY(make_partition(*cfg, n_ranks, kv_heads_per_rank, ffn_cols_per_rank, &part));
+  return slice_of(*cfg, part, rank, tensor_id, row0, n_rows, col0, n_cols);
+}
 extern "C" int tpi_tp_rank_slice(const tpi_config* cfg, int n_ranks, int rank, int tensor_id, int64_t* row0, int64_t* n_rows,
                                  int64_t* col0, int64_t* n_cols) {
-  if (!cfg) return fail(TPI_ERR_INVALID_ARG, "null config");
-  return slice_of(*cfg, n_ranks, rank, tensor_id, row0, n_rows, col0, n_cols);
+  return tpi_tp_rank_slice_p(cfg, n_ranks, rank, nullptr, nullptr, tensor_id, row0, n_rows, col0, n_cols);
 }
 
 extern "C" int tpi_tp_query_arena(const tpi_config* cfg, int n_ranks, int rank, int window_blocks, size_t* dev_bytes,
                                   size_t* host_bytes) {
+  return tpi_tp_query_arena_p(cfg, n_ranks, rank, nullptr, nullptr, window_blocks, dev_bytes, host_bytes);
+}
+extern "C" int tpi_tp_query_arena_p(const tpi_config* cfg, int n_ranks, int rank, const int32_t* kv_heads_per_rank,
+                                    const int32_t* ffn_cols_per_rank, int window_blocks, size_t* dev_bytes, size_t* host_bytes) {
   if (!cfg) return fail(TPI_ERR_INVALID_ARG, "null config");
-  TRY(slice_of(*cfg, n_ranks, rank, TPI_T_WQ, nullptr, nullptr, nullptr, nullptr));
-  const tpi_config l = local_cfg(*cfg, n_ranks, rank);
+  Partition part;
+  TRY(make_partition(*cfg, n_ranks, kv_heads_per_rank, ffn_cols_per_rank, &part));
+  TRY(slice_of(*cfg, part, rank, TPI_T_WQ, nullptr, nullptr, nullptr, nullptr));
+  const tpi_config l = local_cfg(*cfg, part, rank);
   size_t d = 0, hb = 0;
   TRY(tpi_query_arena(&l, 1, window_blocks, window_blocks > 0, &d, &hb));
   if (dev_bytes) *dev_bytes = align_up(d, 256) + tp_tail_bytes(*cfg, n_ranks);
@@ -599,8 +653,14 @@ extern "C" void tpi_tp_free(tpi_tp_group* g) {
 
 extern "C" int tpi_tp_create(const tpi_config* cfg, int n_ranks, const tpi_resources* res, const int* devices, tpi_fill_fn fill,
                              void* user, int window_blocks, tpi_tp_group** out) {
+  return tpi_tp_create_p(cfg, n_ranks, nullptr, nullptr, res, devices, fill, user, window_blocks, out);
+}
+extern "C" int tpi_tp_create_p(const tpi_config* cfg, int n_ranks, const int32_t* kv_heads_per_rank, const int32_t* ffn_cols_per_rank,
+                               const tpi_resources* res, const int* devices, tpi_fill_fn fill, void* user, int window_blocks,
+                               tpi_tp_group** out) {
   if (!cfg || !res || !fill || !out || window_blocks < 0) return fail(TPI_ERR_INVALID_ARG, "null or negative argument");
-  TRY(slice_of(*cfg, n_ranks, 0, TPI_T_WQ, nullptr, nullptr, nullptr, nullptr));
+  Partition part;
+  TRY(make_partition(*cfg, n_ranks, kv_heads_per_rank, ffn_cols_per_rank, &part));
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return fail(TPI_ERR_CUDA, "no CUDA device: this library has no CPU path");
   DeviceGuard guard;
@@ -608,6 +668,7 @@ extern "C" int tpi_tp_create(const tpi_config* cfg, int n_ranks, const tpi_resou
   if (!g) return fail(TPI_ERR_NOMEM, "out of host memory");
   g->cfg = *cfg;
   g->R = n_ranks;
+  g->part = part;
   g->window = window_blocks;
   g->ranks.resize(n_ranks);  // never resized again: the ranks' weight sources are referenced by address
   auto bail = [&](int code) { tpi_tp_free(g); return code; };
@@ -629,10 +690,10 @@ extern "C" int tpi_tp_create(const tpi_config* cfg, int n_ranks, const tpi_resou
   for (int i = 0; i < n_ranks; ++i) {
     TpRank& r = g->ranks[i];
     if (cudaSetDevice(r.device) != cudaSuccess) return bail(fail(TPI_ERR_CUDA, "cudaSetDevice(%d) failed", r.device));
-    r.lcfg = local_cfg(*cfg, n_ranks, i);
-    r.rf.fill = fill; r.rf.user = user; r.rf.cfg = *cfg; r.rf.R = n_ranks; r.rf.rank = i;
+    r.lcfg = local_cfg(*cfg, part, i);
+    r.rf.fill = fill; r.rf.user = user; r.rf.cfg = *cfg; r.rf.R = n_ranks; r.rf.rank = i; r.rf.part = part;
     size_t need_d = 0, need_h = 0;
-    int rc = tpi_tp_query_arena(cfg, n_ranks, i, window_blocks, &need_d, &need_h);
+    int rc = tpi_tp_query_arena_p(cfg, n_ranks, i, kv_heads_per_rank, ffn_cols_per_rank, window_blocks, &need_d, &need_h);
     if (rc) return bail(rc);
     if (res[i].dev_bytes < need_d) return bail(fail(TPI_ERR_NOMEM, "rank %d: device arena too small: need %zu bytes, have %zu", i, need_d, res[i].dev_bytes));
     r.tail_bytes = tp_tail_bytes(*cfg, n_ranks);
@@ -709,10 +770,11 @@ extern "C" int tpi_tp_get_hidden(tpi_tp_group* g, int rank, int layer, int which
 
 extern "C" int tpi_tp_get_kv(tpi_tp_group* g, int layer, int kv_head, int pos0, int n, float* k_dst, float* v_dst) {
   if (!g || kv_head < 0 || kv_head >= g->cfg.n_kv_heads) return fail(TPI_ERR_INVALID_ARG, "bad argument");
-  const int per = g->cfg.n_kv_heads / g->R, owner = kv_head / per;
+  int owner = 0;
+  while (kv_head >= g->part.kv0[owner + 1]) ++owner;
   DeviceGuard guard;
   CK(cudaSetDevice(g->ranks[owner].device));
-  return tpi_get_kv(g->ranks[owner].m, layer, kv_head % per, pos0, n, k_dst, v_dst);
+  return tpi_get_kv(g->ranks[owner].m, layer, kv_head - g->part.kv0[owner], pos0, n, k_dst, v_dst);
 }
 
 extern "C" int tpi_tp_set_option(tpi_tp_group* g, int option, int value) {

@@ -14,6 +14,18 @@ from .binding import (FILL_FN, T_WDOWN, T_WO, TPI_BF16, TpiConfig, TpiResources,
 OPT_EVENTS, OPT_WAIT_POLLS, OPT_DROP_PUSH, OPT_PDL, OPT_BATCHED_PROMPT, OPT_GRAPH = 0, 1, 2, 3, 4, 5
 _P, _I = C.c_void_p, C.c_int
 _I64P = C.POINTER(C.c_int64)
+_I32P = C.POINTER(C.c_int32)
+
+
+def _lists(partition, n_ranks):
+    """(kv heads per rank, FFN columns per rank) -> two int32 arrays (kept alive by the caller) or (None, None)."""
+    if partition is None:
+        return None, None, None
+    kv = np.ascontiguousarray(partition[0], dtype=np.int32)
+    ff = np.ascontiguousarray(partition[1], dtype=np.int32)
+    if kv.shape != (n_ranks,) or ff.shape != (n_ranks,):
+        raise ValueError("one entry per rank in both lists")
+    return kv.ctypes.data_as(_I32P), ff.ctypes.data_as(_I32P), (kv, ff)
 
 
 class TpStats(C.Structure):
@@ -25,6 +37,10 @@ class TpStats(C.Structure):
 TP_SYMBOLS = {
     "tpi_tp_rank_slice": (_I, [C.POINTER(TpiConfig), _I, _I, _I, _I64P, _I64P, _I64P, _I64P]),
     "tpi_tp_query_arena": (_I, [C.POINTER(TpiConfig), _I, _I, _I, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
+    "tpi_tp_rank_slice_p": (_I, [C.POINTER(TpiConfig), _I, _I, _I32P, _I32P, _I, _I64P, _I64P, _I64P, _I64P]),
+    "tpi_tp_query_arena_p": (_I, [C.POINTER(TpiConfig), _I, _I, _I32P, _I32P, _I, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
+    "tpi_tp_create_p": (_I, [C.POINTER(TpiConfig), _I, _I32P, _I32P, C.POINTER(TpiResources), C.POINTER(C.c_int), FILL_FN, _P, _I,
+                             C.POINTER(_P)]),
     "tpi_tp_create": (_I, [C.POINTER(TpiConfig), _I, C.POINTER(TpiResources), C.POINTER(C.c_int), FILL_FN, _P, _I, C.POINTER(_P)]),
     "tpi_tp_free": (None, [_P]),
     "tpi_tp_prefill": (_I, [_P, C.POINTER(C.c_int32), _I, C.POINTER(C.c_int32), C.POINTER(C.c_float)]),
@@ -52,16 +68,19 @@ def _tp():
     return L
 
 
-def rank_slice(cfg: TpiConfig, n_ranks: int, rank: int, tensor_id: int):
-    """(row0, n_rows, col0, n_cols) of the unsharded tensor that `rank` holds (host arithmetic, no GPU)."""
+def rank_slice(cfg: TpiConfig, n_ranks: int, rank: int, tensor_id: int, partition=None):
+    """(row0, n_rows, col0, n_cols) of the unsharded tensor that `rank` holds (host arithmetic, no GPU).
+    partition: (kv heads per rank, FFN columns per rank) or None for the uniform 1/R."""
     v = [C.c_int64() for _ in range(4)]
-    _check(_tp().tpi_tp_rank_slice(C.byref(cfg), n_ranks, rank, tensor_id, *[C.byref(x) for x in v]))
+    kv, ff, _keep = _lists(partition, n_ranks)
+    _check(_tp().tpi_tp_rank_slice_p(C.byref(cfg), n_ranks, rank, kv, ff, tensor_id, *[C.byref(x) for x in v]))
     return tuple(x.value for x in v)
 
 
-def query_arena(cfg: TpiConfig, n_ranks: int, rank: int, window_blocks: int = 0):
+def query_arena(cfg: TpiConfig, n_ranks: int, rank: int, window_blocks: int = 0, partition=None):
     d, h = C.c_size_t(), C.c_size_t()
-    _check(_tp().tpi_tp_query_arena(C.byref(cfg), n_ranks, rank, window_blocks, C.byref(d), C.byref(h)))
+    kv, ff, _keep = _lists(partition, n_ranks)
+    _check(_tp().tpi_tp_query_arena_p(C.byref(cfg), n_ranks, rank, kv, ff, window_blocks, C.byref(d), C.byref(h)))
     return d.value, h.value
 
 
@@ -69,7 +88,7 @@ class Group:
     """R ranks in this process; `devices` gives each rank's CUDA device (default: all on `device`)."""
 
     def __init__(self, cfg: TpiConfig, fill, n_ranks: int, window_blocks: int = 0, devices: Optional[Sequence[int]] = None,
-                 device: int = 0):
+                 device: int = 0, partition=None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2410_00531_b200 needs a CUDA device (sm_100a); there is no CPU path")
@@ -78,7 +97,7 @@ class Group:
         self.dev, self.host, self.streams = [], [], []
         res = (TpiResources * n_ranks)()
         for i in range(n_ranks):
-            d_need, h_need = query_arena(cfg, n_ranks, i, window_blocks)
+            d_need, h_need = query_arena(cfg, n_ranks, i, window_blocks, partition)
             torch.cuda.set_device(devs[i])
             self.dev.append(torch.empty(d_need, dtype=torch.uint8, device=f"cuda:{devs[i]}"))
             self.host.append(torch.empty(h_need, dtype=torch.uint8, pin_memory=True))
@@ -100,7 +119,8 @@ class Group:
         self._cb = FILL_FN(_cb)
         h = _P()
         dv = (C.c_int * n_ranks)(*devs)
-        _check(_tp().tpi_tp_create(C.byref(cfg), n_ranks, res, dv, self._cb, None, window_blocks, C.byref(h)))
+        kv, ff, _keep = _lists(partition, n_ranks)
+        _check(_tp().tpi_tp_create_p(C.byref(cfg), n_ranks, kv, ff, res, dv, self._cb, None, window_blocks, C.byref(h)))
         self.h = h
 
     def prefill(self, tokens, vocab: int = 0):

@@ -11,9 +11,9 @@ from tests.helpers import check_logits, close_elementwise, gpu_session, make_ora
 pytestmark = pytest.mark.gpu
 
 
-def _group(shape, R, max_seq, window=0, max_prefill=None):
+def _group(shape, R, max_seq, window=0, max_prefill=None, partition=None):
     import paper_2410_00531_b200.tp as TP
-    return TP.Group(tpi_config(shape, max_seq, max_prefill or max_seq), S.synth_fill(shape), R, window)
+    return TP.Group(tpi_config(shape, max_seq, max_prefill or max_seq), S.synth_fill(shape), R, window, partition=partition)
 
 
 CASES = {
@@ -116,6 +116,42 @@ def test_prompt_pass_of_the_ranks_gives_the_emulated_model_s_prompt_pass_bits(ca
     for a, b in zip(h_tp, h_em):
         assert np.array_equal(a, b)
     assert np.array_equal(kv_tp[0], kv_em[0]) and np.array_equal(kv_tp[1], kv_em[1])
+
+
+@pytest.mark.parametrize("case", ["f32_gqa", "bf16_8b_widths"])
+def test_ranks_with_unequal_shares_match_the_oracle(case):
+    """Sec. 3.1's proportions p_i on real ranks: every rank holds a different number of kv-head groups and FFN columns
+    (different kernels' shapes per rank), against the oracle's per-device form with the same partition; prompt pass
+    (batched), decode, all ranks' hidden states equal, cache rows on their owners."""
+    if case == "f32_gqa":
+        shape = S.CONFIGS["C1"].with_(n_heads=8, n_kv_heads=4, head_dim=32, hidden=256, ffn=688, n_layers=3)
+        part, T = ([2, 1, 1], [344, 200, 144]), 11
+    else:
+        shape = S.CONFIGS["C3"].with_(n_layers=2, vocab=32000)
+        part, T = ([4, 2, 1, 1], [7168, 3584, 2048, 1536]), 150
+    R, tol = len(part[0]), tol_for(shape)
+    toks = S.prompt_tokens(shape, T)
+    orc = make_oracle(shape)
+    with _group(shape, R, T + 6, partition=part) as g:
+        tok, lg = g.prefill(toks, shape.vocab)
+        want = orc.forward(toks, n_shards=R, partition=part)
+        check_logits(lg, tok, want, tol)
+        for step in range(3):
+            for l in range(shape.n_layers):
+                for which, key in ((0, "attn"), (1, "ffn")):
+                    h0 = g.get_hidden(0, l, which)
+                    assert close_elementwise(h0, orc.taps[(l, key)][-1], tol)
+                    for r in range(1, R):
+                        assert np.array_equal(g.get_hidden(r, l, which), h0)
+            feed = int(np.argmax(want))
+            tok, lg = g.decode_step(feed, shape.vocab)
+            want = orc.forward([feed], n_shards=R, partition=part)
+            check_logits(lg, tok, want, tol)
+        for kvh in range(shape.n_kv_heads):
+            k, v = g.get_kv(shape.n_layers - 1, kvh, 0, T + 3)
+            assert close_elementwise(k, orc.cache.K[-1][kvh], tol) and close_elementwise(v, orc.cache.V[-1][kvh], tol)
+    with pytest.raises(Exception):
+        _group(shape, R, 16, partition=(part[0][::-1][:R - 1] + [1], part[1]))   # heads do not add up
 
 
 def test_one_graph_over_all_ranks_matches_stream_launches():

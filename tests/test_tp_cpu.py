@@ -59,6 +59,28 @@ def test_rank_slices_tile_every_tensor_exactly_once(cfg_name, R):
         assert TP.query_arena(cfg, R, 0)[0] - d1 >= 2 * (sh.vocab - 1) * sh.hidden * esz
 
 
+def test_rank_slices_of_a_heterogeneous_partition():
+    """Sec. 3.1's proportions p_i as slices: whole kv-head groups and contiguous FFN columns in rank order, every element
+    of every matrix on exactly one rank; malformed partitions are refused."""
+    sh = S.CONFIGS["C3"]                                   # 32 heads over 8 kv heads (4 per group), FFN 14336
+    cfg = tpi_config(sh, 64, 16)
+    part = ([4, 2, 1, 1], [7168, 3584, 2048, 1536])
+    d, grp = sh.head_dim, sh.n_heads // sh.n_kv_heads
+    kv0 = np.concatenate([[0], np.cumsum(part[0])])
+    f0 = np.concatenate([[0], np.cumsum(part[1])])
+    for r in range(4):
+        assert TP.rank_slice(cfg, 4, r, S.WQ, part) == (kv0[r] * grp * d, part[0][r] * grp * d, 0, sh.hidden)
+        assert TP.rank_slice(cfg, 4, r, S.WK, part)[:2] == (kv0[r] * d, part[0][r] * d)
+        assert TP.rank_slice(cfg, 4, r, S.WO, part) == (0, sh.hidden, kv0[r] * grp * d, part[0][r] * grp * d)
+        assert TP.rank_slice(cfg, 4, r, S.WUP, part)[:2] == (f0[r], part[1][r])
+        assert TP.rank_slice(cfg, 4, r, S.WDOWN, part) == (0, sh.hidden, f0[r], part[1][r])
+    big, small = TP.query_arena(cfg, 4, 1, 0, part)[0], TP.query_arena(cfg, 4, 3, 0, part)[0]
+    assert big > small                                     # a rank with more heads and columns needs more memory
+    for bad in (([4, 2, 1, 2], part[1]), (part[0], [7168, 3584, 2048, 1535]), ([4, 2, 2, 0], part[1]), ([8], [14336])):
+        with pytest.raises((P.TpiError, ValueError)):
+            TP.rank_slice(cfg, 4, 0, S.WQ, bad)
+
+
 WORKER = textwrap.dedent("""
     import os, sys, json
     sys.path.insert(0, %r)
