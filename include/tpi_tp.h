@@ -16,8 +16,8 @@
  *    into every rank's receive buffer (plain stores into the consumer's own
  *    memory, then one flag per source), and every rank adds the R partial sums
  *    in ascending rank order and the shortcut last (Eq. 1-2), so all ranks hold
- *    the same bits.  No rank ever loads from another rank's memory, there is no
- *    multicast of any kind, and every wait for a flag is bounded: when it runs
+ *    the same bits.  No rank ever loads from another rank's memory, every store
+ *    names a single destination, and every wait for a flag is bounded: when it runs
  *    out the kernel returns, the device error word reads "wait timeout", and
  *    the call returns TPI_ERR_TIMEOUT.
  *

@@ -1,7 +1,7 @@
 // Exchange kernels of the one-shard-per-rank form (Sec. 3.2's star allreduce in its one-hop shape): a rank stores its
 // partial sums into every rank's receive area with plain stores and then sets one flag per destination; the consumer
 // waits for the flags with a limit, adds the partial sums in rank order and the shortcut last.  Remote memory is only
-// ever WRITTEN, never read; nothing here is a multicast.
+// ever WRITTEN, never read, and every store names one destination.
 #include "common.cuh"
 #include "gemv_bodies.cuh"
 #include "kernels.h"
