@@ -78,7 +78,7 @@ def ttft_roofline(shape, T, ttft_ms, weight_bytes, hbm_gbs):
 
 def traffic_from_profile(workload: str):
     """DRAM bytes per launch of the dominant kernel, from the committed ncu summary (or None)."""
-    p = os.path.join(ROOT, "profiles", f"gemv_gateup_{workload.lower()}.md")
+    p = os.path.join(ROOT, "profiles", f"wstream_gateup_{workload.lower()}.md")
     if os.path.exists(p):
         m = re.search(r"traffic_bytes_per_launch:\s*([0-9.eE+]+)", open(p).read())
         if m:
@@ -533,7 +533,7 @@ def run_gpu(args, shape):
         "ttft_roofline": ttft_roofline(shape, T, r["ttft_ms"], st["weight_bytes_per_token"], peak),
         "token_roofline": {"bound": "hbm", "bytes_per_token": r["token_bytes"], "achieved": r["token_gbs"], "peak": peak,
                            "unit": "GB/s", "frac": r["token_gbs"] / peak, "peak_kind": peak_kind},
-        "roofline": {"bound": "hbm", "kernel": "gemv_cols_kernel<bf16,EPI_SWIGLU> (gate/up + SwiGLU)",
+        "roofline": {"bound": "hbm", "kernel": "wstream_cols_kernel<bf16,EPI_SWIGLU> (gate/up + SwiGLU)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak if achieved else None, "traffic": traffic_from_profile(args.workload),
                      "bytes_per_launch": sp["dominant_kernel_bytes"], "ms_per_launch": sp["dominant_kernel_ms"],

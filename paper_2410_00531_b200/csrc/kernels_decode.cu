@@ -66,7 +66,7 @@ static void balance_split(long long items, int* grid, int* warps) {
 }
 
 template <typename WT, int R, int EPI, int WARPS>
-__global__ void __launch_bounds__(WARPS * 32) gemv_kernel(const GemvArgs A) {
+__global__ void __launch_bounds__(WARPS * 32) wstream_rows_kernel(const GemvArgs A) {
   extern __shared__ __align__(16) float xs[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int bps = (A.items_per_shard + WARPS - 1) / WARPS;
@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(WARPS * 32) gemv_kernel(const GemvArgs A) {
 
 
 template <typename WT, int EPI, int WARPS>
-__global__ void __launch_bounds__(lb_threads(WARPS), lb_blocks(WARPS)) gemv_cols_kernel(const GemvArgs A) {
+__global__ void __launch_bounds__(lb_threads(WARPS), lb_blocks(WARPS)) wstream_cols_kernel(const GemvArgs A) {
   extern __shared__ __align__(16) float xs[];
   cols_body<WT, EPI, WARPS>(A, xs, blockIdx.x, gridDim.x);
 }
@@ -233,7 +233,7 @@ static cudaError_t launch_gemv_cols_w(const LaunchCtx& c, GemvArgs& A) {
     balance_split(total, &g, &warps);
     grid = g;
   }
-  auto kern = gemv_cols_kernel<WT, EPI, WARPS>;
+  auto kern = wstream_cols_kernel<WT, EPI, WARPS>;
   static PerDeviceOnce attr_done;
   if (!attr_done.get()) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
@@ -262,7 +262,7 @@ static cudaError_t launch_gemv_t(const LaunchCtx& c, GemvArgs& A) {
   A.kc = pick_kc(A.K);
   const int bps = (A.items_per_shard + WARPS - 1) / WARPS;
   const size_t smem = (size_t)A.kc * sizeof(float);
-  auto kern = gemv_kernel<WT, R, EPI, WARPS>;
+  auto kern = wstream_rows_kernel<WT, R, EPI, WARPS>;
   static PerDeviceOnce attr_done;
   if (!attr_done.get()) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
@@ -352,7 +352,7 @@ cudaError_t launch_head_argmax(const LaunchCtx& c, int dt, const void* Whead, co
 
 template <typename WT, int R, int NS, int WARPS>
 __global__ void __launch_bounds__(lb_threads(WARPS), lb_blocks(WARPS))
-    gemv_rowshard_fused_kernel(const RowFusedArgs A) {
+    wstream_rowshard_fused_kernel(const RowFusedArgs A) {
   extern __shared__ __align__(16) float xs[];
   rowfused_body<WT, R, NS, WARPS>(A, xs, blockIdx.x, gridDim.x);
 }
@@ -368,7 +368,7 @@ bool rowshard_fused_supported(int Ks, int n_shards) { return (size_t)Ks * n_shar
 
 template <typename WT, int R, int NS, int WARPS>
 static cudaError_t launch_rowfused_w(const LaunchCtx& c, RowFusedArgs& A) {
-  auto kern = gemv_rowshard_fused_kernel<WT, R, NS, WARPS>;
+  auto kern = wstream_rowshard_fused_kernel<WT, R, NS, WARPS>;
   static PerDeviceOnce attr_done;
   if (!attr_done.get()) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
@@ -448,7 +448,7 @@ cudaError_t launch_gemv_rowshard_fused_unequal(const LaunchCtx& c, int dt, const
   RowFusedArgs L = A;
   auto go = [&](auto wt) -> cudaError_t {
     using WT = decltype(wt);
-    auto kern = gemv_rowshard_fused_kernel<WT, 1, 0, 0>;
+    auto kern = wstream_rowshard_fused_kernel<WT, 1, 0, 0>;
     static PerDeviceOnce attr_done;
     if (!attr_done.get()) {
       cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
