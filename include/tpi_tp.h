@@ -117,7 +117,9 @@ int tpi_tp_get_kv(tpi_tp_group *g, int layer, int kv_head, int pos0, int n, floa
 /* Options.  TPI_TP_OPT_EVENTS (default 1): order every exchange by CUDA events
  * between the ranks' streams; 0 is refused while two ranks share a device.
  * TPI_TP_OPT_WAIT_POLLS: poll limit of the device-side flag waits (default
- * 2097152, about a quarter of a second).  TPI_TP_OPT_DROP_PUSH = r + 1: failure
+ * 2097152, about a quarter of a second, while events order the exchange and the
+ * wait is a backstop; 67108864, about ten seconds, once events are off and a
+ * consumer really waits for ranks that run at their own pace).  TPI_TP_OPT_DROP_PUSH = r + 1: failure
  * injection on the host - rank r's next push computes its partial sums but
  * never publishes them (a rank that "never joins"); the other ranks' waits then
  * run out and the call returns TPI_ERR_TIMEOUT; one-shot, 0 clears it.

@@ -784,6 +784,11 @@ extern "C" int tpi_tp_set_option(tpi_tp_group* g, int option, int value) {
       if (!value && share_a_device(g))
         return fail(TPI_ERR_STATE, "ranks that share a device must be ordered by events: a kernel may not wait for a kernel that is not running");
       g->events = value != 0;
+      // Without events a consumer really waits for its peers (they run on other GPUs at their own pace: first-launch
+      // set-up, a window stall), so the default limit grows from a quarter of a second to about ten seconds.
+      if (!g->events && g->wait_polls == (1 << 21)) g->wait_polls = 1 << 26;
+      if (g->events && g->wait_polls == (1 << 26)) g->wait_polls = 1 << 21;
+      drop_group_graph(g);
       return TPI_OK;
     case TPI_TP_OPT_GRAPH:
       g->use_graph = value != 0;
