@@ -820,10 +820,12 @@ extern "C" int tpi_tp_get_stats(tpi_tp_group* g, tpi_tp_stats* out) {
   s.exchanges_total = g->exchanges;
   s.exchange_bytes_per_token = (uint64_t)2 * c.n_layers * c.hidden * 4 * (g->R - 1);  // a worker; the master adds one broadcast
   const uint64_t B = elem_size(c.dtype);
-  const uint64_t layer = (((uint64_t)(c.n_heads + 2 * c.n_kv_heads) * c.head_dim * c.hidden + (uint64_t)c.hidden * c.n_heads * c.head_dim +
-                           3ull * c.hidden * c.ffn) / g->R) * B + 2ull * c.hidden * 4;
-  s.weight_bytes_worker = layer * c.n_layers;
-  s.weight_bytes_rank0 = s.weight_bytes_worker + (uint64_t)c.vocab * c.hidden * B + (uint64_t)c.hidden * 4;
+  auto layers_of = [&](const tpi_config& l) {  // the bytes of its slices that a rank streams per decoded token
+    return (((uint64_t)(l.n_heads + 2 * l.n_kv_heads) * l.head_dim * l.hidden + (uint64_t)l.hidden * l.n_heads * l.head_dim +
+             3ull * l.hidden * l.ffn) * B + 2ull * l.hidden * 4) * l.n_layers;
+  };
+  s.weight_bytes_worker = layers_of(g->ranks[g->R > 1 ? 1 : 0].lcfg);  // rank 1's share (every worker's, when p_i is uniform)
+  s.weight_bytes_rank0 = layers_of(g->ranks[0].lcfg) + (uint64_t)c.vocab * c.hidden * B + (uint64_t)c.hidden * 4;
   s.last_decode_ms = g->last_decode_ms;
   *out = s;
   return TPI_OK;
