@@ -220,10 +220,10 @@ def whole_job_value(steps: int, ms: float, world: int) -> float:
 
 
 # ------------------------------------------------------------------ GPU arm
-def open_session(P, shape, local, max_seq, prefill_chunk, window=0, retain=0):
+def open_session(P, shape, local, max_seq, prefill_chunk, window=0, retain=0, longest_prompt=0):
     """Load a model (weights from the seeded generator) into fresh arenas; returns (session, seconds)."""
     import torch
-    cfg = tpi_config(shape, max_seq, min(shape.prompt_len, prefill_chunk))
+    cfg = tpi_config(shape, max_seq, min(max(shape.prompt_len, longest_prompt), prefill_chunk))
     t0 = time.perf_counter()
     extra = 0
     if window > 0 and retain > 0:      # room for the kept FFN blocks beside the window (Prop. 6)
@@ -292,16 +292,33 @@ def resident_decode(P, ses, shape, local, K, W, world=1, n_ttft=4):
             "token_bytes": token_bytes, "token_gbs": token_bytes / (dev_ms / K * 1e-3) / 1e9, "barrier": barrier}
 
 
-def resident_leg(P, name, shape, local, K, W, prefill_chunk):
-    """One more resident workload in compact form (tokens/s, whole-token HBM fraction, TTFT and its fraction)."""
+def resident_leg(P, name, shape, local, K, W, prefill_chunk, long_ctx=0):
+    """One more resident workload in compact form (tokens/s, whole-token HBM fraction, TTFT and its fraction).
+    long_ctx > 0: on the same loaded model, also a prompt of that many tokens (TTFT, one pass) and 16 decoded tokens on
+    top of it, reported under "long_context"."""
     T = shape.prompt_len
-    ses, load_s = open_session(P, shape, local, T + W + K + 8, prefill_chunk)
+    peak, kind = measured_peaks()
+    ses, load_s = open_session(P, shape, local, max(T + W + K, long_ctx + 24) + 8, prefill_chunk, longest_prompt=long_ctx)
+    extra = None
     try:
         r = resident_decode(P, ses, shape, local, K, W, n_ttft=3)
+        if long_ctx:
+            sl = shape.with_(prompt_len=long_ctx)
+            rl = resident_decode(P, ses, sl, local, 16, 3, n_ttft=1)
+            trl = ttft_roofline(sl, long_ctx, rl["ttft_ms"], rl["stats"]["weight_bytes_per_token"], peak)
+            extra = {"context": f"{long_ctx + 3}..{long_ctx + 19}", "steps": 16, "tokens_per_s": round(16 / (rl["dev_ms"] * 1e-3), 2),
+                     "hbm_frac": round(rl["token_gbs"] / peak, 4), "ttft_ms": round(rl["ttft_ms"], 1), "ttft_prompt_tokens": long_ctx,
+                     "ttft_bound": trl["bound"], "ttft_frac": round(trl["frac"], 4), "clocks": short_clocks(rl["clocks"])}
     finally:
         close_session(ses)
-    peak, kind = measured_peaks()
     tr = ttft_roofline(shape, T, r["ttft_ms"], r["stats"]["weight_bytes_per_token"], peak)
+    out = _resident_leg_dict(name, shape, K, W, T, r, peak, tr)
+    if extra:
+        out["long_context"] = extra
+    return out
+
+
+def _resident_leg_dict(name, shape, K, W, T, r, peak, tr):
     return {"workload": f"{name} {shape.name} N={shape.n_shards} resident", "steps": K,
             "context": f"{T + W}..{T + W + K}", "tokens_per_s": round(K / (r["dev_ms"] * 1e-3), 2),
             "ms_per_step": round(r["dev_ms"] / K, 4), "hbm_gbs": round(r["token_gbs"], 1),
@@ -444,7 +461,7 @@ def extra_legs(P, args, local):
     if "C3" in want:
         run("C3", lambda: resident_leg(P, "C3", S.CONFIGS["C3"], local, 256, 5, args.prefill_chunk))
     if "C5" in want:
-        run("C5", lambda: resident_leg(P, "C5", S.CONFIGS["C5"], local, 32, 4, args.prefill_chunk))
+        run("C5", lambda: resident_leg(P, "C5", S.CONFIGS["C5"], local, 32, 4, args.prefill_chunk, long_ctx=8192))
     if "TP" in want:
         run("C2_4_ranks_one_gpu", lambda: tp_one_gpu_leg(P, S.CONFIGS["C2"], local, 4, 32, 4))
     if "S5" in want or "S4" in want:
