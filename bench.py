@@ -378,6 +378,15 @@ def streamed_decode(P, ses, shape, local, K, W):
 
 
 def streamed_leg(P, name, shape, local, K, W, window, link_peak, retain=0):
+    # The first launch of a kernel in a process loads its code (tens of milliseconds per kernel): a one-layer resident
+    # model of the same widths runs the prompt pass and two tokens first, so that the TTFT below times the streamed pass.
+    warm = shape.with_(n_layers=1, vocab=1024)
+    wses, _ = open_session(P, warm, local, warm.prompt_len + 8, 4096)
+    try:
+        t, _ = P.prefill(wses.h, S.prompt_tokens(warm), 0)
+        P.decode_run(wses.h, t, 2)
+    finally:
+        close_session(wses)
     ses, load_s = open_session(P, shape, local, shape.prompt_len + W + K + 16, 4096, window, retain)
     try:
         r = streamed_decode(P, ses, shape, local, K, W)
@@ -395,6 +404,8 @@ def streamed_leg(P, name, shape, local, K, W, window, link_peak, retain=0):
             "steps": K, "tokens_per_s": round(r["tokens_per_s"], 4), "ms_per_step": round(r["wall_s"] / K * 1e3, 2),
             "link_GB_per_token": round(r["region_bytes"] / K / 1e9, 3), "link_gbs": round(r["link_gbs"], 2),
             "link_peak_gbs": round(link_peak, 2), "link_frac": round(r["link_gbs"] / link_peak, 4),
+            "ttft_ms": round(r["ttft_ms"], 1), "ttft_prompt_tokens": shape.prompt_len,
+            "ttft_link_frac": round(r["region_bytes"] / K / (r["ttft_ms"] * 1e-3) / 1e9 / link_peak, 4),
             "tau_over_t": [round(sched["tau_attn_ms"] / max(sched["t_attn_ms"], 1e-9), 1),
                            round(sched["tau_ffn_ms"] / max(sched["t_ffn_ms"], 1e-9), 1)],
             "loose_holds": sched["loose_holds"], "clocks": short_clocks(r["clocks"])}
@@ -467,10 +478,10 @@ def extra_legs(P, args, local):
     if "S5" in want or "S4" in want:
         link_peak = host_link_peak(torch, local)
         if "S5" in want:
-            run("C5_streamed", lambda: streamed_leg(P, "C5-shaped", S.CONFIGS["C5"].with_(n_layers=10, prompt_len=64),
+            run("C5_streamed", lambda: streamed_leg(P, "C5-shaped", S.CONFIGS["C5"].with_(n_layers=10, prompt_len=512),
                                                     local, 16, 2, 8, link_peak))
         if "S4" in want:
-            run("C4_streamed", lambda: streamed_leg(P, "C4-shaped", S.CONFIGS["C4"].with_(n_layers=5, prompt_len=64),
+            run("C4_streamed", lambda: streamed_leg(P, "C4-shaped", S.CONFIGS["C4"].with_(n_layers=5, prompt_len=512),
                                                     local, 16, 2, 8, link_peak))
     return legs
 

@@ -280,10 +280,106 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const float* __restrict_
   }
 }
 
+// The same contraction on 128 x 64 tiles for more than 64 positions: 8 x 4 outputs per thread, the next 16-deep slice
+// in flight (registers) while the current one is multiplied.  Every output is still ONE thread's running sum over k in
+// ascending order with the fold every 512, so the bits equal the 64 x 64 kernel's.
+template <typename WT>
+__global__ void __launch_bounds__(256) gemm_simt_wide_kernel(const float* __restrict__ X, long long xbs, int ldx,
+                                                             const WT* __restrict__ W, long long wbs,
+                                                             float* __restrict__ Y, long long ybs, int ldy, int T,
+                                                             int n_out, int K) {
+  pdl_launch_dependents();
+  pdl_wait();  // inputs come from the previous kernel in the stream
+  constexpr int BM = 128, BN = 64, BK = 16, FOLD = 512;
+  __shared__ __align__(16) float Xs[2][BK][BM + 4];
+  __shared__ __align__(16) float Ws[2][BK][BN + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;  // thread: rows ty*4 + {0..3} and 64 + ty*4 + {0..3}, cols tx*4 + {0..3}
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  X += (size_t)blockIdx.z * xbs;
+  W += (size_t)blockIdx.z * wbs;
+  Y += (size_t)blockIdx.z * ybs;
+  const int lrow = tid >> 2, lk = (tid & 3) * 4;  // loader: rows lrow and lrow + 64 of X, row lrow of W, 4 consecutive k
+  float acc[8][4], tot[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = tot[i][j] = 0.f;
+  float4 xa, xb, wv;
+  auto fetch = [&](int k0) {
+    xa = xb = wv = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (k0 + lk < K) {
+      if (m0 + lrow < T) xa = *reinterpret_cast<const float4*>(X + (size_t)(m0 + lrow) * ldx + k0 + lk);
+      if (m0 + 64 + lrow < T) xb = *reinterpret_cast<const float4*>(X + (size_t)(m0 + 64 + lrow) * ldx + k0 + lk);
+      if (n0 + lrow < n_out) {
+        const WT* wp = W + (size_t)(n0 + lrow) * K + k0 + lk;
+        if constexpr (sizeof(WT) == 2) {
+          const uint2 v = *reinterpret_cast<const uint2*>(wp);
+          wv = make_float4(bf16lo(v.x), bf16hi(v.x), bf16lo(v.y), bf16hi(v.y));
+        } else {
+          wv = *reinterpret_cast<const float4*>(wp);
+        }
+      }
+    }
+  };
+  auto stash = [&](int buf) {
+    Xs[buf][lk + 0][lrow] = xa.x; Xs[buf][lk + 1][lrow] = xa.y; Xs[buf][lk + 2][lrow] = xa.z; Xs[buf][lk + 3][lrow] = xa.w;
+    Xs[buf][lk + 0][64 + lrow] = xb.x; Xs[buf][lk + 1][64 + lrow] = xb.y; Xs[buf][lk + 2][64 + lrow] = xb.z; Xs[buf][lk + 3][64 + lrow] = xb.w;
+    Ws[buf][lk + 0][lrow] = wv.x; Ws[buf][lk + 1][lrow] = wv.y; Ws[buf][lk + 2][lrow] = wv.z; Ws[buf][lk + 3][lrow] = wv.w;
+  };
+  fetch(0);
+  stash(0);
+  __syncthreads();
+  int buf = 0;
+  for (int k0 = 0; k0 < K; k0 += BK) {
+    if (k0 && k0 % FOLD == 0) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { tot[i][j] += acc[i][j]; acc[i][j] = 0.f; }
+    }
+    const bool more = k0 + BK < K;
+    if (more) fetch(k0 + BK);  // in flight while this slice is multiplied
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      const float4 a0 = *reinterpret_cast<const float4*>(&Xs[buf][kk][ty * 4]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&Xs[buf][kk][64 + ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&Ws[buf][kk][tx * 4]);
+      const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    if (more) {
+      stash(buf ^ 1);  // the other buffer was last read one iteration ago, behind the barrier below
+      __syncthreads();
+      buf ^= 1;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int m = m0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + (i - 4));
+    if (m >= T) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n < n_out) Y[(size_t)m * ldy + n] = tot[i][j] + acc[i][j];
+    }
+  }
+}
+
 cudaError_t launch_gemm_simt(const LaunchCtx& c, int dt, const float* X, long long x_batch_stride, int ldx,
                              const void* W, long long w_batch_stride_elems, float* Y,
                              long long y_batch_stride, int ldy, int T, int n_out, int K, int n_batch) {
   LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
+  if (T > 64) {
+    dim3 gridw((n_out + 63) / 64, (T + 127) / 128, n_batch);
+    if (dt == DT_BF16)
+      return launch_kernel(nc, gemm_simt_wide_kernel<__nv_bfloat16>, gridw, dim3(256), 0, X, x_batch_stride, ldx,
+                           (const __nv_bfloat16*)W, w_batch_stride_elems, Y, y_batch_stride, ldy, T, n_out, K);
+    return launch_kernel(nc, gemm_simt_wide_kernel<float>, gridw, dim3(256), 0, X, x_batch_stride, ldx, (const float*)W,
+                         w_batch_stride_elems, Y, y_batch_stride, ldy, T, n_out, K);
+  }
   dim3 grid((n_out + 63) / 64, (T + 63) / 64, n_batch);
   if (dt == DT_BF16)
     return launch_kernel(nc, gemm_simt_kernel<__nv_bfloat16>, grid, dim3(256), 0, X, x_batch_stride, ldx,
