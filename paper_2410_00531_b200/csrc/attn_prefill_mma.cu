@@ -48,7 +48,7 @@ __device__ __forceinline__ void store_out(void* base, size_t i, size_t lo_off, f
   }
 }
 
-constexpr int QB = 64, KB = 64;
+constexpr int KB = 64;  // keys per tile of the prompt kernel
 // decode kernel: DW warps per CTA, each takes DKB-key tiles (shorter tiles, more warps: a shorter dependent MMA chain per warp)
 constexpr int DW = 8, DKB = 32;
 
@@ -58,8 +58,9 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) {
   return (uint32_t)(r * (D * 2) + (((c & ~7) | ((c ^ r) & 7)) << 4));
 }
 
-template <int D, int MODE>
-__global__ void __launch_bounds__(128) prefill_attn_mma_kernel(const float* __restrict__ Q, const __nv_bfloat16* kc,
+// QBT queries per CTA (16 per warp): 64, or 32 when 64-query tiles would leave most of the machine idle
+template <int D, int MODE, int QBT>
+__global__ void __launch_bounds__(QBT * 2) prefill_attn_mma_kernel(const float* __restrict__ Q, const __nv_bfloat16* kc,
                                                                const __nv_bfloat16* vc, int T, int pos0, int a, int b,
                                                                int max_seq, void* O, size_t lo_off) {
   constexpr int KS = D / 16;       // k-steps of the QK^T contraction
@@ -72,16 +73,16 @@ __global__ void __launch_bounds__(128) prefill_attn_mma_kernel(const float* __re
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int j = blockIdx.y, kvh = j / (a / b);
-  const int q0 = blockIdx.x * QB;                      // first query row of the CTA
+  const int q0 = blockIdx.x * QBT;                      // first query row of the CTA
   const int row_lo = q0 + warp * 16 + g, row_hi = row_lo + 8;
-  const int n_keys = min(pos0 + min(q0 + QB, T), pos0 + T);  // keys any row of this CTA may see
+  const int n_keys = min(pos0 + min(q0 + QBT, T), pos0 + T);  // keys any row of this CTA may see
   const __nv_bfloat16* kg = kc + (size_t)kvh * max_seq * D;
   const __nv_bfloat16* vg = vc + (size_t)kvh * max_seq * D;
   const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
 
   auto stage_tile = [&](int stage, int k0) {
     // 64 rows x CPR chunks for K and for V; rows beyond the cache's valid range are zero-filled
-    for (int i = threadIdx.x; i < KB * CPR; i += 128) {
+    for (int i = threadIdx.x; i < KB * CPR; i += QBT * 2) {
       const int r = i / CPR, c = i - r * CPR;
       const uint32_t dk = smem_base + stage * 2 * TILE + tile_off<D>(r, c);
       const uint32_t dv = dk + TILE;
@@ -222,10 +223,10 @@ __global__ void __launch_bounds__(128) prefill_attn_mma_kernel(const float* __re
   }
 }
 
-template <int D, int MODE>
-cudaError_t launch_t(const LaunchCtx& c, const float* Q, const void* kc, const void* vc, int T, int pos0, int a, int b,
-                     int max_seq, void* O) {
-  auto kern = prefill_attn_mma_kernel<D, MODE>;
+template <int D, int MODE, int QBT>
+cudaError_t launch_tq(const LaunchCtx& c, const float* Q, const void* kc, const void* vc, int T, int pos0, int a, int b,
+                      int max_seq, void* O) {
+  auto kern = prefill_attn_mma_kernel<D, MODE, QBT>;
   const size_t smem = (size_t)2 * 2 * KB * D * 2;
   static PerDeviceOnce attr_done;
   if (!attr_done.get() && smem > 48 * 1024) {
@@ -233,8 +234,20 @@ cudaError_t launch_t(const LaunchCtx& c, const float* Q, const void* kc, const v
     if (e != cudaSuccess) return e;
     attr_done.set();
   }
-  return launch_kernel(c, kern, dim3((T + QB - 1) / QB, a), dim3(128), smem, Q, (const __nv_bfloat16*)kc,
+  return launch_kernel(c, kern, dim3((T + QBT - 1) / QBT, a), dim3(QBT * 2), smem, Q, (const __nv_bfloat16*)kc,
                        (const __nv_bfloat16*)vc, T, pos0, a, b, max_seq, O, (size_t)T * a * D);
+}
+
+template <int D, int MODE>
+cudaError_t launch_t(const LaunchCtx& c, const float* Q, const void* kc, const void* vc, int T, int pos0, int a, int b,
+                     int max_seq, void* O) {
+  // 64-query tiles unless they would fill less than one CTA per SM: then 32-query tiles (twice the CTAs, half the
+  // serial work of each; a row's arithmetic does not depend on the tile it sits in, so the bits are the same)
+  int sms = 148, dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if ((long long)((T + 63) / 64) * a < sms) return launch_tq<D, MODE, 32>(c, Q, kc, vc, T, pos0, a, b, max_seq, O);
+  return launch_tq<D, MODE, 64>(c, Q, kc, vc, T, pos0, a, b, max_seq, O);
 }
 
 }  // namespace
