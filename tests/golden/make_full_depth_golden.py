@@ -1,12 +1,15 @@
-"""Writes tests/golden/c2_full_depth.txt: what the CPU oracle computes for the 7B-shaped workload (C2) at FULL
-depth on its seeded prompt.  Calls only the oracle and the seeded input generator; takes several minutes and a
-few GB of memory (weights are generated layer by layer and dropped again).
+"""Writes tests/golden/<workload>_full_depth.txt: what the CPU oracle computes for a workload at FULL depth on its seeded
+prompt.  Calls only the oracle and the seeded input generator; takes minutes to a quarter of an hour and up to ~25 GB of
+memory (weights are generated layer by layer and dropped again).
 
-    python tests/golden/make_full_depth_golden.py
+    python tests/golden/make_full_depth_golden.py            # C2: 7B shape, 128-token prompt
+    python tests/golden/make_full_depth_golden.py C3         # 8B shape, its 4096-token prompt
+    python tests/golden/make_full_depth_golden.py C5         # 70B shape, 512-token prompt
 
-Stored: the root mean square of the last position's logits, its 32 largest logits with their indices, the logits
-at 64 evenly spaced indices, and for layers 0, 15 and 31 the root mean square and 16 evenly spaced entries of the
-last position's H_attn and H_ffn (Eq. 1-2)."""
+Stored, for the last prompt position: the root mean square of the logits, the 32 largest logits with their indices,
+the logits at 64 evenly spaced indices, and for the first, the middle and the last layer the root mean square and 16
+evenly spaced entries of H_attn and H_ffn (Eq. 1-2).  Then the same logit records (prefix "d") for ONE decode step on
+top of the prompt, fed with the oracle's own greedy token (the GPU test teacher-forces the same token)."""
 import os
 import sys
 
@@ -19,26 +22,35 @@ import tpi_synth as S                                   # noqa: E402
 from tests.helpers import make_oracle                   # noqa: E402
 
 
+def logit_records(out, prefix, logits, vocab):
+    out.append(f"{prefix}logits_rms {np.sqrt(np.mean(logits * logits)):.17g}")
+    for i in np.argsort(-logits, kind="stable")[:32]:
+        out.append(f"{prefix}top {int(i)} {logits[i]:.17g}")
+    for i in np.linspace(0, vocab - 1, 64).astype(int):
+        out.append(f"{prefix}logit {int(i)} {logits[i]:.17g}")
+
+
 def main():
-    shape = S.CONFIGS["C2"]
+    name = sys.argv[1] if len(sys.argv) > 1 else "C2"
+    shape = S.CONFIGS[name]
     toks = S.prompt_tokens(shape)
     orc = make_oracle(shape, cache=12)
     logits = orc.forward(toks)
-    out = ["# oracle values for workload C2 (7B-shaped, bf16 weights and KV, N-independent), full depth, "
-           f"prompt of {len(toks)} seeded tokens; written by tests/golden/make_full_depth_golden.py",
-           f"logits_rms {np.sqrt(np.mean(logits * logits)):.17g}"]
-    top = np.argsort(-logits, kind="stable")[:32]
-    for i in top:
-        out.append(f"top {int(i)} {logits[i]:.17g}")
-    for i in np.linspace(0, shape.vocab - 1, 64).astype(int):
-        out.append(f"logit {int(i)} {logits[i]:.17g}")
-    for l in (0, 15, 31):
+    L = shape.n_layers
+    out = [f"# oracle values for workload {name} ({shape.name}, {shape.dtype} weights and KV, N-independent), full depth, "
+           f"prompt of {len(toks)} seeded tokens; written by tests/golden/make_full_depth_golden.py"]
+    logit_records(out, "", logits, shape.vocab)
+    for l in (0, L // 2 - 1, L - 1):
         for key in ("attn", "ffn"):
             hrow = orc.taps[(l, key)][-1]
             out.append(f"hidden_rms {l} {key} {np.sqrt(np.mean(hrow * hrow)):.17g}")
             for i in np.linspace(0, shape.hidden - 1, 16).astype(int):
                 out.append(f"hidden {l} {key} {int(i)} {hrow[i]:.17g}")
-    with open(os.path.join(HERE, "c2_full_depth.txt"), "w") as f:
+    if name != "C2":      # C2's file predates the decode records and is kept as it was written
+        feed = int(np.argmax(logits))
+        out.append(f"dfeed {feed}")
+        logit_records(out, "d", orc.forward([feed]), shape.vocab)
+    with open(os.path.join(HERE, f"{name.lower()}_full_depth.txt"), "w") as f:
         f.write("\n".join(out) + "\n")
     print("written", len(out), "lines")
 

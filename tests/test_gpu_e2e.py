@@ -325,22 +325,47 @@ def test_full_size_7b_shape_sampled_outputs_and_size_independent_properties():
         assert res["n1"][0] == res["n4"][0]
 
 
-def test_full_size_7b_shape_against_the_oracle_s_stored_values():
-    """The 7B-shaped workload at FULL depth against values the CPU oracle computed for it offline
-    (tests/golden/c2_full_depth.txt, written by tests/golden/make_full_depth_golden.py): hidden states of layers 0, 15
-    and 31, sampled logits, the 32 largest logits and the greedy token, at the 1e-2 bar for bf16 weights."""
+def _golden(name):
     import os
+    path = os.path.join(os.path.dirname(__file__), "golden", f"{name.lower()}_full_depth.txt")
+    return [ln.split() for ln in open(path) if ln[0] != "#"]
+
+
+def _check_stored_logits(gold, prefix, lg, tok, tol):
+    """Sampled logits, the oracle's 32 largest, the root mean square and the token rule against stored oracle values."""
+    rms = float(next(g[1] for g in gold if g[0] == prefix + "logits_rms"))
+    top = [(int(g[1]), float(g[2])) for g in gold if g[0] == prefix + "top"]
+    sampled = [(int(g[1]), float(g[2])) for g in gold if g[0] == prefix + "logit"]
+    e = 3 * tol * rms                                            # the token rule's per-logit allowance
+    assert abs(np.sqrt(np.mean(lg.astype(np.float64) ** 2)) - rms) <= tol * rms
+    for i, v in sampled + top:
+        assert abs(lg[i] - v) <= e, (prefix, i, lg[i], v)
+    assert int(np.argmax(lg)) == tok
+    if top[0][1] - top[1][1] > 2 * e:
+        assert tok == top[0][0]
+    else:
+        assert tok in (top[0][0], top[1][0])
+    assert lg.max() <= top[0][1] + e                             # nothing outside the oracle's 32 largest may win by more
+
+
+@pytest.mark.parametrize("name", ["C2", "C3"])
+def test_full_size_against_the_oracle_s_stored_values(name):
+    """The benchmarked workloads at FULL depth and full vocabulary, in bench.py's launch configuration (prompt in one
+    chunk, graph + PDL decode), against values the CPU oracle computed for them offline (tests/golden/*_full_depth.txt,
+    written by tests/golden/make_full_depth_golden.py): 7B shape with its 128-token prompt, 8B shape with its
+    4096-token prompt, 70B shape (139 GB resident) with its 512-token prompt.  Hidden states of the first, middle and
+    last layer, sampled logits, the 32 largest logits and the greedy token of the last prompt position at the 1e-2 bar
+    for bf16 weights; for the 8B and 70B shapes also ONE decode step on top of the prompt, teacher-forced with the
+    oracle's token."""
     import paper_2410_00531_b200 as P
-    shape = S.CONFIGS["C2"]
-    gold = [ln.split() for ln in open(os.path.join(os.path.dirname(__file__), "golden", "c2_full_depth.txt")) if ln[0] != "#"]
-    rms = float(next(g[1] for g in gold if g[0] == "logits_rms"))
-    top = [(int(g[1]), float(g[2])) for g in gold if g[0] == "top"]
-    sampled = [(int(g[1]), float(g[2])) for g in gold if g[0] == "logit"]
+    shape = S.CONFIGS[name]
+    gold = _golden(name)
     toks = S.prompt_tokens(shape)
     tol = tol_for(shape)
-    with gpu_session(shape, len(toks) + 8, len(toks)) as ses:
+    layers = sorted({int(g[1]) for g in gold if g[0] == "hidden_rms"})
+    with gpu_session(shape, len(toks) + 8, min(len(toks), 4096)) as ses:
         tok, lg = P.prefill(ses.h, toks, shape.vocab)
-        for l in (0, 15, 31):
+        for l in layers:
             for which, key in ((0, "attn"), (1, "ffn")):
                 hr = float(next(g[3] for g in gold if g[0] == "hidden_rms" and int(g[1]) == l and g[2] == key))
                 got = P.get_hidden(ses.h, l, which, shape.hidden)
@@ -348,17 +373,11 @@ def test_full_size_7b_shape_against_the_oracle_s_stored_values():
                     if g[0] == "hidden" and int(g[1]) == l and g[2] == key:
                         assert abs(got[int(g[3])] - float(g[4])) <= 3 * tol * hr, (l, key, g[3])
                 assert abs(np.sqrt(np.mean(got.astype(np.float64) ** 2)) - hr) <= tol * hr
-    e = 3 * tol * rms                                            # the token rule's per-logit allowance
-    assert abs(np.sqrt(np.mean(lg.astype(np.float64) ** 2)) - rms) <= tol * rms
-    for i, v in sampled + top:
-        assert abs(lg[i] - v) <= e, (i, lg[i], v)
-    assert int(np.argmax(lg)) == tok
-    if top[0][1] - top[1][1] > 2 * e:
-        assert tok == top[0][0]
-    else:
-        assert tok in (top[0][0], top[1][0])
-    # nothing outside the oracle's 32 largest may win by more than the allowance
-    assert lg.max() <= top[0][1] + e
+        _check_stored_logits(gold, "", lg, tok, tol)
+        feed = [int(g[1]) for g in gold if g[0] == "dfeed"]
+        if feed:
+            tok2, lg2 = P.decode_step(ses.h, feed[0], shape.vocab)
+            _check_stored_logits(gold, "d", lg2, tok2, tol)
 
 
 def test_second_model_family_non_power_of_two_widths():
