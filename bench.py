@@ -630,6 +630,58 @@ def run_streamed(args, shape, local, rank):
         print(json.dumps(line), flush=True)
 
 
+def run_timeline(args, shape):
+    """One layer's schedule inside the graph-replayed decode step, from the kernels' own time stamps (a library built
+    with TPI_TIMELINE=1; see paper_2410_00531_b200/build.py).  Prints, per kernel of the LAST layer, when its CTAs
+    start, when their dependency wait returns, when their inputs are staged and when they end, in microseconds from
+    the first CTA of the layer's QKV kernel, then one JSON line with the same numbers.  Not a benchmark line."""
+    import ctypes
+    import numpy as np
+    import torch
+    import paper_2410_00531_b200 as P
+    from paper_2410_00531_b200 import binding
+    lib = binding.lib()
+    fn = lib.tpi_internal_timeline
+    fn.argtypes, fn.restype = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int)], ctypes.c_int
+    lay = (ctypes.c_int * 4)()
+    if not fn(None, lay):
+        raise SystemExit("this library carries no time stamps: TPI_TIMELINE=1 python -m paper_2410_00531_b200.build, "
+                         "then TPI_TIMELINE=1 python bench.py --timeline ...")
+    n_k, n_c, n_s, w0 = lay[0], lay[1], lay[2], lay[3]
+    torch.cuda.set_device(0)
+    buf = torch.zeros(n_k * n_c * n_s, dtype=torch.int64, device="cuda")
+    fn(buf.data_ptr(), lay)
+    ses, _ = open_session(P, shape, 0, shape.prompt_len + args.steps + args.warmup + 8, args.prefill_chunk)
+    try:
+        first, _ = P.prefill(ses.h, S.prompt_tokens(shape), 0)
+        P.decode_run(ses.h, first, args.warmup + args.steps)
+        torch.cuda.synchronize()
+        t = buf.cpu().numpy().reshape(n_k, n_c, n_s)
+    finally:
+        fn(None, lay)
+        close_session(ses)
+    names = [(0, "qkv"), (6, "attention"), (4, "o_proj"), (1, "gate_up"), (5, "down_proj"), (3, "head")]
+    t0, rows = None, {}
+    for k, name in names:
+        e = t[k][(t[k][:, 0] > 0) & (t[k][:, w0:].max(axis=1) > 0)]       # CTAs that did work (an idle split leaves no end stamp)
+        if not len(e):
+            continue
+        t0 = e[:, 0].min() if t0 is None else t0
+        us = lambda x: round(float(x - t0) / 1e3, 2)
+        end = e[:, w0:].max(axis=1)
+        rows[name] = {"ctas": int(len(e)), "entry": [us(e[:, 0].min()), us(e[:, 0].max())],
+                      "wait_returned": [us(e[:, 1].min()), us(e[:, 1].max())],
+                      "staged": [us(e[:, 2].min()), us(e[:, 2].max())] if e[:, 2].max() > 0 else None,
+                      "cta_end": [us(end.min()), us(float(np.median(end))), us(end.max())]}
+        r = rows[name]
+        print(f"{name:10s} ctas {r['ctas']:3d}  entry {r['entry'][0]:7.2f}..{r['entry'][1]:7.2f}  wait returned "
+              f"{r['wait_returned'][0]:7.2f}..{r['wait_returned'][1]:7.2f}  staged "
+              + (f"{r['staged'][0]:7.2f}..{r['staged'][1]:7.2f}" if r["staged"] else "      -         ")
+              + f"  CTA end min {r['cta_end'][0]:7.2f} median {r['cta_end'][1]:7.2f} max {r['cta_end'][2]:7.2f}", file=sys.stderr)
+    print(json.dumps({"timeline_us": rows, "config": {"workload": f"{args.workload} {shape.name}", "layers": shape.n_layers,
+                                                      "context": shape.prompt_len + args.warmup + args.steps}}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -654,6 +706,9 @@ def main():
     ap.add_argument("--tp", type=int, default=0,
                     help="run the workload as this many ranks with one shard each, all on this GPU, and print that leg alone")
     ap.add_argument("--layers", type=int, default=0, help="override the depth (small captures under a profiler)")
+    ap.add_argument("--timeline", action="store_true",
+                    help="print one layer's kernel schedule inside the replayed decode step instead of a benchmark line "
+                         "(needs TPI_TIMELINE=1, which selects the library built with time stamps)")
     args = ap.parse_args()
     shape = S.CONFIGS[args.workload]
     if args.layers:
@@ -664,6 +719,8 @@ def main():
         shape = shape.with_(n_shards=args.shards)
     if args.impl == "reference":
         run_reference(args, shape)
+    elif args.timeline:
+        run_timeline(args, shape)
     else:
         run_gpu(args, shape)
 

@@ -102,14 +102,17 @@ def lib() -> C.CDLL:
     """Load libtpi.so (built in-tree by ``paper_2410_00531_b200.build``)."""
     global _LIB
     if _LIB is None:
-        if not os.path.exists(LIB_PATH):   # a fresh checkout: compile it once (nvcc), or fail loudly
+        path = LIB_PATH
+        if os.environ.get("TPI_TIMELINE", "0") not in ("", "0"):   # the instrumented twin (see build.py)
+            path = os.path.join(_HERE, "libtpi_timeline.so")
+        if not os.path.exists(path):   # a fresh checkout: compile it once (nvcc), or fail loudly
             try:
                 from . import build as _build
                 _build.build()
             except Exception as e:
-                raise ImportError(f"{LIB_PATH} is missing and could not be built ({e}): run "
+                raise ImportError(f"{path} is missing and could not be built ({e}): run "
                                   "`python -m paper_2410_00531_b200.build` (this package has no CPU fallback)") from e
-        L = C.CDLL(LIB_PATH)
+        L = C.CDLL(path)
         for name, (res, args) in SYMBOLS.items():
             fn = getattr(L, name)
             fn.restype, fn.argtypes = res, args

@@ -13,6 +13,9 @@
 #include "launch.cuh"
 
 namespace tpi {
+#ifdef TPI_TIMELINE
+void set_timeline_attn(void* dev_buf) { cudaMemcpyToSymbol(g_tl, &dev_buf, sizeof dev_buf); }
+#endif
 
 namespace {
 
@@ -277,6 +280,7 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int kvh = blockIdx.x, split = blockIdx.y;
+  if (threadIdx.x == 0) TL(TL_ID_ATTN, blockIdx.x + gridDim.x * blockIdx.y, TL_ENTRY);
   // The position counter was advanced by the previous token's task head, and the embedding kernel that opens a step
   // lets no later kernel of the step start before that head has completed; only the cache row of the newest position
   // (and the queries) come from the kernel just before this one.  Read through L2: the line may sit stale in this
@@ -320,6 +324,7 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
   if (early0) issue_half(0);
   if (early0 && early1) issue_half(1);
   pdl_wait();
+  if (threadIdx.x == 0) TL(TL_ID_ATTN, blockIdx.x + gridDim.x * blockIdx.y, TL_WAIT);
   if (!early0) issue_half(0);
   if (!(early0 && early1)) issue_half(1);
 
@@ -451,16 +456,20 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
       if (dd == 0) { part[hh * (D + 2)] = M; part[hh * (D + 2) + 1] = L; }
     }
   }
+  if (threadIdx.x == 0) TL(TL_ID_ATTN, blockIdx.x + gridDim.x * blockIdx.y, TL_WARP0);
   if (nact == 1) return;
-  __threadfence();
+  // One thread publishes the CTA's partial results (the barrier orders every thread's stores before its fence, the
+  // fence before the ticket) and, in the CTA that arrives last, fences again before the barrier that lets the other
+  // threads read the other splits' results through L2: one fence per CTA on either side instead of one per thread.
   __syncthreads();
   if (threadIdx.x == 0) {
+    __threadfence();
     const unsigned tk = atomicAdd(tickets + kvh, 1u);
     s_last = (tk == (unsigned)nact - 1);
+    __threadfence();
   }
   __syncthreads();
   if (!s_last) return;
-  __threadfence();
   const float* pg = scratch + (size_t)kvh * nsplit * grp * (D + 2);
   constexpr int MAXN = 24, EPT = 2;  // register path: up to MAXN splits, up to EPT outputs per thread
   if (nact <= MAXN && grp * D <= EPT * DW * 32) {
@@ -499,6 +508,7 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
       }
     }
     if (threadIdx.x == 0) tickets[kvh] = 0u;
+    if (threadIdx.x == 0) TL(TL_ID_ATTN, blockIdx.x + gridDim.x * blockIdx.y, TL_WARP0 + 1);  // merge done
     return;
   }
   // All partial results of this kv head come into shared memory in one batch of independent loads (one trip to L2
@@ -539,6 +549,7 @@ __global__ void __launch_bounds__(DW * 32) decode_attn_mma_kernel(const float* _
     o_out[(size_t)(kvh * grp + hh) * D + dd] = A;
   }
   if (threadIdx.x == 0) tickets[kvh] = 0u;
+  if (threadIdx.x == 0) TL(TL_ID_ATTN, blockIdx.x + gridDim.x * blockIdx.y, TL_WARP0 + 1);  // merge done
 }
 
 template <int D>

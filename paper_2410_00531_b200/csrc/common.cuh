@@ -8,6 +8,32 @@
 
 namespace tpi {
 
+// Device-side timeline of the decode kernels (builds with -DTPI_TIMELINE only; compiled out otherwise): a CTA stamps
+// the global nanosecond timer when it starts, when its dependency wait returns, when its inputs are staged and when
+// each of its warps ends, into a caller-provided buffer [TL_KERNELS][TL_CTAS][TL_SLOTS] of 64-bit words.  Each launch
+// of a kernel overwrites the stamps of the launch before, so after a run the buffer holds the LAST layer's kernels:
+// one layer's schedule under graph replay with programmatic dependent launch, gaps between kernels included.
+#ifdef TPI_TIMELINE
+static __device__ unsigned long long* g_tl;  // one copy per translation unit, all set by set_timeline_*()
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define TL(id, cta, slot)                                                                              \
+  do {                                                                                                 \
+    if (g_tl && (cta) < TL_CTAS) {                                                                     \
+      g_tl[((id) * TL_CTAS + (cta)) * TL_SLOTS + (slot)] = global_ns();                                \
+      if ((slot) == TL_ENTRY) {  /* which SM runs this CTA (slow SMs show up as late CTAs) */          \
+        unsigned sm_;                                                                                  \
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_));                                               \
+        g_tl[((id) * TL_CTAS + (cta)) * TL_SLOTS + TL_SMID] = sm_ + 1;                                 \
+      }                                                                                                \
+    }                                                                                                  \
+  } while (0)
+#else
+#define TL(id, cta, slot) do {} while (0)
+#endif
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");

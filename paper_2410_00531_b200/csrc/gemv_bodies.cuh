@@ -112,6 +112,7 @@ __device__ __forceinline__ void cols_body(const GemvArgs& A, float* xs, const in
   const long long total = (long long)A.items_per_shard * A.n_shards;
   const int lo = (int)(total * cta / ncta), hi = (int)(total * (cta + 1) / ncta);
   const uint32_t row_bytes = (uint32_t)(A.K * sizeof(WT));
+  if (threadIdx.x == 0) TL(EPI, cta, TL_ENTRY);
 
   auto row_ptrs = [&](int it, int& shard, int& item, const uint4* (&wp)[R]) {
     shard = it / A.items_per_shard;
@@ -147,6 +148,7 @@ __device__ __forceinline__ void cols_body(const GemvArgs& A, float* xs, const in
     if (k < A.K) gr[j] = A.gain ? *reinterpret_cast<const float4*>(A.gain + k) : make_float4(1.f, 1.f, 1.f, 1.f);
   }
   pdl_wait();  // x (and its norm statistics) come from the previous kernel
+  if (threadIdx.x == 0) TL(EPI, cta, TL_WAIT);
 
   // ---- prologue: one round trip to L2 for the statistics and x
   float ss = 0.f;
@@ -182,6 +184,7 @@ __device__ __forceinline__ void cols_body(const GemvArgs& A, float* xs, const in
     *reinterpret_cast<float4*>(xs + k) = v;
   }
   __syncthreads();
+  if (threadIdx.x == 0) TL(EPI, cta, TL_STAGED);
 
   // ---- main loop over this CTA's row pairs
   const int nvec = A.K / Elem<WT>::VEC;
@@ -246,6 +249,7 @@ __device__ __forceinline__ void cols_body(const GemvArgs& A, float* xs, const in
       }
     }
   }
+  if (lane == 0) TL(EPI, cta, TL_WARP0 + warp);
   if constexpr (EPI == EPI_LOGITS) {
     __shared__ float s_val[WARPS > 0 ? WARPS : 32];
     __shared__ int s_idx[WARPS > 0 ? WARPS : 32];
@@ -318,6 +322,8 @@ __device__ __forceinline__ void rowfused_body(const RowFusedArgs& A, float* xs, 
   const int lo = (int)((long long)groups * cta / ncta);
   const int hi = (int)((long long)groups * (cta + 1) / ncta);
   const WT* Wall = reinterpret_cast<const WT*>(A.W);
+  [[maybe_unused]] const int tlid = (A.Ks * A.n_shards == A.rows) ? TL_ID_O : TL_ID_DOWN;  // timeline id (square: O)
+  if (threadIdx.x == 0) TL(tlid, cta, TL_ENTRY);
   if (lo + warp < hi && !A.unequal) {
     const uint32_t pf = min((uint32_t)(R * A.Ks * sizeof(WT)), (uint32_t)A.prefetch_bytes) & ~15u;
     for (int sh = lane; sh < A.n_shards; sh += 32)
@@ -325,11 +331,13 @@ __device__ __forceinline__ void rowfused_body(const RowFusedArgs& A, float* xs, 
   }
   pdl_launch_dependents();
   pdl_wait();
+  if (threadIdx.x == 0) TL(tlid, cta, TL_WAIT);
 
   const int ktot = A.unequal ? A.k0[A.n_shards] : A.n_shards * A.Ks;
   for (int k = threadIdx.x * 4; k < ktot; k += nw * 32 * 4)
     *reinterpret_cast<float4*>(xs + k) = *reinterpret_cast<const float4*>(A.x_in + k);
   __syncthreads();
+  if (threadIdx.x == 0) TL(tlid, cta, TL_STAGED);
 
   constexpr int VEC = Elem<WT>::VEC;
   const int nvec = A.Ks / VEC;
@@ -408,6 +416,7 @@ __device__ __forceinline__ void rowfused_body(const RowFusedArgs& A, float* xs, 
       }
     }
   }
+  if (lane == 0) TL(tlid, cta, TL_WARP0 + warp);
   if (lane == 0) s_sq[warp] = sq;
   __syncthreads();
   if (threadIdx.x == 0) {

@@ -183,6 +183,17 @@ cudaError_t launch_reduce_residual_norm_rows(const LaunchCtx& c, const float* pa
 cudaError_t launch_rmsnorm_stat_row(const LaunchCtx& c, const float* xrow, int h, float eps, float* x,
                                     float* xhat, float* ss_part, int n_parts, int* pos, int pos_value);
 
+// Timeline buffer layout (see common.cuh): kernel ids 0 QKV, 1 gate/up, 3 task head (the column-sharded GEMVs' epilogue
+// ids), 4 O projection, 5 down projection, 6 decode attention; slots TL_ENTRY, TL_WAIT (dependency wait returned),
+// TL_STAGED (inputs in shared memory), TL_SMID (1 + the SM the CTA ran on), then one per warp from TL_WARP0 (the
+// warp's last row is done).
+enum { TL_KERNELS = 7, TL_CTAS = 160, TL_SLOTS = 40, TL_ENTRY = 0, TL_WAIT = 1, TL_STAGED = 2, TL_SMID = 3, TL_WARP0 = 4,
+       TL_ID_O = 4, TL_ID_DOWN = 5, TL_ID_ATTN = 6 };
+#ifdef TPI_TIMELINE
+void set_timeline_decode(void* dev_buf);
+void set_timeline_attn(void* dev_buf);
+#endif
+
 // tuning knobs (0: CTAs per SM of the column-sharded GEMVs, 1: of the fused row-sharded GEMVs,
 // 2: L2 prefetch bytes per row before the dependency wait)
 void set_tuning(int key, int value);

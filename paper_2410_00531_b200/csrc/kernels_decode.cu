@@ -12,6 +12,9 @@
 #include "launch.cuh"
 
 namespace tpi {
+#ifdef TPI_TIMELINE
+void set_timeline_decode(void* dev_buf) { cudaMemcpyToSymbol(g_tl, &dev_buf, sizeof dev_buf); }
+#endif
 
 // =====================================================================================
 // GEMV family
@@ -691,16 +694,18 @@ __global__ void __launch_bounds__(256) decode_attn_kernel(const float* __restric
     part[hh * (D + 2) + 2 + dd] = A;
     if (dd == 0) { part[hh * (D + 2)] = M; part[hh * (D + 2) + 1] = L; }
   }
-  // ---- the last CTA of this kv head to arrive merges the splits in split order
-  __threadfence();
+  // ---- the last CTA of this kv head to arrive merges the splits in split order (one thread fences for the CTA:
+  // the barrier orders every thread's stores before its fence, and its second fence precedes the barrier after which
+  // the last CTA reads the other splits' results through L2)
   __syncthreads();
   if (threadIdx.x == 0) {
+    __threadfence();
     const unsigned t = atomicAdd(tickets + g, 1u);
     s_last = (t == (unsigned)nsplit - 1);
+    __threadfence();
   }
   __syncthreads();
   if (!s_last) return;
-  __threadfence();
   const int nact = (n + chunk - 1) / chunk;  // splits that saw at least one position
   const float* pg = scratch + (size_t)g * nsplit * GRP * (D + 2);
   // weights of the splits first (one exp2 per head and split, kept in shared memory; the row-group

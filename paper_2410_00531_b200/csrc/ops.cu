@@ -162,5 +162,20 @@ extern "C" int tpi_op_prefill_attention(int dtype, const float* Q, const void* k
   return e == cudaErrorInvalidValue ? TPI_ERR_SHAPE : cu(e);
 }
 
+// Internal hook (not part of the public interface): hands the decode kernels a device buffer of
+// layout[0] * layout[1] * layout[2] 64-bit words for their timeline stamps (NULL switches it off again).
+// Returns 1, or 0 when the library was built without -DTPI_TIMELINE (the kernels then carry no stamps).
+extern "C" int tpi_internal_timeline(void* dev_buf, int* layout) {
+  if (layout) { layout[0] = TL_KERNELS; layout[1] = TL_CTAS; layout[2] = TL_SLOTS; layout[3] = TL_WARP0; }
+#ifdef TPI_TIMELINE
+  set_timeline_decode(dev_buf);
+  set_timeline_attn(dev_buf);
+  return 1;
+#else
+  (void)dev_buf;
+  return 0;
+#endif
+}
+
 // Internal tuning hook (not part of the public interface): see kernels.h set_tuning.
 extern "C" void tpi_internal_tune(int key, int value) { set_tuning(key, value); }
