@@ -213,7 +213,7 @@ static bool gemm_pair_enabled() {
 static cudaError_t launch_gemm_tc_any(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
                                       const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T,
                                       int n_out, int K, int n_batch, int* err, void* act, int act_ld, long long act_lo_off,
-                                      int act_split, int wait_polls = 0, int starve = 0) {
+                                      int act_split, int wait_polls = 0, int starve = 0, bool chunk_k = false) {
   // Tile width: one CTA computes 128 positions x BN outputs and, per 64-wide k-block, pulls the activation tile(s)
   // plus BN weight rows through shared memory; a CTA's ingest rate is what bounds it, so the cost of a choice is
   // (waves of CTAs over the SMs) x (bytes per k-block), and widths that leave SMs idle or spill into another wave lose.
@@ -236,6 +236,10 @@ static cudaError_t launch_gemm_tc_any(const LaunchCtx& c, const void* A_bf16, co
                                  : (double)waves * ((K / kBK) * tile_us[i] + 4.0 + bn / 64.0);
     if (cost < best - 1e-9) { best = cost; BN = bn; best_us = cost; }
   }
+  // long contractions of the column-sharded projections: chunks of the contraction, added in registers
+  if (chunk_k && A_lo_bf16 && n_batch == 1 && a_col_batch == 0 && gemm_pair_enabled() && !starve &&
+      gemm_tc_chunked_supported(T, K, lda, n_out, ldy, act != nullptr))
+    return launch_gemm_tc_chunked(c, A_bf16, A_lo_bf16, lda, W_bf16, Y, ldy, T, n_out, K, err, act, act_ld, act_lo_off, act_split);
   if (A_lo_bf16 && T > kBM && gemm_pair_enabled() && !starve) {  // a CTA pair (M = 256) pulls half the weight bytes per MMA
     double pair_us = 0;
     const int shape = gemm_tc_pair_choose(T, n_out, K, n_batch, nsm, &pair_us);
@@ -265,9 +269,9 @@ static cudaError_t launch_gemm_tc_any(const LaunchCtx& c, const void* A_bf16, co
 
 cudaError_t launch_gemm_tc(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
                            const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T,
-                           int n_out, int K, int n_batch, int* err) {
+                           int n_out, int K, int n_batch, int* err, bool chunk_k) {
   return launch_gemm_tc_any(c, A_bf16, A_lo_bf16, lda, a_col_batch, W_bf16, w_row_batch, Y, y_batch_stride, ldy, T, n_out, K,
-                            n_batch, err, nullptr, 0, 0, 0);
+                            n_batch, err, nullptr, 0, 0, 0, 0, 0, chunk_k);
 }
 
 cudaError_t launch_gemm_tc_starved(const LaunchCtx& c, const void* A_bf16, int lda, const void* W_bf16, float* Y, int ldy, int T,
@@ -282,7 +286,7 @@ cudaError_t launch_gemm_tc_swiglu(const LaunchCtx& c, const void* A_bf16, const 
                                   void* ACT, int out_mode, int T, int s, int K, int* err) {
   if (out_mode != 1 && out_mode != 2) return cudaErrorInvalidValue;
   return launch_gemm_tc_any(c, A_bf16, A_lo_bf16, lda, 0, Wgu_bf16, 2 * s, nullptr, 0, 2 * s, T, 2 * s, K, 1, err, ACT, s,
-                            (long long)T * s, out_mode == 2);
+                            (long long)T * s, out_mode == 2, 0, 0, true);
 }
 
 }  // namespace tpi

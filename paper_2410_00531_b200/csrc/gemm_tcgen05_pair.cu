@@ -229,16 +229,35 @@ __global__ void __launch_bounds__(192) gemm_tc_pair_kernel(const __grid_constant
 // memory (two accumulator buffers, so shard i+1 multiplies while shard i is read back); 8 epilogue warps per CTA
 // keep the running sum ((P_0 + P_1) + ...) in registers (one row and 128 columns per thread), add the shortcut X
 // last and write the new residual stream over X.  The partial sums never reach memory.
+//
+//
+// The same kernel runs the COLUMN-sharded projections (QKV, gate/up; modes 1: plain store, 2: SwiGLU) with their
+// contraction over the whole hidden state cut into CHUNKS of 512 inputs that take the place of the shards: each chunk
+// is formed in tensor memory by itself and added to the running sum in registers.  The reason is the tensor core's
+// accumulator: every tcgen05.mma step adds 16 products to the fp32 value in tensor memory and TRUNCATES the result,
+// so a chain of K / 16 steps (twice that with the hi + lo activations) drifts towards zero by about 2^-26 of the sum
+// per step: measured 9e-6 of the output's norm at K = 4096 and 1.9e-5 at K = 8192, against 2.4e-6 for the hi + lo
+// split itself.  In chunks of 512 inputs, added in registers with round to nearest, the chain is 64 steps long
+// whatever K is (1.1e-6).  On the 70B shape at full depth this halves the distance to the fp64 oracle (logits 2.0e-2
+// -> 0.9e-2; with fp32 SIMT GEMMs throughout it is 0.6e-2).  A shard's contraction (512 to 3584 inputs) stays one
+// chain: cutting it as well changed nothing measurable at full depth, and the partial sum P_i of a shard keeps the
+// bits a real rank computes for it.
 constexpr int RS_BN = 256, RS_THREADS = 320;
 constexpr uint32_t RS_A_BYTES = kMH * kBK * 2, RS_B_BYTES = (RS_BN / 2) * kBK * 2, RS_STAGE = 2 * RS_A_BYTES + RS_B_BYTES;
 constexpr int RS_STAGES = (226 * 1024 - 1024) / RS_STAGE;
 
 struct RowSumArgs {
-  float* X;  // [T][ldx] fp32, residual in, new residual out
-  int ldx, T, n_out, K, n_shards;
+  float* X;  // [T][ldx] fp32: mode 0 residual in, new residual out; mode 1 output
+  int ldx, T, n_out, K, n_shards;  // K: contraction length of one shard
   int a_col_batch;  // A's column offset per shard (elements)
   int w_row_batch;  // W's row offset per shard
   int* err;
+  int chunks;       // chunks per shard; chunk c of a shard covers its k-blocks [c * kb_chunk, min((c + 1) * kb_chunk, K / 64))
+  int kb_chunk;     // 64-wide k-blocks per chunk
+  int mode;         // 0: X <- sum + X (star sum + shortcut); 1: X <- sum; 2: act <- SwiGLU(sum) as bf16 hi (+ lo)
+  __nv_bfloat16* act;
+  long long act_lo_off;
+  int act_ld, act_split;
 };
 
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
@@ -291,7 +310,7 @@ __global__ void __launch_bounds__(RS_THREADS) gemm_tc_pair_rowsum_kernel(const _
       int it = 0;
       bool ok = true;
       for (int sh = 0; sh < a.n_shards && ok; ++sh)
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {  // the loader does not care where a chunk ends
           const int s = it % RS_STAGES;
           const uint32_t ph = (it / RS_STAGES) & 1;
           if (!mbar_wait(&empty[s], ph ^ 1, a.err)) { ok = false; break; }
@@ -305,18 +324,20 @@ __global__ void __launch_bounds__(RS_THREADS) gemm_tc_pair_rowsum_kernel(const _
         }
     }
   } else if (warp == 1) {
-    if (lane == 0 && rank == 0) {  // ---- the leader issues the pair's MMAs; shard sh accumulates in buffer sh & 1
+    if (lane == 0 && rank == 0) {  // ---- the leader issues the pair's MMAs; chunk g (counted over all shards) accumulates in buffer g & 1
       constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(RS_BN >> 3) << 17) | ((uint32_t)((2 * kMH) >> 4) << 24);
       const uint32_t empty0_peer = map_to_cta(smem_u32(&empty[0]), 1);
       int it = 0;
       bool ok = true;
-      for (int sh = 0; sh < a.n_shards && ok; ++sh) {
-        const int bi = sh & 1;
-        ok = mbar_wait(&acc_free[bi], ((sh >> 1) & 1) ^ 1, a.err);  // both CTAs have read this buffer's previous shard back
+      const int n_seg = a.n_shards * a.chunks;
+      for (int g = 0; g < n_seg && ok; ++g) {
+        const int bi = g & 1;
+        ok = mbar_wait(&acc_free[bi], ((g >> 1) & 1) ^ 1, a.err);  // both CTAs have read this buffer's previous chunk back
         if (!ok) break;
         tc_fence_after();
         const uint32_t d = tmem_acc + (uint32_t)bi * RS_BN;
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        const int kb0 = (g % a.chunks) * a.kb_chunk, kb1 = min(kb0 + a.kb_chunk, kblocks);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % RS_STAGES;
           const uint32_t ph = (it / RS_STAGES) & 1;
           ok = mbar_wait(&full[s], ph, a.err);
@@ -325,7 +346,7 @@ __global__ void __launch_bounds__(RS_THREADS) gemm_tc_pair_rowsum_kernel(const _
           const uint32_t sa = smem_u32(smem + (size_t)s * RS_STAGE);
           const uint64_t dh = umma_desc_sw128(sa), dl = umma_desc_sw128(sa + RS_A_BYTES), db = umma_desc_sw128(sa + 2 * RS_A_BYTES);
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k) umma2_bf16(d, dh + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
+          for (int k = 0; k < kBK / 16; ++k) umma2_bf16(d, dh + 2 * k, db + 2 * k, idesc, (kb > kb0 || k) ? 1u : 0u);
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k) umma2_bf16(d, dl + 2 * k, db + 2 * k, idesc, 1u);
           umma2_commit(smem_u32(&empty[s]));
@@ -341,7 +362,8 @@ __global__ void __launch_bounds__(RS_THREADS) gemm_tc_pair_rowsum_kernel(const _
     const uint32_t free0 = map_to_cta(smem_u32(&acc_free[0]), 0);
     float sum[128];
     bool ok = true;
-    for (int sh = 0; sh < a.n_shards && ok; ++sh) {
+    const int n_seg = a.n_shards * a.chunks;
+    for (int sh = 0; sh < n_seg && ok; ++sh) {  // sh counts chunks over all shards
       const int bi = sh & 1;
       ok = mbar_wait(&acc_ready[bi], (sh >> 1) & 1, a.err);
       if (!ok) break;
@@ -358,19 +380,44 @@ __global__ void __launch_bounds__(RS_THREADS) gemm_tc_pair_rowsum_kernel(const _
       if (lane == 0) mbar_arrive_cluster(free0 + (uint32_t)bi * 8);  // on the leader's barrier: its MMA thread reuses the buffer
     }
     const int row = m0 + q * 32 + lane;
-    if (ok && row < a.T && a.n_shards > 0 && kblocks > 0) {
+    if (ok && row < a.T && a.n_shards > 0 && kblocks > 0 && a.mode == 2) {
+      // SwiGLU on the (gate, up) column pairs: 16 columns -> 8 activations -> one 16-byte store of the high halves
+      // (and one of the low halves); n_out is a multiple of 32 here, so a group of 16 columns is whole or absent
+      __nv_bfloat16* arow = a.act + (size_t)row * a.act_ld + ((n0 + hs * 128) >> 1);
+#pragma unroll
+      for (int c = 0; c < 128; c += 16) {
+        if (n0 + hs * 128 + c + 16 > a.n_out) break;
+        uint32_t hi[4], lo[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          float v[2];
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const float g = sum[c + 4 * j + 2 * e], u = sum[c + 4 * j + 2 * e + 1];
+            v[e] = g / (1.f + expf(-g)) * u;
+          }
+          const __nv_bfloat16 h0 = __float2bfloat16_rn(v[0]), h1 = __float2bfloat16_rn(v[1]);
+          hi[j] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+          const __nv_bfloat16 l0 = __float2bfloat16_rn(v[0] - __bfloat162float(h0)), l1 = __float2bfloat16_rn(v[1] - __bfloat162float(h1));
+          lo[j] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+        }
+        *reinterpret_cast<uint4*>(arow + (c >> 1)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        if (a.act_split) *reinterpret_cast<uint4*>(arow + a.act_lo_off + (c >> 1)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      }
+    } else if (ok && row < a.T && a.n_shards > 0 && kblocks > 0) {
       // column hs*128 + c of the CTA's tile is weight row n0 + hs * 128 + c (the leader's half first)
       float* x = a.X + (size_t)row * a.ldx + n0 + hs * 128;
+      const bool add = a.mode == 0;  // the shortcut comes after the star sum; the column-sharded projections have none
 #pragma unroll
       for (int c = 0; c < 128; c += 4) {
         const int col = n0 + hs * 128 + c;
         if (col + 4 <= a.n_out) {
-          const float4 v = *reinterpret_cast<const float4*>(x + c);
+          const float4 v = add ? *reinterpret_cast<const float4*>(x + c) : make_float4(0.f, 0.f, 0.f, 0.f);
           *reinterpret_cast<float4*>(x + c) = make_float4(sum[c] + v.x, sum[c + 1] + v.y, sum[c + 2] + v.z, sum[c + 3] + v.w);
         } else {
 #pragma unroll
           for (int e = 0; e < 4; ++e)
-            if (col + e < a.n_out) x[c + e] = sum[c + e] + x[c + e];
+            if (col + e < a.n_out) x[c + e] = add ? sum[c + e] + x[c + e] : sum[c + e];
         }
       }
     }
@@ -469,15 +516,60 @@ bool gemm_tc_rowsum_supported(int T, int K, int a_cols_total, int n_out, int ldx
   return !(e && e[0] == '0') && T > kMH && K > 0 && K % kBK == 0 && a_cols_total % 8 == 0 && ldx % 4 == 0 && n_out % 4 == 0;
 }
 
+static cudaError_t launch_rowsum_args(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, const void* W_bf16,
+                                      uint64_t w_cols, uint64_t w_rows, const RowSumArgs& a);
+
+int gemm_tc_chunk_len() {
+  static int len = -1;
+  if (len < 0) {
+    const char* e = getenv("TPI_GEMM_CHUNK");  // development aid: 0 = one accumulation chain per contraction, else the longest chunk
+    len = e ? atoi(e) : 512;
+    if (len < 0 || len % kBK) len = 512;
+  }
+  return len;
+}
+// chunks of a contraction of K inputs: as few as keep every chunk within the limit, of equal length up to one k-block
+static void chunking(int K, int* chunks, int* kb_chunk) {
+  const int len = gemm_tc_chunk_len(), kblocks = K / kBK;
+  const int n = len > 0 ? (K + len - 1) / len : 1;
+  *chunks = n < 1 ? 1 : n;
+  *kb_chunk = (kblocks + *chunks - 1) / *chunks;
+  if (*kb_chunk < 1) *kb_chunk = 1;
+  *chunks = (kblocks + *kb_chunk - 1) / *kb_chunk;
+  if (*chunks < 1) *chunks = 1;
+}
+
 cudaError_t launch_gemm_tc_rowsum(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
                                   const void* W_bf16, int w_row_batch, float* X, int ldx, int T, int n_out, int K, int n_shards,
                                   int* err) {
   if (!A_lo_bf16 || n_shards < 1) return cudaErrorInvalidValue;
+  RowSumArgs a{X, ldx, T, n_out, K, n_shards, a_col_batch, w_row_batch, err, 1, K / kBK, 0, nullptr, 0, 0, 0};  // one chain per shard
+  return launch_rowsum_args(c, A_bf16, A_lo_bf16, lda, W_bf16, (uint64_t)K, (uint64_t)(n_shards - 1) * w_row_batch + n_out, a);
+}
+
+// Column-sharded projection (one matrix, no shortcut): Y[t][o] = sum over the chunks of the contraction.
+// act != nullptr: SwiGLU epilogue as in launch_gemm_tc_swiglu (act_ld, act_lo_off, act_split), nothing is written to Y.
+bool gemm_tc_chunked_supported(int T, int K, int lda, int n_out, int ldy, bool swiglu) {
+  const int len = gemm_tc_chunk_len();
+  return len > 0 && T > kMH && K > len && K % kBK == 0 && lda % 8 == 0 && n_out % 4 == 0 && (swiglu ? n_out % 32 == 0 : ldy % 4 == 0);
+}
+cudaError_t launch_gemm_tc_chunked(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, const void* W_bf16, float* Y,
+                                   int ldy, int T, int n_out, int K, int* err, void* act, int act_ld, long long act_lo_off,
+                                   int act_split) {
+  if (!A_lo_bf16) return cudaErrorInvalidValue;
+  int chunks, kb_chunk;
+  chunking(K, &chunks, &kb_chunk);
+  RowSumArgs a{Y, ldy, T, n_out, K, 1, 0, 0, err, chunks, kb_chunk, act ? 2 : 1, (__nv_bfloat16*)act, act_lo_off, act_ld, act_split};
+  return launch_rowsum_args(c, A_bf16, A_lo_bf16, lda, W_bf16, (uint64_t)K, (uint64_t)n_out, a);
+}
+
+static cudaError_t launch_rowsum_args(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, const void* W_bf16,
+                                      uint64_t w_cols, uint64_t w_rows, const RowSumArgs& a) {
+  const int T = a.T, n_out = a.n_out;
   CUtensorMap tmA, tmAlo, tmW;
-  const uint64_t w_rows = (uint64_t)(n_shards - 1) * w_row_batch + n_out;
   if (!make_map(&tmA, A_bf16, (uint64_t)lda, (uint64_t)T, (uint64_t)lda, kMH)) return cudaErrorInvalidValue;
   if (!make_map(&tmAlo, A_lo_bf16, (uint64_t)lda, (uint64_t)T, (uint64_t)lda, kMH)) return cudaErrorInvalidValue;
-  if (!make_map(&tmW, W_bf16, (uint64_t)K, w_rows, (uint64_t)K, RS_BN / 2)) return cudaErrorInvalidValue;
+  if (!make_map(&tmW, W_bf16, w_cols, w_rows, w_cols, RS_BN / 2)) return cudaErrorInvalidValue;
   auto kern = gemm_tc_pair_rowsum_kernel;
   const size_t smem = (size_t)RS_STAGES * RS_STAGE + 1024;
   static PerDeviceOnce attr_done;
@@ -487,7 +579,6 @@ cudaError_t launch_gemm_tc_rowsum(const LaunchCtx& c, const void* A_bf16, const 
     attr_done.set();
   }
   if (c.launches) ++*c.launches;
-  RowSumArgs a{X, ldx, T, n_out, K, n_shards, a_col_batch, w_row_batch, err};
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(2 * ((T + 2 * kMH - 1) / (2 * kMH)), (n_out + RS_BN - 1) / RS_BN, 1);
   cfg.blockDim = dim3(RS_THREADS);

@@ -126,7 +126,9 @@ bool gemm_tc_supported(int K, int a_cols_total, int ldy);
 // A_lo_bf16 (may be null): second bf16 tensor of the same shape with A = A_bf16 + A_lo_bf16 (split activations).
 cudaError_t launch_gemm_tc(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
                            const void* W_bf16, int w_row_batch, float* Y, long long y_batch_stride, int ldy, int T,
-                           int n_out, int K, int n_batch, int* err);
+                           int n_out, int K, int n_batch, int* err, bool chunk_k = false);
+// (chunk_k: a single-batch contraction over more than 128 positions is accumulated in chunks, see
+// launch_gemm_tc_chunked; the column-sharded projections ask for it, the per-shard partial sums do not)
 // Gate/up projection with the SwiGLU of launch_swiglu_rows applied in the epilogue (same arithmetic, same bits):
 // Wgu rows interleaved gate_j, up_j; ACT [T][s] bf16 (out_mode 1) or split bf16 (2: lo at + T*s elements).
 // CTA-pair tiles (tcgen05.mma.cta_group::2) for the same contract, split activations only.  gemm_tc_pair_choose returns
@@ -139,6 +141,12 @@ cudaError_t launch_gemm_tc_pair(const LaunchCtx& c, int shape, const void* A_bf1
 // Row-sharded projection of T > 128 positions with the star sum in its epilogue: X[t][o] = ((P_0 + P_1) + ... ) + X[t][o],
 // P_i[t][o] = sum_k (A_hi + A_lo)[t][i*a_col_batch + k] * W[i*w_row_batch + o][k]; the partial sums stay on chip.
 bool gemm_tc_rowsum_supported(int T, int K, int a_cols_total, int n_out, int ldx);
+// The same pair kernel for the column-sharded projections, the contraction cut into chunks whose partial sums are added
+// in registers (the tensor core truncates its fp32 accumulator at every step; short chains keep that drift small).
+bool gemm_tc_chunked_supported(int T, int K, int lda, int n_out, int ldy, bool swiglu);
+cudaError_t launch_gemm_tc_chunked(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, const void* W_bf16, float* Y,
+                                   int ldy, int T, int n_out, int K, int* err, void* act, int act_ld, long long act_lo_off,
+                                   int act_split);
 cudaError_t launch_gemm_tc_rowsum(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, int a_col_batch,
                                   const void* W_bf16, int w_row_batch, float* X, int ldx, int T, int n_out, int K, int n_shards,
                                   int* err);

@@ -115,7 +115,7 @@ extern "C" int tpi_op_gemm_bf16(const void* A, const void* A_lo, int lda, int a_
   if (!A || !W || !Y || !err_word || T < 1 || n_out < 1 || K < 1 || n_batch < 1) return TPI_ERR_INVALID_ARG;
   if (!gemm_tc_supported(K, lda, ldy) || a_col_batch % 8) return TPI_ERR_SHAPE;
   const cudaError_t e = launch_gemm_tc(ctx(stream), A, A_lo, lda, a_col_batch, W, w_row_batch, Y, y_bs, ldy, T, n_out, K,
-                                       n_batch, err_word);
+                                       n_batch, err_word, true);
   return e == cudaErrorInvalidValue ? TPI_ERR_SHAPE : cu(e);
 }
 

@@ -32,11 +32,11 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
   int* err = dptr<int>(m, p.err);
   // Y[b] = A[:, b*a_col : b*a_col+K] . W[b]^T for n_batch shards (1 for the column-sharded projections)
   auto proj = [&](const float* A, int lda, int a_col, const void* W, int w_rows_b, float* Y, long long y_bs, int ldy,
-                  int n_out, int K, int n_batch) -> int {
+                  int n_out, int K, int n_batch, bool chunk_k = false) -> int {
     if (tc) {  // split mode: the low halves sit T * lda bf16 elements after the high halves
       const __nv_bfloat16* hi = reinterpret_cast<const __nv_bfloat16*>(A);
       CK(launch_gemm_tc(lc, hi, act_mode == 2 ? hi + (size_t)T * lda : nullptr, lda, a_col, W, w_rows_b, Y, y_bs, ldy, T,
-                        n_out, K, n_batch, err));
+                        n_out, K, n_batch, err, chunk_k));
     }
     else CK(launch_gemm_simt(lc, dt, A, a_col, lda, W, (long long)w_rows_b * K, Y, y_bs, ldy, T, n_out, K, n_batch));
     return TPI_OK;
@@ -88,7 +88,7 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
     void* kc = m->dev + p.kcache + (size_t)l * p.kv_layer_bytes;
     void* vc = m->dev + p.vcache + (size_t)l * p.kv_layer_bytes;
     if (!normed) CK(launch_rmsnorm_rows(lc, X, (const float*)br.base, T, h, c.rms_eps, Xn, act_mode));
-    TRY(proj(Xn, h, 0, br.base + bl.off_qkv, qkv_cols, QKV, 0, qkv_cols, qkv_cols, h, 1));
+    TRY(proj(Xn, h, 0, br.base + bl.off_qkv, qkv_cols, QKV, 0, qkv_cols, qkv_cols, h, 1, true));
     CK(launch_rope_kv_rows(lc, dt, QKV, T, pos0, Nc, a, b, d, c.max_seq, rope, Q, kc, vc));
     if (m->opt_tensor && prefill_attention_tc_supported(dt, d, T))
       CK(launch_prefill_attention_tc(lc, Q, kc, vc, T, pos0, a, b, c.max_seq, O, act_mode, err));
@@ -105,7 +105,7 @@ static int enqueue_prefill_chunk(tpi_model* m, LaunchCtx& lc, int pos0, int T, b
       const __nv_bfloat16* hi = reinterpret_cast<const __nv_bfloat16*>(Xn);
       CK(launch_gemm_tc_swiglu(lc, hi, act_mode == 2 ? hi + (size_t)T * h : nullptr, h, br.base + bl.off_gu, ACT, act_mode, T, s, h, err));
     } else {
-      TRY(proj(Xn, h, 0, br.base + bl.off_gu, 2 * s, GU, 0, 2 * s, 2 * s, h, 1));
+      TRY(proj(Xn, h, 0, br.base + bl.off_gu, 2 * s, GU, 0, 2 * s, 2 * s, h, 1, true));
       CK(launch_swiglu_rows(lc, GU, T, s, ACT, act_mode));
     }
     float* tap_f = last ? dptr<float>(m, p.taps) + (size_t)(2 * l + 1) * h : nullptr;

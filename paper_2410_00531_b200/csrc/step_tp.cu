@@ -296,10 +296,11 @@ int enqueue_prompt_chunk(tpi_tp_group* g, int pos0, int T, bool last, int* launc
   }
   const int act_mode = tc ? 2 : 0;
   const bool fuse_norm = g->window <= 0;  // a streamed rank may not hold the next block's gain yet
-  auto gemm = [&](TpRank& r, LaunchCtx& lc, const float* A, int lda, const void* W, float* Y, int ldy, int n_out, int K) -> int {
+  auto gemm = [&](TpRank& r, LaunchCtx& lc, const float* A, int lda, const void* W, float* Y, int ldy, int n_out, int K,
+                  bool chunk_k = false) -> int {
     if (tc) {
       const __nv_bfloat16* hi = reinterpret_cast<const __nv_bfloat16*>(A);
-      CK(launch_gemm_tc(lc, hi, hi + (size_t)T * lda, lda, 0, W, n_out, Y, 0, ldy, T, n_out, K, 1, dptr<int>(r.m, r.m->plan.err)));
+      CK(launch_gemm_tc(lc, hi, hi + (size_t)T * lda, lda, 0, W, n_out, Y, 0, ldy, T, n_out, K, 1, dptr<int>(r.m, r.m->plan.err), chunk_k));
     } else {
       CK(launch_gemm_simt(lc, dt, A, 0, lda, W, 0, Y, 0, ldy, T, n_out, K, 1));
     }
@@ -359,7 +360,7 @@ int enqueue_prompt_chunk(tpi_tp_group* g, int pos0, int T, bool last, int* launc
           float *QKV = dptr<float>(m, p.pQKV), *Q = dptr<float>(m, p.pQ), *O = dptr<float>(m, p.pO);
           void* kc = m->dev + p.kcache + (size_t)l * p.kv_layer_bytes;
           void* vc = m->dev + p.vcache + (size_t)l * p.kv_layer_bytes;
-          TRY(gemm(r, lc, Xn, h, br.base + bl.off_qkv, QKV, qkv_cols, qkv_cols, h));
+          TRY(gemm(r, lc, Xn, h, br.base + bl.off_qkv, QKV, qkv_cols, qkv_cols, h, true));
           CK(launch_rope_kv_rows(lc, dt, QKV, T, pos0, 1, al, bl_, d, c.max_seq, dptr<float2>(m, p.rope), Q, kc, vc));
           if (m->opt_tensor && prefill_attention_tc_supported(dt, d, T))
             CK(launch_prefill_attention_tc(lc, Q, kc, vc, T, pos0, al, bl_, c.max_seq, O, act_mode, dptr<int>(m, p.err)));
@@ -374,7 +375,7 @@ int enqueue_prompt_chunk(tpi_tp_group* g, int pos0, int T, bool last, int* launc
             const __nv_bfloat16* hi = reinterpret_cast<const __nv_bfloat16*>(Xn);
             CK(launch_gemm_tc_swiglu(lc, hi, hi + (size_t)T * h, h, br.base + bl.off_gu, ACT, act_mode, T, sl, h, dptr<int>(m, p.err)));
           } else {
-            TRY(gemm(r, lc, Xn, h, br.base + bl.off_gu, GU, 2 * sl, 2 * sl, h));
+            TRY(gemm(r, lc, Xn, h, br.base + bl.off_gu, GU, 2 * sl, 2 * sl, h, true));
             CK(launch_swiglu_rows(lc, GU, T, sl, ACT, act_mode));
           }
           TRY(gemm(r, lc, ACT, sl, br.base + bl.off_down, PART, h, h, sl));
