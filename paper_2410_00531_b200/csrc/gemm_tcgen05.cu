@@ -237,7 +237,7 @@ static cudaError_t launch_gemm_tc_any(const LaunchCtx& c, const void* A_bf16, co
     if (cost < best - 1e-9) { best = cost; BN = bn; best_us = cost; }
   }
   // long contractions of the column-sharded projections: chunks of the contraction, added in registers
-  if (chunk_k && A_lo_bf16 && n_batch == 1 && a_col_batch == 0 && gemm_pair_enabled() && !starve &&
+  if (chunk_k && A_lo_bf16 && n_batch == 1 && gemm_pair_enabled() && !starve &&
       gemm_tc_chunked_supported(T, K, lda, n_out, ldy, act != nullptr))
     return launch_gemm_tc_chunked(c, A_bf16, A_lo_bf16, lda, W_bf16, Y, ldy, T, n_out, K, err, act, act_ld, act_lo_off, act_split);
   if (A_lo_bf16 && T > kBM && gemm_pair_enabled() && !starve) {  // a CTA pair (M = 256) pulls half the weight bytes per MMA

@@ -308,7 +308,8 @@ def test_rowshard_fused_is_bit_identical_to_partials_then_sum(T, cfg, n_shards, 
 
 
 @pytest.mark.parametrize("Tn,K,n_out,nb", [(128, 4096, 12288, 1), (100, 4096, 1024, 1), (300, 1024, 4096, 4),
-                                           (128, 2752, 4096, 4), (37, 64, 200, 2), (512, 3584, 640, 8)])
+                                           (128, 2752, 4096, 4), (37, 64, 200, 2), (512, 3584, 640, 8),
+                                           (300, 4160, 1000, 1), (513, 8192, 2048, 1)])
 @pytest.mark.parametrize("split", [False, True])
 def test_gemm_tensor_core_bf16(T, Tn, K, n_out, nb, split):
     """Prompt-pass projection on tcgen05: bf16 inputs, fp32 accumulation, against fp64 on the same
@@ -333,8 +334,10 @@ def test_gemm_tensor_core_bf16(T, Tn, K, n_out, nb, split):
     got = Y.cpu().numpy()
     assert np.isfinite(got).all()
     # products of bf16 pairs are exact in fp32; what is left is the tensor core's fp32 accumulation
-    # over K / 16 (split: K / 8) partial sums, observed <= 1e-5
+    # over K / 16 (split: K / 8) steps, each of which truncates: 9.3e-6 at K = 4096 in one chain
     assert rel_l2(got, want) < 2e-5
+    if split and nb == 1 and Tn > 128 and K > 512:   # accumulated in chunks of 512 inputs (ragged last chunk included)
+        assert rel_l2(got, want) < 3e-6
 
 
 @pytest.mark.parametrize("shape", [0, 1, 2, 3])
@@ -400,7 +403,7 @@ def test_gemm_rowsum_star_sum_in_epilogue(T, Tn, K, n_out, nb):
     assert np.array_equal(Xb.cpu().numpy(), got)
 
 
-@pytest.mark.parametrize("Tn,K,s", [(128, 4096, 11008), (70, 1024, 1360), (300, 512, 48)])
+@pytest.mark.parametrize("Tn,K,s", [(128, 4096, 11008), (70, 1024, 1360), (300, 512, 48), (300, 4160, 496), (513, 8192, 1360)])
 @pytest.mark.parametrize("split_out", [False, True])
 def test_gemm_tensor_core_swiglu_epilogue(T, Tn, K, s, split_out):
     """Eq. 2's gate/up projection for T positions with SwiGLU applied in the GEMM's epilogue (gate_j, up_j rows
