@@ -243,3 +243,25 @@ def test_steady_conditions_match_the_oracle_and_the_worked_example():
     assert P.steady_conditions(11, 17, 14, 18, 30, 32) == P.steady_conditions(25, 31, 0, 18, 30, 32)
     with pytest.raises(P.TpiError):
         P.steady_conditions(-1, 1, 1, 1, 1, 4)
+
+
+def test_timeline_variant_compiles_and_the_plain_library_carries_no_stamps(tmp_path):
+    """The decode kernels' device-side timeline is an opt-in build (-DTPI_TIMELINE, see build.py): the translation units
+    that hold its macro, a stamped kernel, and the hook must compile for sm_100a with the flag, and the plain library's
+    hook must answer 0 ("no stamps here") while still reporting the buffer layout."""
+    import shutil
+    import subprocess
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    if not (os.path.exists(nvcc) or shutil.which("nvcc")):
+        pytest.skip("no nvcc on this machine")
+    csrc = os.path.join(os.path.dirname(P.__file__), "csrc")
+    procs = [subprocess.Popen([nvcc if os.path.exists(nvcc) else "nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-O1",
+                               "-std=c++17", "-Xcompiler", "-fPIC", "-DTPI_TIMELINE", "-c", os.path.join(csrc, src), "-o",
+                               str(tmp_path / (src + ".o"))]) for src in ("attn_prefill_mma.cu", "ops.cu")]
+    assert all(p.wait() == 0 for p in procs)
+    fn = P.lib().tpi_internal_timeline
+    fn.argtypes, fn.restype = [C.c_void_p, C.POINTER(C.c_int)], C.c_int
+    lay = (C.c_int * 4)()
+    if os.environ.get("TPI_TIMELINE", "0") in ("", "0"):
+        assert fn(None, lay) == 0
+    assert lay[0] >= 7 and lay[1] >= 148 and lay[2] >= 4 + 32 and lay[3] == 4
