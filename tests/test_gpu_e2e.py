@@ -82,6 +82,32 @@ def test_chunked_prefill_matches():
     _run_and_compare(shape, 2, prompt_len=23, max_prefill=8, n_decode=3)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_degenerate_prompts(dtype):
+    """The smallest and the tightest cases of Algorithm 1's loop: a prompt of ONE token (no earlier key to attend to),
+    a prompt whose last chunk holds one position (chunks 8, 8, 1), a prompt that fills the cache to its last slot (the
+    step after it must be refused, nothing may be written past the cache), and an empty prompt (refused)."""
+    import paper_2410_00531_b200 as P
+    shape = S.CONFIGS["C1"].with_(dtype=dtype, seed=91)
+    _run_and_compare(shape, 2, prompt_len=1, n_decode=3)
+    _run_and_compare(shape, 2, prompt_len=17, max_prefill=8, n_decode=2)
+    toks = S.prompt_tokens(shape, 24)
+    orc = make_oracle(shape)
+    want = orc.forward(toks)
+    with gpu_session(shape, 24, 24, 2) as ses:               # max_seq == prompt length
+        with pytest.raises(P.TpiError) as e:
+            P.prefill(ses.h, [], 0)
+        assert e.value.code == -1 and P.position(ses.h) == 0
+        tok, lg = P.prefill(ses.h, toks, shape.vocab)
+        check_logits(lg, tok, want, tol_for(shape))
+        k, v = P.get_kv(ses.h, shape.n_layers - 1, shape.n_kv_heads - 1, 23, 1, shape.head_dim)   # the last slot
+        assert close_elementwise(k, orc.cache.K[-1][-1][23:24], tol_for(shape))
+        assert P.position(ses.h) == 24
+        with pytest.raises(P.TpiError) as e:
+            P.decode_step(ses.h, tok, 0)
+        assert e.value.code == -4 and P.position(ses.h) == 24
+
+
 def test_small_bf16_gqa():
     shape = S.CONFIGS["C1"].with_(dtype="bf16", n_heads=8, n_kv_heads=2, head_dim=32, seed=77, rope_base=500000.0)
     _run_and_compare(shape, 2)
