@@ -29,6 +29,12 @@ constexpr int stages_for(int bn, int split) {
 // SPLIT = 1: the activations come as two bf16 tensors, A = A_hi + A_lo (A_lo = bf16(A - A_hi)), and every
 // k-block issues the MMAs twice onto the same accumulator.  That keeps ~16 mantissa bits of the fp32
 // activations while the weights stay exact bf16; the weight tile in shared memory is shared by both.
+//
+// n_acc = 2: the first and the second half of the k-blocks accumulate in two accumulators side by side in tensor
+// memory, added in fp32 in the epilogue.  The tensor core truncates its fp32 accumulator at every step (16 products),
+// so a chain drifts towards zero by about 2^-26 of the sum per step (9.3e-6 of the result at K = 4096 with the two
+// products per k-block); two half chains added with round to nearest halve that.  (Four accumulators halve it again
+// but take all of tensor memory for tiles of 160 outputs and measured 6 % slower at 128 positions.)
 template <int BN, int STAGES, int SPLIT>
 __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
                                                       const __grid_constant__ CUtensorMap tmAlo,
@@ -37,7 +43,9 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
   __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES], acc_ready;
   __shared__ uint32_t tmem_base_s;
   static_assert(BN % 32 == 0 && BN <= 256, "the epilogue reads 32 accumulator columns at a time");
-  constexpr uint32_t TCOLS = tmem_cols(BN);
+  constexpr uint32_t ACOLS = tmem_cols(BN);  // columns of one accumulator
+  const int n_acc = (a.n_acc >= 2 && a.K / kBK >= 2) ? 2 : 1;
+  const uint32_t TCOLS = ACOLS * (uint32_t)n_acc;
   constexpr uint32_t A_BYTES = kBM * kBK * 2, B_BYTES = BN * kBK * 2, STAGE_BYTES = (1 + SPLIT) * A_BYTES + B_BYTES;
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -81,21 +89,24 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
       // instruction descriptor: D fp32, A and B bf16, both K-major, N = BN, M = 128
       constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
       bool ok = true;
+      const int kb_half = n_acc == 2 ? kblocks / 2 : kblocks;  // the second accumulator takes the k-blocks from here on
       for (int kb = 0; kb < kblocks && ok; ++kb) {
         const int s = kb % STAGES;
         const uint32_t ph = (kb / STAGES) & 1;
         ok = mbar_wait(&full[s], ph, a.err, polls);
         if (!ok) break;
         tc_fence_after();
+        const uint32_t d = tmem_acc + (kb >= kb_half ? ACOLS : 0u);
+        const bool first = kb == 0 || kb == kb_half;
         const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
         const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sa + (1 + SPLIT) * A_BYTES);
 #pragma unroll
         for (int k = 0; k < kBK / 16; ++k)  // 16 bf16 = 32 bytes per step inside the swizzle atom
-          umma_bf16(tmem_acc, da + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
+          umma_bf16(d, da + 2 * k, db + 2 * k, idesc, (!first || k) ? 1u : 0u);
         if (SPLIT) {
           const uint64_t dl = umma_desc_sw128(sa + A_BYTES);
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k) umma_bf16(tmem_acc, dl + 2 * k, db + 2 * k, idesc, 1u);
+          for (int k = 0; k < kBK / 16; ++k) umma_bf16(d, dl + 2 * k, db + 2 * k, idesc, 1u);
         }
         umma_commit(&empty[s]);  // the stage is free once these MMAs have read it
       }
@@ -113,7 +124,16 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         uint32_t r[32];
-        tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+        if (n_acc == 2) {  // both halves of the contraction: two loads in flight, one wait, first half + second half
+          uint32_t r2[32];
+          tmem_ld32_nowait(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+          tmem_ld32_nowait(tmem_acc + ((uint32_t)(q * 32) << 16) + ACOLS + (uint32_t)c0, r2);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r2[i]));
+        } else {
+          tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+        }
         if (row < a.T && a.act) {
           __nv_bfloat16* arow = a.act + (size_t)row * a.act_ld + ((n0 + c0) >> 1);
           uint32_t hi[8], lo[8];
@@ -253,8 +273,11 @@ static cudaError_t launch_gemm_tc_any(const LaunchCtx& c, const void* A_bf16, co
   if (!make_map(&tmAlo, A_lo_bf16 ? A_lo_bf16 : A_bf16, (uint64_t)lda, (uint64_t)T, (uint64_t)lda, kBM)) return cudaErrorInvalidValue;
   const uint64_t w_rows = (uint64_t)(n_batch - 1) * w_row_batch + n_out;
   if (!make_map(&tmW, W_bf16, (uint64_t)K, w_rows, (uint64_t)K, (uint32_t)BN)) return cudaErrorInvalidValue;
+  // up to 128 positions no other kernel computes the same outputs, and the contraction is spread over two accumulators
+  // whatever the tile width (so the bits do not depend on it); beyond, the single chain that the CTA-pair kernels
+  // and the star sum in their epilogue reproduce
   GemmTcArgs a{Y, y_batch_stride, ldy, T, n_out, K, a_col_batch, w_row_batch, err, (__nv_bfloat16*)act, act_lo_off, act_ld, act_split,
-               wait_polls, starve};
+               wait_polls, starve, T <= kBM ? 2 : 1};
 #define TPI_TC(BNV) \
   return A_lo_bf16 ? launch_tc_t<BNV, stages_for(BNV, 1), 1>(c, tmA, tmAlo, tmW, a, n_batch) \
                    : launch_tc_t<BNV, stages_for(BNV, 0), 0>(c, tmA, tmAlo, tmW, a, n_batch)

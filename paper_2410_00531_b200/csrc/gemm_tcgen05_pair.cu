@@ -501,7 +501,7 @@ cudaError_t launch_gemm_tc_pair(const LaunchCtx& c, int shape, const void* A_bf1
                                 int K, int n_batch, int* err, void* act, int act_ld, long long act_lo_off, int act_split) {
   if (shape < 0 || shape >= kNumShapes || !A_lo_bf16) return cudaErrorInvalidValue;
   const uint64_t w_rows = (uint64_t)(n_batch - 1) * w_row_batch + n_out;
-  GemmTcArgs a{Y, y_batch_stride, ldy, T, n_out, K, a_col_batch, w_row_batch, err, (__nv_bfloat16*)act, act_lo_off, act_ld, act_split};
+  GemmTcArgs a{Y, y_batch_stride, ldy, T, n_out, K, a_col_batch, w_row_batch, err, (__nv_bfloat16*)act, act_lo_off, act_ld, act_split, 0, 0, 1};
   switch (shape) {
     case 0: return launch_pair_t<128, 1>(c, A_bf16, A_lo_bf16, lda, W_bf16, w_rows, a, n_batch);
     case 1: return launch_pair_t<192, 1>(c, A_bf16, A_lo_bf16, lda, W_bf16, w_rows, a, n_batch);
