@@ -1,6 +1,6 @@
 """Writes tests/golden/<workload>_full_depth.txt: what the CPU oracle computes for a workload at FULL depth on its seeded
-prompt.  Calls only the oracle and the seeded input generator; takes minutes to a quarter of an hour and up to ~25 GB of
-memory (weights are generated layer by layer and dropped again).
+prompt.  Calls only the oracle and the seeded input generator; on 8 cores C2 takes ~4 minutes, C3 ~30 minutes, C5 ~1 hour,
+with up to ~25 GB of memory (weights are generated layer by layer and dropped again).
 
     python tests/golden/make_full_depth_golden.py            # C2: 7B shape, 128-token prompt
     python tests/golden/make_full_depth_golden.py C3         # 8B shape, its 4096-token prompt
