@@ -340,6 +340,40 @@ def test_gemm_tensor_core_bf16(T, Tn, K, n_out, nb, split):
         assert rel_l2(got, want) < 3e-6
 
 
+def test_tensor_core_accumulator_drift_and_what_the_chunks_do_about_it(T):
+    """Why long contractions are accumulated in pieces: the tensor core truncates its fp32 accumulator at every step, so
+    a long chain comes out too SMALL in magnitude (a systematic bias, not noise).  A batch of 2 forces the one-chain
+    form at 300 positions: at K = 8192 its result is biased towards zero by about 1.6e-5 of the mean magnitude; the
+    single batch at the same size runs in 512-input chunks and is ten times closer to the exact product of the same
+    bf16 values; at 128 positions the two half chains sit in between."""
+    import paper_2410_00531_b200.ops as KK
+    rng = np.random.default_rng(5)
+    K, n_out = 8192, 512
+    err = T.zeros(1, dtype=T.int32, device="cuda")
+
+    def run(Tn, nb):
+        A32 = rng.standard_normal((Tn, nb * K)).astype(np.float32)
+        A = S.f32_to_bf16_bits(A32).reshape(Tn, nb * K)
+        Alo = S.f32_to_bf16_bits(A32 - S.bf16_bits_to_f32(A).reshape(A32.shape)).reshape(Tn, nb * K)
+        W = S.f32_to_bf16_bits((rng.standard_normal((nb, n_out, K)) * 0.02).astype(np.float32)).reshape(nb, n_out, K)
+        Y = T.zeros((nb, Tn, n_out), dtype=T.float32, device="cuda")
+        KK.gemm_bf16(dev(T, A).data_ptr(), nb * K, K, dev(T, W).data_ptr(), n_out, Y.data_ptr(), Tn * n_out, n_out,
+                     Tn, n_out, K, nb, err.data_ptr(), A_lo=dev(T, Alo).data_ptr())
+        T.cuda.synchronize()
+        assert int(err[0]) == 0
+        A64, W64 = S.as_f64(A) + S.as_f64(Alo), S.as_f64(W)
+        want = np.stack([A64[:, b * K:(b + 1) * K] @ W64[b].T for b in range(nb)])
+        d = Y.cpu().numpy().astype(np.float64) - want
+        return rel_l2(Y.cpu().numpy(), want), float((d * np.sign(want)).mean() / np.abs(want).mean())
+
+    one_chain, bias = run(300, 2)
+    assert 1e-5 < one_chain < 3e-5 and -3e-5 < bias < -1e-5, (one_chain, bias)
+    chunked, bias_c = run(300, 1)
+    assert chunked < 2e-6 and abs(bias_c) < 2e-6, (chunked, bias_c)
+    halves, bias_h = run(128, 1)
+    assert chunked < halves < one_chain and bias_h < 0, (halves, bias_h)
+
+
 @pytest.mark.parametrize("shape", [0, 1, 2, 3])
 @pytest.mark.parametrize("Tn,K,n_out,nb", [(300, 1024, 1000, 2), (513, 192, 2048, 1)])
 def test_gemm_tensor_core_pair_shapes(T, monkeypatch, shape, Tn, K, n_out, nb):
