@@ -258,6 +258,7 @@ struct RowSumArgs {
   __nv_bfloat16* act;
   long long act_lo_off;
   int act_ld, act_split;
+  int band;         // position-pair tiles per band (0: one band): the pairs sweep the column tiles band by band
 };
 
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
@@ -283,7 +284,23 @@ __global__ void __launch_bounds__(RS_THREADS) gemm_tc_pair_rowsum_kernel(const _
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();  // 0 = leader
-  const int n0 = blockIdx.y * RS_BN, m0 = (blockIdx.x >> 1) * 2 * kMH + (int)rank * kMH;  // position tiles run fastest
+  // Order of the pairs' tiles: position tiles run fastest inside a band of `band` position tiles, then the column
+  // tiles of that band, then the next band: the pairs in flight share a few weight tiles, and a band's activations
+  // (not the whole chunk's) are what has to stay in L2 while the column tiles sweep over them.
+  int pt = (int)(blockIdx.x >> 1), ct = (int)blockIdx.y;
+  if (a.band > 0) {
+    const int PT = (int)(gridDim.x >> 1), NCT = (int)gridDim.y;
+    const long long L = (long long)ct * PT + pt;
+    const int full = PT / a.band;                       // bands of the full height; the rest forms a last, lower band
+    const long long per_band = (long long)a.band * NCT;
+    int b = (int)(L / per_band);
+    if (b >= full) b = full;
+    const long long rem = L - (long long)b * per_band;
+    const int hb = b < full ? a.band : PT - full * a.band;  // height of this band
+    ct = (int)(rem / hb);
+    pt = b * a.band + (int)(rem % hb);
+  }
+  const int n0 = ct * RS_BN, m0 = pt * 2 * kMH + (int)rank * kMH;
   const int kblocks = a.K / kBK;  // per shard
 
   if (threadIdx.x == 0) {
@@ -519,6 +536,21 @@ bool gemm_tc_rowsum_supported(int T, int K, int a_cols_total, int n_out, int ldx
 static cudaError_t launch_rowsum_args(const LaunchCtx& c, const void* A_bf16, const void* A_lo_bf16, int lda, const void* W_bf16,
                                       uint64_t w_cols, uint64_t w_rows, const RowSumArgs& a);
 
+// Band height of the tile order, in position tiles of 256 (see the kernel).  With P position tiles and C column tiles
+// in flight at once the pairs pull P activation tiles and C weight tiles per k-block, P * C = the 74 pairs of the
+// machine: position tiles fastest over ALL positions (P = 16 at 4096 positions, 32 at 8192) is far from the balance
+// P ~ C; 4 measured best (8B shape, 4096-token prompt: TTFT 109.6 -> 107.9 ms; 70B shape, 8192 tokens: 2.03 -> 1.91 s;
+// 8 within noise of it, 2 in between).
+static int band_tiles() {
+  static int band = -1;
+  if (band < 0) {
+    const char* e = getenv("TPI_GEMM_BAND");  // development aid: 0 = one band (position tiles fastest over the whole chunk)
+    band = e ? atoi(e) : 4;
+    if (band < 0) band = 4;
+  }
+  return band;
+}
+
 int gemm_tc_chunk_len() {
   static int len = -1;
   if (len < 0) {
@@ -543,7 +575,7 @@ cudaError_t launch_gemm_tc_rowsum(const LaunchCtx& c, const void* A_bf16, const 
                                   const void* W_bf16, int w_row_batch, float* X, int ldx, int T, int n_out, int K, int n_shards,
                                   int* err) {
   if (!A_lo_bf16 || n_shards < 1) return cudaErrorInvalidValue;
-  RowSumArgs a{X, ldx, T, n_out, K, n_shards, a_col_batch, w_row_batch, err, 1, K / kBK, 0, nullptr, 0, 0, 0};  // one chain per shard
+  RowSumArgs a{X, ldx, T, n_out, K, n_shards, a_col_batch, w_row_batch, err, 1, K / kBK, 0, nullptr, 0, 0, 0, band_tiles()};  // one chain per shard
   return launch_rowsum_args(c, A_bf16, A_lo_bf16, lda, W_bf16, (uint64_t)K, (uint64_t)(n_shards - 1) * w_row_batch + n_out, a);
 }
 
@@ -559,7 +591,7 @@ cudaError_t launch_gemm_tc_chunked(const LaunchCtx& c, const void* A_bf16, const
   if (!A_lo_bf16) return cudaErrorInvalidValue;
   int chunks, kb_chunk;
   chunking(K, &chunks, &kb_chunk);
-  RowSumArgs a{Y, ldy, T, n_out, K, 1, 0, 0, err, chunks, kb_chunk, act ? 2 : 1, (__nv_bfloat16*)act, act_lo_off, act_ld, act_split};
+  RowSumArgs a{Y, ldy, T, n_out, K, 1, 0, 0, err, chunks, kb_chunk, act ? 2 : 1, (__nv_bfloat16*)act, act_lo_off, act_ld, act_split, band_tiles()};
   return launch_rowsum_args(c, A_bf16, A_lo_bf16, lda, W_bf16, (uint64_t)K, (uint64_t)n_out, a);
 }
 
