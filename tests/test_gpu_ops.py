@@ -309,7 +309,7 @@ def test_rowshard_fused_is_bit_identical_to_partials_then_sum(T, cfg, n_shards, 
 
 @pytest.mark.parametrize("Tn,K,n_out,nb", [(128, 4096, 12288, 1), (100, 4096, 1024, 1), (300, 1024, 4096, 4),
                                            (128, 2752, 4096, 4), (37, 64, 200, 2), (512, 3584, 640, 8),
-                                           (300, 4160, 1000, 1), (513, 8192, 2048, 1)])
+                                           (300, 4160, 1000, 1), (513, 8192, 2048, 1), (1400, 1024, 768, 1)])
 @pytest.mark.parametrize("split", [False, True])
 def test_gemm_tensor_core_bf16(T, Tn, K, n_out, nb, split):
     """Prompt-pass projection on tcgen05: bf16 inputs, fp32 accumulation, against fp64 on the same
@@ -400,7 +400,8 @@ def test_gemm_tensor_core_pair_shapes(T, monkeypatch, shape, Tn, K, n_out, nb):
     assert rel_l2(got[:nb * Tn * n_out].reshape(nb, Tn, n_out), want) < 2e-5
 
 
-@pytest.mark.parametrize("Tn,K,n_out,nb", [(300, 512, 1000, 4), (513, 192, 4096, 8), (129, 64, 260, 1), (1024, 1792, 512, 3)])
+@pytest.mark.parametrize("Tn,K,n_out,nb", [(300, 512, 1000, 4), (513, 192, 4096, 8), (129, 64, 260, 1), (1024, 1792, 512, 3),
+                                           (1700, 256, 1024, 2)])   # 7 position tiles: a band of 4 and a lower last band of 3
 def test_gemm_rowsum_star_sum_in_epilogue(T, Tn, K, n_out, nb):
     """Row-sharded projection with the star sum and shortcut in the GEMM's epilogue (Eq. 1-2 for T positions): against
     fp64, and bit for bit against the two-kernel path (partial sums in memory, then the rank-ordered sum)."""
