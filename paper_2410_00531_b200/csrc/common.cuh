@@ -65,13 +65,17 @@ struct Elem;
 template <>
 struct Elem<float> {
   static constexpr int VEC = 4;
-  static __device__ __forceinline__ float dot(uint4 w, const float* x, float acc) {
+  // fp32 weights are held to 1e-5 against an fp64 oracle over a whole network: a lane's running sum over hundreds of
+  // products would alone lose ~1e-6 per projection.  The four products of one vector are summed in fp32 and the
+  // vectors in fp64 (free in a kernel that waits for HBM); the result is rounded to fp32 once, after the warp's sum.
+  using Acc = double;
+  static __device__ __forceinline__ double dot(uint4 w, const float* x, double acc) {
     const float4 a = *reinterpret_cast<const float4*>(x);
-    acc = fmaf(__uint_as_float(w.x), a.x, acc);
-    acc = fmaf(__uint_as_float(w.y), a.y, acc);
-    acc = fmaf(__uint_as_float(w.z), a.z, acc);
-    acc = fmaf(__uint_as_float(w.w), a.w, acc);
-    return acc;
+    float p = __uint_as_float(w.x) * a.x;
+    p = fmaf(__uint_as_float(w.y), a.y, p);
+    p = fmaf(__uint_as_float(w.z), a.z, p);
+    p = fmaf(__uint_as_float(w.w), a.w, p);
+    return acc + (double)p;
   }
   static __device__ __forceinline__ void unpack(uint4 w, float* f) {
     f[0] = __uint_as_float(w.x); f[1] = __uint_as_float(w.y);
@@ -83,6 +87,7 @@ struct Elem<float> {
 template <>
 struct Elem<__nv_bfloat16> {
   static constexpr int VEC = 8;
+  using Acc = float;
   static __device__ __forceinline__ float dot(uint4 w, const float* x, float acc) {
     const float4 a = *reinterpret_cast<const float4*>(x);
     const float4 b = *reinterpret_cast<const float4*>(x + 4);
@@ -110,6 +115,12 @@ __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
   return v;
+}
+// the same tree in fp64, rounded to fp32 at the end (the fp32-weight GEMVs)
+__device__ __forceinline__ float warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return (float)v;
 }
 
 // Sum over a block in a fixed order (warp trees, then warp 0 over the per-warp sums).

@@ -69,6 +69,9 @@ __device__ __forceinline__ void warp_dot(const uint4* const (&wp)[R], int v0, co
                                          int lane, float (&acc)[R]) {
   constexpr int VEC = Elem<WT>::VEC;
   constexpr int U = 4;
+  typename Elem<WT>::Acc a[R];  // fp32 weights: the vectors' partial sums are added in fp64 (see Elem<float>)
+#pragma unroll
+  for (int r = 0; r < R; ++r) a[r] = acc[r];
   int v = lane;
   for (; v + 32 * (U - 1) < nvec; v += 32 * U) {
     uint4 w[U][R];
@@ -79,7 +82,7 @@ __device__ __forceinline__ void warp_dot(const uint4* const (&wp)[R], int v0, co
 #pragma unroll
     for (int u = 0; u < U; ++u)
 #pragma unroll
-      for (int r = 0; r < R; ++r) acc[r] = Elem<WT>::dot(w[u][r], xs + (v + 32 * u) * VEC, acc[r]);
+      for (int r = 0; r < R; ++r) a[r] = Elem<WT>::dot(w[u][r], xs + (v + 32 * u) * VEC, a[r]);
   }
   if (v < nvec) {  // ragged tail: one more batch with the out-of-range loads masked, still issued together
     uint4 w[U][R];
@@ -92,9 +95,11 @@ __device__ __forceinline__ void warp_dot(const uint4* const (&wp)[R], int v0, co
     for (int u = 0; u < U; ++u)
       if (v + 32 * u < nvec) {
 #pragma unroll
-        for (int r = 0; r < R; ++r) acc[r] = Elem<WT>::dot(w[u][r], xs + (v + 32 * u) * VEC, acc[r]);
+        for (int r = 0; r < R; ++r) a[r] = Elem<WT>::dot(w[u][r], xs + (v + 32 * u) * VEC, a[r]);
       }
   }
+#pragma unroll
+  for (int r = 0; r < R; ++r) acc[r] = (float)a[r];
 }
 
 // -------------------------------------------------------------------------------------
@@ -351,11 +356,11 @@ __device__ __forceinline__ void rowfused_body(const RowFusedArgs& A, float* xs, 
       // Every shard's slice of these rows is requested in the same batch (NS * R * U 16-byte loads
       // per lane in flight); each shard keeps its own accumulator, so the partial sums stay per device.
       constexpr int U = (8 / (NS * R)) > 0 ? (8 / (NS * R)) : 1;
-      float acc[NS][R];
+      typename Elem<WT>::Acc acc[NS][R];
 #pragma unroll
       for (int sh = 0; sh < NS; ++sh)
 #pragma unroll
-        for (int r = 0; r < R; ++r) acc[sh][r] = 0.f;
+        for (int r = 0; r < R; ++r) acc[sh][r] = 0;
       const uint4* base = reinterpret_cast<const uint4*>(Wall + (size_t)row0 * A.Ks);
       const size_t sstride = (size_t)A.shard_stride / VEC, rstride = (size_t)nvec;
       for (int v = lane; v < nvec; v += 32 * U) {
@@ -380,9 +385,9 @@ __device__ __forceinline__ void rowfused_body(const RowFusedArgs& A, float* xs, 
       }
 #pragma unroll
       for (int r = 0; r < R; ++r) {
-        sum[r] = warp_sum(acc[0][r]);                               // the master's own partial sum
+        sum[r] = warp_sum((float)acc[0][r]);                               // the master's own partial sum
 #pragma unroll
-        for (int sh = 1; sh < NS; ++sh) sum[r] += warp_sum(acc[sh][r]);  // + workers', in rank order
+        for (int sh = 1; sh < NS; ++sh) sum[r] += warp_sum((float)acc[sh][r]);  // + workers', in rank order
       }
     } else {
 #pragma unroll

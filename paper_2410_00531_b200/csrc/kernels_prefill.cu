@@ -221,22 +221,25 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const float* __restrict_
   W += (size_t)blockIdx.z * wbs;
   Y += (size_t)blockIdx.z * ybs;
   const int lrow = tid >> 2, lk = (tid & 3) * 4;
-  // Two-level accumulation: products are added into `acc` for 512 consecutive k, then `acc` is folded into `tot`.
-  // A single fp32 running sum over K = 8192 terms loses ~2e-6 of relative accuracy per projection, too close to the
-  // 1e-5 bar that fp32 models are held to over a whole network; with the fold it stays below 1e-6.
-  constexpr int FOLD = 512;
-  float acc[4][4], tot[4][4];
+  // Two-level accumulation: products are added into `acc` (fp32) for 64 consecutive k, then `acc` is folded into
+  // `tot` (fp64).  A single fp32 running sum over K = 8192 terms loses ~2e-6 of relative accuracy per projection, too
+  // close to the 1e-5 bar that fp32 models are held to over a whole network (an fp32 fold every 512: 1e-6, which over
+  // 16 layers of the 70B widths still added up to the whole bar); with 64-term chains and an fp64 total it is ~3e-7,
+  // for one conversion and one fp64 add per 64 products.
+  constexpr int FOLD = 64;
+  float acc[4][4];
+  double tot[4][4];
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = tot[i][j] = 0.f;
+    for (int j = 0; j < 4; ++j) { acc[i][j] = 0.f; tot[i][j] = 0.0; }
 
   for (int k0 = 0; k0 < K; k0 += BK) {
     if (k0 && k0 % FOLD == 0) {
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) { tot[i][j] += acc[i][j]; acc[i][j] = 0.f; }
+        for (int j = 0; j < 4; ++j) { tot[i][j] += (double)acc[i][j]; acc[i][j] = 0.f; }
     }
     float xv[4] = {0.f, 0.f, 0.f, 0.f}, wv[4] = {0.f, 0.f, 0.f, 0.f};
     if (m0 + lrow < T && k0 + lk < K) {
@@ -275,22 +278,22 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const float* __restrict_
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int n = n0 + tx * 4 + j;
-      if (n < n_out) Y[(size_t)m * ldy + n] = tot[i][j] + acc[i][j];
+      if (n < n_out) Y[(size_t)m * ldy + n] = (float)(tot[i][j] + (double)acc[i][j]);
     }
   }
 }
 
 // The same contraction on 128 x 64 tiles for more than 64 positions: 8 x 4 outputs per thread, the next 16-deep slice
 // in flight (registers) while the current one is multiplied.  Every output is still ONE thread's running sum over k in
-// ascending order with the fold every 512, so the bits equal the 64 x 64 kernel's.
+// ascending order with the fold (into an fp64 total) every 64, so the bits equal the 64 x 64 kernel's.
 template <typename WT>
-__global__ void __launch_bounds__(256) gemm_simt_wide_kernel(const float* __restrict__ X, long long xbs, int ldx,
+__global__ void __launch_bounds__(256, 2) gemm_simt_wide_kernel(const float* __restrict__ X, long long xbs, int ldx,
                                                              const WT* __restrict__ W, long long wbs,
                                                              float* __restrict__ Y, long long ybs, int ldy, int T,
                                                              int n_out, int K) {
   pdl_launch_dependents();
   pdl_wait();  // inputs come from the previous kernel in the stream
-  constexpr int BM = 128, BN = 64, BK = 16, FOLD = 512;
+  constexpr int BM = 128, BN = 64, BK = 16, FOLD = 64;
   __shared__ __align__(16) float Xs[2][BK][BM + 4];
   __shared__ __align__(16) float Ws[2][BK][BN + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;  // thread: rows ty*4 + {0..3} and 64 + ty*4 + {0..3}, cols tx*4 + {0..3}
@@ -299,11 +302,14 @@ __global__ void __launch_bounds__(256) gemm_simt_wide_kernel(const float* __rest
   W += (size_t)blockIdx.z * wbs;
   Y += (size_t)blockIdx.z * ybs;
   const int lrow = tid >> 2, lk = (tid & 3) * 4;  // loader: rows lrow and lrow + 64 of X, row lrow of W, 4 consecutive k
-  float acc[8][4], tot[8][4];
+  // The fp64 totals live in shared memory (slot [output][thread]: no two threads share one, no barrier needed, no bank
+  // conflict); in registers they would take the kernel from two CTAs per SM to one.
+  extern __shared__ double tot_s[];  // [32][256]
+  float acc[8][4];
 #pragma unroll
   for (int i = 0; i < 8; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = tot[i][j] = 0.f;
+    for (int j = 0; j < 4; ++j) { acc[i][j] = 0.f; tot_s[(i * 4 + j) * 256 + tid] = 0.0; }
   float4 xa, xb, wv;
   auto fetch = [&](int k0) {
     xa = xb = wv = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -335,7 +341,7 @@ __global__ void __launch_bounds__(256) gemm_simt_wide_kernel(const float* __rest
 #pragma unroll
       for (int i = 0; i < 8; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) { tot[i][j] += acc[i][j]; acc[i][j] = 0.f; }
+        for (int j = 0; j < 4; ++j) { tot_s[(i * 4 + j) * 256 + tid] += (double)acc[i][j]; acc[i][j] = 0.f; }
     }
     const bool more = k0 + BK < K;
     if (more) fetch(k0 + BK);  // in flight while this slice is multiplied
@@ -363,7 +369,7 @@ __global__ void __launch_bounds__(256) gemm_simt_wide_kernel(const float* __rest
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int n = n0 + tx * 4 + j;
-      if (n < n_out) Y[(size_t)m * ldy + n] = tot[i][j] + acc[i][j];
+      if (n < n_out) Y[(size_t)m * ldy + n] = (float)(tot_s[(i * 4 + j) * 256 + tid] + (double)acc[i][j]);
     }
   }
 }
@@ -374,10 +380,18 @@ cudaError_t launch_gemm_simt(const LaunchCtx& c, int dt, const float* X, long lo
   LaunchCtx nc = c;  // PDL allowed: every kernel below waits on its predecessor before touching memory
   if (T > 64) {
     dim3 gridw((n_out + 63) / 64, (T + 127) / 128, n_batch);
+    constexpr size_t tot_bytes = 32 * 256 * sizeof(double);  // the fp64 totals, one slot per output and thread
+    static PerDeviceOnce attr_done;
+    if (!attr_done.get()) {
+      cudaError_t e = cudaFuncSetAttribute(gemm_simt_wide_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tot_bytes);
+      if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_simt_wide_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tot_bytes);
+      if (e != cudaSuccess) return e;
+      attr_done.set();
+    }
     if (dt == DT_BF16)
-      return launch_kernel(nc, gemm_simt_wide_kernel<__nv_bfloat16>, gridw, dim3(256), 0, X, x_batch_stride, ldx,
+      return launch_kernel(nc, gemm_simt_wide_kernel<__nv_bfloat16>, gridw, dim3(256), tot_bytes, X, x_batch_stride, ldx,
                            (const __nv_bfloat16*)W, w_batch_stride_elems, Y, y_batch_stride, ldy, T, n_out, K);
-    return launch_kernel(nc, gemm_simt_wide_kernel<float>, gridw, dim3(256), 0, X, x_batch_stride, ldx, (const float*)W,
+    return launch_kernel(nc, gemm_simt_wide_kernel<float>, gridw, dim3(256), tot_bytes, X, x_batch_stride, ldx, (const float*)W,
                          w_batch_stride_elems, Y, y_batch_stride, ldy, T, n_out, K);
   }
   dim3 grid((n_out + 63) / 64, (T + 63) / 64, n_batch);
